@@ -1,0 +1,272 @@
+"""CPU oracle for the Parallel Track (PT) transformer forward pass.  TEST INFRASTRUCTURE.
+
+A plain, slow, float64 NumPy statement of what the PT forward computes, written
+from the paper's Algorithm 1 ("Track Parallelism for PT Transformer", Section 2.2)
+and the layer recipe of the workloads (pre-norm RMSNorm with eps inside the square
+root, rotary embedding on half-split pairs, causal softmax attention with grouped
+KV heads, SwiGLU feed-forward, no biases).  It exists only to check the CUDA path:
+only tests, the smoke check and the CPU-baseline leg of the benchmark may import
+it, and it shares no code with the CUDA path.
+
+Every function below is pinned by the CPU tests to something other than itself
+(closed forms, library routines, an independently written single-track decoder,
+invariants of Algorithm 1, brute-force page enumeration); no function here is
+"parity unpinned".  Declared conventions that nothing in the paper fixes (any
+consistent choice is valid): rotary pairs are (j, j + dh/2); query head i reads
+KV head i // G; the all-reduce of Algorithm 1 is a SUM (MEAN is available as an
+option); "Set h_i = h" of Algorithm 1 is read as inside the if-block (its own
+comment says it follows the all-reduce).
+
+Shapes: T tracks, L layers, D track-block depth, H per-track hidden, nq / nkv
+query / KV heads per track, dh = H / nq, G = nq / nkv, F feed-forward width.
+Weights are [out, in]; y = x @ W.T.  Positions are 0-based.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+import numpy as np
+
+
+@dataclass(frozen=True)
+class PTConfig:
+    """Architecture numbers of a PT stack (Algorithm 1's n, L, D; Table 1's per-track heads)."""
+    T: int
+    D: int
+    L: int
+    hidden: int
+    heads: int
+    kv_heads: int
+    ffn: int
+    rope_base: float = 10000.0
+    rms_eps: float = 1e-6
+    sync_op: str = "sum"          # "sum" (the all-reduce of Algorithm 1) or "mean"
+
+    def __post_init__(self):
+        if self.T < 1 or self.L < 1 or self.D < 1:
+            raise ValueError("T, L, D must be positive")
+        if self.L % self.D:
+            # Algorithm 1 returns the h of the last sync: trailing layers would be dropped.
+            raise ValueError("L must be a multiple of D")
+        if self.hidden % self.heads or self.heads % self.kv_heads:
+            raise ValueError("hidden % heads and heads % kv_heads must be 0")
+        if (self.hidden // self.heads) % 2:
+            raise ValueError("head_dim must be even for rotary pairs")
+        if self.sync_op not in ("sum", "mean"):
+            raise ValueError("sync_op")
+
+    @property
+    def head_dim(self) -> int:
+        return self.hidden // self.heads
+
+    @property
+    def group(self) -> int:
+        return self.heads // self.kv_heads
+
+
+def sync_points_pt(L: int, D: int) -> int:
+    """Number of synchronisation points of a PT stack: one per track block (Section 2.2)."""
+    return L // D
+
+
+def sync_points_tp(L: int) -> int:
+    """Tensor parallelism synchronises after attention and after the feed-forward
+    of every layer (Section 2.1)."""
+    return 2 * L
+
+
+def sync_fraction_removed(L: int, D: int) -> float:
+    """Share of tensor parallelism's sync points that PT removes (Section 2.2)."""
+    return 1.0 - sync_points_pt(L, D) / sync_points_tp(L)
+
+
+# ----------------------------------------------------------------------------- layer pieces
+
+def rmsnorm(h: np.ndarray, g: np.ndarray, eps: float) -> np.ndarray:
+    """h / sqrt(mean_k h_k^2 + eps) * g over the last axis."""
+    ms = np.mean(h * h, axis=-1, keepdims=True)
+    return h / np.sqrt(ms + eps) * g
+
+
+def rope(u: np.ndarray, pos: np.ndarray, base: float) -> np.ndarray:
+    """Rotate the pairs (j, j + dh/2) of u[..., S, heads, dh] by pos * base**(-2j/dh)."""
+    dh = u.shape[-1]
+    half = dh // 2
+    j = np.arange(half, dtype=np.float64)
+    theta = np.float64(base) ** (-2.0 * j / dh)
+    ang = np.asarray(pos, np.float64)[:, None] * theta[None, :]        # [S, half]
+    c = np.cos(ang)[:, None, :]
+    s = np.sin(ang)[:, None, :]
+    lo, hi = u[..., :half], u[..., half:]
+    return np.concatenate([lo * c - hi * s, hi * c + lo * s], axis=-1)
+
+
+def silu(z: np.ndarray) -> np.ndarray:
+    return z / (1.0 + np.exp(-z))
+
+
+def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, qpos: np.ndarray) -> np.ndarray:
+    """Causal softmax attention for one sequence of one track.
+
+    q [S, nq, dh] at absolute positions qpos[S]; k, v [N, nkv, dh] hold positions
+    0..N-1.  Query head i reads KV head i // G and sees key j iff j <= qpos.
+    Returns [S, nq, dh].
+    """
+    S, nq, dh = q.shape
+    N, nkv, _ = k.shape
+    G = nq // nkv
+    out = np.empty_like(q)
+    keypos = np.arange(N)
+    visible = keypos[None, :] <= np.asarray(qpos)[:, None]             # [S, N]
+    for i in range(nq):
+        kh, vh = k[:, i // G, :], v[:, i // G, :]
+        s = (q[:, i, :] @ kh.T) / np.sqrt(np.float64(dh))              # [S, N]
+        s = np.where(visible, s, -np.inf)
+        s = s - np.max(s, axis=-1, keepdims=True)
+        p = np.exp(s)
+        p = p / np.sum(p, axis=-1, keepdims=True)
+        out[:, i, :] = p @ vh
+    return out
+
+
+# ----------------------------------------------------------------------------- paged KV cache
+
+def kv_slot_offset(cfg: PTConfig, num_pages: int, page_size: int,
+                   t: int, l: int, page: int, kv: int, head: int, slot: int) -> int:
+    """Element offset of the first of the dh values of one cached K (kv=0) or V (kv=1)
+    vector in the pool laid out as [T][L][page][K|V][kv_head][slot][dh]."""
+    return (((((t * cfg.L + l) * num_pages + page) * 2 + kv) * cfg.kv_heads + head)
+            * page_size + slot) * cfg.head_dim
+
+
+class PagedKVCache:
+    """Per-track, per-layer paged KV cache with a host page allocator.
+
+    The pool is one float64 array indexed exactly like ``kv_slot_offset``.  Pages
+    are handed out from the front of a free list (ascending page ids unless
+    ``free_order`` gives another order); one page id serves every (track, layer)
+    slab of the pool.  ``block_table[seq][i]`` is the page holding positions
+    i*page_size .. (i+1)*page_size-1 of sequence ``seq``.
+    """
+
+    def __init__(self, cfg: PTConfig, num_pages: int, page_size: int = 16, free_order=None):
+        self.cfg, self.num_pages, self.page_size = cfg, num_pages, page_size
+        self.pool = np.zeros((cfg.T, cfg.L, num_pages, 2, cfg.kv_heads, page_size, cfg.head_dim))
+        order = list(range(num_pages)) if free_order is None else [int(p) for p in free_order]
+        if sorted(order) != list(range(num_pages)):
+            raise ValueError("free_order must be a permutation of the page ids")
+        self.free = order
+        self.block_table: dict[int, list[int]] = {}
+        self.length: dict[int, int] = {}
+
+    def reserve(self, seq: int, new_len: int) -> None:
+        """Make room for positions < new_len of ``seq`` (does not change its length)."""
+        table = self.block_table.setdefault(seq, [])
+        self.length.setdefault(seq, 0)
+        need = -(-new_len // self.page_size)
+        if need - len(table) > len(self.free):
+            raise MemoryError("KV cache full")
+        while len(table) < need:
+            table.append(self.free.pop(0))
+
+    def release(self, seq: int) -> None:
+        """Return a sequence's pages to the back of the free list, in table order."""
+        self.free.extend(self.block_table.pop(seq, []))
+        self.length.pop(seq, None)
+
+    def locate(self, seq: int, pos: int) -> tuple[int, int]:
+        return self.block_table[seq][pos // self.page_size], pos % self.page_size
+
+    def _pages_slots(self, seq: int, pos: np.ndarray):
+        pos = np.asarray(pos, np.int64)
+        table = np.asarray(self.block_table[seq], np.int64)
+        return table[pos // self.page_size], pos % self.page_size
+
+    def write(self, t: int, l: int, seq: int, pos: np.ndarray, k: np.ndarray, v: np.ndarray) -> None:
+        """Store k, v [n, nkv, dh] at positions pos[n] of ``seq``."""
+        pages, slots = self._pages_slots(seq, pos)
+        self.pool[t, l, pages, 0, :, slots, :] = k
+        self.pool[t, l, pages, 1, :, slots, :] = v
+
+    def gather(self, t: int, l: int, seq: int, n: int) -> tuple[np.ndarray, np.ndarray]:
+        """K and V of positions 0..n-1 as [n, nkv, dh] each."""
+        pages, slots = self._pages_slots(seq, np.arange(n))
+        return self.pool[t, l, pages, 0, :, slots, :], self.pool[t, l, pages, 1, :, slots, :]
+
+
+# ----------------------------------------------------------------------------- the PT forward
+
+def _layer(cfg: PTConfig, w: dict, h: np.ndarray, cache: PagedKVCache, t: int, l: int,
+           seq_ids, start, taps: dict | None) -> np.ndarray:
+    """One standard pre-norm transformer layer of track t on h[B, S, H]."""
+    B, S, H = h.shape
+    nq, nkv, dh = cfg.heads, cfg.kv_heads, cfg.head_dim
+    W = {k: np.asarray(a, np.float64) for k, a in w.items()}
+    a = rmsnorm(h, W["g1"], cfg.rms_eps)
+    q = (a @ W["wq"].T).reshape(B, S, nq, dh)
+    k = (a @ W["wk"].T).reshape(B, S, nkv, dh)
+    v = (a @ W["wv"].T).reshape(B, S, nkv, dh)
+    o = np.empty((B, S, nq, dh))
+    for b in range(B):
+        pos = start[b] + np.arange(S)
+        qb = rope(q[b], pos, cfg.rope_base)
+        kb = rope(k[b], pos, cfg.rope_base)
+        cache.write(t, l, seq_ids[b], pos, kb, v[b])
+        kk, vv = cache.gather(t, l, seq_ids[b], start[b] + S)
+        o[b] = attention(qb, kk, vv, pos)
+    attn_delta = o.reshape(B, S, nq * dh) @ W["wo"].T
+    h = h + attn_delta
+    c = rmsnorm(h, W["g2"], cfg.rms_eps)
+    ffn_delta = (silu(c @ W["wg"].T) * (c @ W["wu"].T)) @ W["wd"].T
+    if taps is not None:
+        taps.setdefault("attn_delta", {})[(t, l)] = attn_delta
+        taps.setdefault("ffn_delta", {})[(t, l)] = ffn_delta
+    return h + ffn_delta
+
+
+def pt_prefill(cfg: PTConfig, weights, x: np.ndarray, cache: PagedKVCache, seq_ids,
+               taps: dict | None = None) -> np.ndarray:
+    """Algorithm 1 on x[T, B, S, H]; returns h[B, S, H].
+
+    ``weights.get(t, l)`` gives the weight dict of track t, layer l (0-based).  The
+    S tokens of batch row b are appended to sequence seq_ids[b] after the tokens it
+    already holds.  ``x[t]`` is track t's starting state (Algorithm 1 uses the same
+    x for every track; pass T equal slices for that case).  If ``taps`` is a dict it
+    receives ``taps["h"][l]`` = the [T, B, S, H] residual stream after layer l
+    (after the sync when l closes a track block) and the per-layer deltas.
+    """
+    x = np.asarray(x, np.float64)
+    T, B, S, H = x.shape
+    assert T == cfg.T and H == cfg.hidden and len(seq_ids) == B
+    start = []
+    for b in range(B):
+        cache.reserve(seq_ids[b], cache.length.get(seq_ids[b], 0) + S)
+        start.append(cache.length[seq_ids[b]])
+    h = [x[t].copy() for t in range(T)]                       # Set h_i = x
+    syncs = 0
+    for l in range(cfg.L):                                    # for each layer
+        for t in range(T):                                    # every track, independently
+            h[t] = _layer(cfg, weights.get(t, l), h[t], cache, t, l, seq_ids, start, taps)
+        if (l + 1) % cfg.D == 0:                              # one sync point per track block
+            total = h[0].copy()
+            for t in range(1, T):
+                total = total + h[t]                          # all-reduce (sum)
+            if cfg.sync_op == "mean":
+                total = total / T
+            h = [total.copy() for _ in range(T)]              # every track continues from h
+            syncs += 1
+        if taps is not None:
+            taps.setdefault("h", {})[l] = np.stack(h)
+    for b in range(B):
+        cache.length[seq_ids[b]] = start[b] + S
+    if taps is not None:
+        taps["syncs"] = syncs
+    assert syncs == sync_points_pt(cfg.L, cfg.D)
+    return h[0]
+
+
+def pt_decode_step(cfg: PTConfig, weights, x: np.ndarray, cache: PagedKVCache, seq_ids,
+                   taps: dict | None = None) -> np.ndarray:
+    """One new token per sequence: x[T, B, H] -> h[B, H].  The token of row b is
+    written at position length[seq] and attends positions 0..length[seq]."""
+    x = np.asarray(x, np.float64)
+    return pt_prefill(cfg, weights, x[:, :, None, :], cache, seq_ids, taps)[:, 0, :]
