@@ -1,0 +1,128 @@
+// Internal declarations shared by the translation units of libpt.so.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <cuda.h>
+
+#include <atomic>
+#include <cstdint>
+#include <cstdio>
+#include <deque>
+#include <unordered_map>
+#include <vector>
+
+#include "pt.h"
+
+namespace pt {
+
+constexpr int kStatusWords = 16;          // device status word block (int32 each)
+constexpr int kSsqTile = 128;             // columns covered by one partial sum of squares
+
+// Location codes written next to PT_ERR_DEVICE_* in the status block.
+enum : int {
+    LOC_ROPE_PAGE = 1, LOC_ATTN_PAGE = 2, LOC_GEMM_TMA_WAIT = 3, LOC_GEMM_MMA_WAIT = 4,
+    LOC_GEMM_EPI_WAIT = 5, LOC_GEMM_EMPTY_WAIT = 6, LOC_DECODE_PAGE = 7, LOC_FLASH_PAGE = 8,
+    LOC_GEMM_ACC_WAIT = 9,
+};
+
+extern std::atomic<long long> g_launches;
+void set_error(const char* fmt, ...);
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Seq {
+    std::vector<int32_t> pages;
+    int32_t len = 0;
+};
+
+}  // namespace pt
+
+struct pt_model {
+    pt_config cfg;
+    int dh, G, QD, KVD, Nqkv;             // head_dim, heads/kv_heads, nq*dh, nkv*dh, QD+2*KVD
+    size_t esz;                           // bytes per element of the model dtype
+    bool tc;                              // bf16 tensor-core path (else SIMT)
+    // byte offsets inside the bound weight buffer; matrices are [L][T][rows][cols]
+    size_t off_wqkv, off_wo, off_wgu, off_wd, off_g1, off_g2, off_cos, off_sin, off_status, total_bytes;
+    char* wbuf = nullptr;
+    int tap_layer = -2;
+    float* tap_buf = nullptr;
+    std::vector<char> meta_host;          // staging for the per-call metadata upload
+    // TMA descriptors of the packed weights (tensor-core path), built at bind time
+    CUtensorMap tm_wqkv, tm_wo, tm_wgu, tm_wd;
+
+    size_t wqkv_layer() const { return (size_t)cfg.T * Nqkv * cfg.hidden; }     // elements
+    size_t wo_layer() const { return (size_t)cfg.T * cfg.hidden * QD; }
+    size_t wgu_layer() const { return (size_t)cfg.T * 2 * cfg.ffn * cfg.hidden; }
+    size_t wd_layer() const { return (size_t)cfg.T * cfg.hidden * cfg.ffn; }
+    int* status() const { return (int*)(wbuf + off_status); }
+    const float* gain(int which, int l) const {
+        return (const float*)(wbuf + (which ? off_g2 : off_g1)) + (size_t)l * cfg.T * cfg.hidden;
+    }
+    const float* rope_cos() const { return (const float*)(wbuf + off_cos); }
+    const float* rope_sin() const { return (const float*)(wbuf + off_sin); }
+};
+
+struct pt_kv_cache {
+    const pt_model* m;
+    int32_t num_pages, ps;
+    char* pool;
+    size_t bytes;
+    int64_t page_elems;                   // 2 * nkv * ps * dh
+    int64_t slab_elems;                   // num_pages * page_elems : one (track, layer)
+    std::deque<int32_t> free_list;
+    std::unordered_map<int32_t, pt::Seq> seqs;
+};
+
+namespace pt {
+
+// Per-call device metadata (lives at the head of the workspace).
+struct Meta {
+    const int64_t* row_kvoff;   // [M] element offset, inside a (track, layer) slab, of K head 0 of the row's slot
+    const int32_t* row_pos;     // [M] absolute position of the row's token
+    const int32_t* row_b;       // [M] batch row
+    const int32_t* kvlen;       // [B] cached length including this call's tokens
+    const int32_t* bt;          // [B][maxp] block table rows
+    int32_t maxp;
+};
+
+// Workspace carve-up for one call.
+struct Work {
+    Meta meta;
+    float* hT;      // [T][M][H] per-track residual stream
+    float* hS;      // [M][H] post-sync stream (read with track stride 0)
+    void* a;        // [T][M][H] model dtype: normalised activations (SIMT) / gain-scaled bf16 stream (tc)
+    void* qkv;      // [T][M][Nqkv]
+    void* o;        // [T][M][QD]
+    void* gu;       // [T][M][2F] (SIMT only)
+    void* z;        // [T][M][F]
+    float* ssq;     // [T][M][H/kSsqTile] partial sums of squares (tc)
+    float* part;    // decode split-KV partials
+    size_t total;
+};
+
+struct Call {
+    pt_model* m;
+    pt_kv_cache* c;
+    int B, S, M;
+    const void* x;
+    int64_t x_stride;
+    float* out;
+    Work w;
+    cudaStream_t st;
+    bool decode;
+    // decode split plan (host): items of (b, first key, key count)
+    int n_items, max_splits;
+    const int32_t* items;     // device [n_items][4]: b, start, count, split index
+    const int32_t* nsplit;    // device [B]
+};
+
+// pt_simt.cu
+pt_status simt_forward(Call& k);
+void launch_pack(const pt_model* m, int kind, const void* src, void* dst_matrix_base, cudaStream_t st);
+
+// pt_tc.cu (bf16 tensor-core path)
+pt_status tc_build_weight_maps(pt_model* m);
+pt_status tc_forward(Call& k);
+
+}  // namespace pt

@@ -1,0 +1,289 @@
+"""Thin ctypes binding over libpt.so (see include/pt.h for the contract of every call).
+
+Only argument marshalling lives here; every step of the forward pass runs in the library's
+CUDA kernels.  PyTorch is used for device memory and streams: the ``Model`` helper owns the
+torch tensors that back the packed weights, the KV pool and the workspace, and hands their
+raw pointers to the C ABI.  Without the compiled library every call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpt.so")
+
+PT_OK = 0
+STATUS = {0: "PT_OK", 1: "PT_ERR_INVALID_ARG", 2: "PT_ERR_BAD_CONFIG", 3: "PT_ERR_UNSUPPORTED",
+          4: "PT_ERR_BUFFER_TOO_SMALL", 5: "PT_ERR_CACHE_FULL", 6: "PT_ERR_MISALIGNED", 7: "PT_ERR_CUDA",
+          8: "PT_ERR_DEVICE_BOUNDS", 9: "PT_ERR_DEVICE_TIMEOUT", 10: "PT_ERR_STATE"}
+PT_F32, PT_BF16 = 0, 1
+KIND = {"wq": 0, "wk": 1, "wv": 2, "wo": 3, "wg": 4, "wu": 5, "wd": 6, "g1": 7, "g2": 8}
+
+
+class PtError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"{STATUS.get(code, code)}: {msg}")
+        self.code = code
+
+
+class pt_config(C.Structure):
+    _fields_ = [("T", C.c_int32), ("D", C.c_int32), ("L", C.c_int32), ("hidden", C.c_int32),
+                ("heads", C.c_int32), ("kv_heads", C.c_int32), ("ffn", C.c_int32),
+                ("rope_base", C.c_float), ("rms_eps", C.c_float), ("dtype", C.c_int32),
+                ("sync_op", C.c_int32), ("max_pos", C.c_int32), ("flags", C.c_int32)]
+
+
+_P, _I32, _I64, _SZ = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
+_PROTOS = {
+    "pt_model_create": (_I32, [C.POINTER(pt_config), C.POINTER(_P)]),
+    "pt_model_destroy": (None, [_P]),
+    "pt_model_weight_bytes": (_I32, [_P, C.POINTER(_SZ)]),
+    "pt_model_bind_weights": (_I32, [_P, _P, _SZ]),
+    "pt_model_set_weight": (_I32, [_P, _I32, _I32, _I32, _P, _P]),
+    "pt_sync_count": (_I32, [_P]),
+    "pt_kv_cache_bytes": (_I32, [_P, _I32, _I32, C.POINTER(_SZ)]),
+    "pt_kv_cache_alloc": (_I32, [_P, _I32, _I32, _P, _SZ, C.POINTER(_P)]),
+    "pt_kv_cache_free": (None, [_P]),
+    "pt_kv_set_free_list": (_I32, [_P, C.POINTER(_I32), _I32]),
+    "pt_kv_seq_reserve": (_I32, [_P, _I32, _I32]),
+    "pt_kv_seq_release": (_I32, [_P, _I32]),
+    "pt_kv_seq_len": (_I32, [_P, _I32, C.POINTER(_I32)]),
+    "pt_kv_seq_truncate": (_I32, [_P, _I32, _I32]),
+    "pt_kv_block_table": (_I32, [_P, _I32, C.POINTER(_I32), _I32, C.POINTER(_I32)]),
+    "pt_kv_slot": (_I32, [_P, _I32, _I32, _I32, _I32, _I32, _I32, C.POINTER(_I64)]),
+    "pt_workspace_bytes": (_I32, [_P, _I64, _I32, _I32, C.POINTER(_SZ)]),
+    "pt_prefill": (_I32, [_P, _P, _P, _I64, _I32, _I32, C.POINTER(_I32), _P, _P, _SZ, _P]),
+    "pt_decode_step": (_I32, [_P, _P, _P, _I64, _I32, C.POINTER(_I32), _P, _P, _SZ, _P]),
+    "pt_set_debug_tap": (_I32, [_P, _I32, _P]),
+    "pt_device_status": (_I32, [_P, _P, C.POINTER(_I32), C.POINTER(_I32)]),
+    "pt_launch_count": (_I64, []),
+    "pt_last_error": (C.c_char_p, []),
+}
+EXPORTS = tuple(_PROTOS)
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load libpt.so once; raise if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2602_07306_b200.build` "
+                               "(there is no CPU fallback)")
+        l = C.CDLL(LIB_PATH)
+        for name, (res, args) in _PROTOS.items():
+            f = getattr(l, name)
+            f.restype, f.argtypes = res, args
+        _lib = l
+    return _lib
+
+
+def check(code: int) -> None:
+    if code != PT_OK:
+        raise PtError(code, lib().pt_last_error().decode())
+
+
+def _i32arr(a):
+    a = np.ascontiguousarray(a, dtype=np.int32)
+    return a, a.ctypes.data_as(C.POINTER(_I32))
+
+
+class Model:
+    """A PT model with its packed weights on one CUDA device (torch owns the memory)."""
+
+    def __init__(self, *, T, D, L, hidden, heads, kv_heads, ffn, dtype="bf16", rope_base=10000.0,
+                 rms_eps=1e-6, sync_op="sum", max_pos=4096, simt=False, device="cuda:0"):
+        import torch
+        self.torch = torch
+        self.device = torch.device(device)
+        self.cfg = pt_config(T, D, L, hidden, heads, kv_heads, ffn, rope_base, rms_eps,
+                             PT_BF16 if dtype == "bf16" else PT_F32, 1 if sync_op == "mean" else 0,
+                             max_pos, 1 if simt else 0)
+        self.dtype = dtype
+        self.tdtype = torch.bfloat16 if dtype == "bf16" else torch.float32
+        self.h = _P()
+        check(lib().pt_model_create(C.byref(self.cfg), C.byref(self.h)))
+        if not torch.cuda.is_available():
+            raise RuntimeError("a CUDA device is required: there is no CPU path")
+        n = _SZ()
+        check(lib().pt_model_weight_bytes(self.h, C.byref(n)))
+        self.weight_bytes = n.value
+        with torch.cuda.device(self.device):
+            self.wbuf = torch.empty(n.value, dtype=torch.uint8, device=self.device)
+            check(lib().pt_model_bind_weights(self.h, self.wbuf.data_ptr(), n.value))
+        self.ws = None
+        self.ws_key = (0, 0, 0)
+        self._tap = None
+
+    def close(self):
+        if self.h:
+            lib().pt_model_destroy(self.h)
+            self.h = _P()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _stream(self):
+        return self.torch.cuda.current_stream(self.device).cuda_stream
+
+    def set_weight(self, t: int, l: int, kind: str, w) -> None:
+        """w: numpy float32 array or torch tensor, [out, in] (gains: [hidden])."""
+        torch = self.torch
+        if isinstance(w, np.ndarray):
+            w = torch.from_numpy(np.ascontiguousarray(w))
+        want = torch.float32 if kind in ("g1", "g2") else self.tdtype
+        w = w.to(device=self.device, dtype=want).contiguous()
+        with torch.cuda.device(self.device):
+            check(lib().pt_model_set_weight(self.h, t, l, KIND[kind], w.data_ptr(), self._stream()))
+            torch.cuda.current_stream().synchronize()      # w may be freed after return
+
+    def load(self, source) -> None:
+        """source.get(t, l) -> dict kind -> float32 numpy array."""
+        for l in range(self.cfg.L):
+            for t in range(self.cfg.T):
+                for k, w in source.get(t, l).items():
+                    self.set_weight(t, l, k, w)
+
+    def init_random(self, seed: int = 0, std: float = 0.02) -> None:
+        """Weights N(0, std), gains 1, drawn on the device (for timing runs)."""
+        torch = self.torch
+        c = self.cfg
+        dh = c.hidden // c.heads
+        g = torch.Generator(device=self.device).manual_seed(seed)
+        shapes = {"wq": (c.heads * dh, c.hidden), "wk": (c.kv_heads * dh, c.hidden), "wv": (c.kv_heads * dh, c.hidden),
+                  "wo": (c.hidden, c.heads * dh), "wg": (c.ffn, c.hidden), "wu": (c.ffn, c.hidden), "wd": (c.hidden, c.ffn)}
+        ones = torch.ones(c.hidden, dtype=torch.float32, device=self.device)
+        with torch.cuda.device(self.device):
+            for l in range(c.L):
+                for t in range(c.T):
+                    for k, shp in shapes.items():
+                        w = (torch.randn(shp, generator=g, device=self.device, dtype=torch.float32) * std).to(self.tdtype)
+                        check(lib().pt_model_set_weight(self.h, t, l, KIND[k], w.data_ptr(), self._stream()))
+                    for k in ("g1", "g2"):
+                        check(lib().pt_model_set_weight(self.h, t, l, KIND[k], ones.data_ptr(), self._stream()))
+            torch.cuda.synchronize()
+
+    def sync_count(self) -> int:
+        return lib().pt_sync_count(self.h)
+
+    def new_cache(self, num_pages: int, page_size: int = 16, free_order=None) -> "Cache":
+        return Cache(self, num_pages, page_size, free_order)
+
+    def workspace(self, tokens: int, batch: int, page_size: int):
+        if self.ws is None or tokens > self.ws_key[0] or batch > self.ws_key[1] or page_size < self.ws_key[2]:
+            n = _SZ()
+            check(lib().pt_workspace_bytes(self.h, tokens, batch, page_size, C.byref(n)))
+            self.ws = None
+            self.ws = self.torch.empty(n.value, dtype=self.torch.uint8, device=self.device)
+            self.ws_key = (tokens, batch, page_size)
+        return self.ws
+
+    def set_tap(self, layer: int | None, tokens: int = 0):
+        """layer None: off; -1: all layers.  Returns the tap tensor [nl, 2, T, tokens, hidden]."""
+        torch = self.torch
+        if layer is None:
+            check(lib().pt_set_debug_tap(self.h, 0, None))
+            self._tap = None
+            return None
+        nl = self.cfg.L if layer == -1 else 1
+        self._tap = torch.zeros((nl, 2, self.cfg.T, tokens, self.cfg.hidden), dtype=torch.float32, device=self.device)
+        check(lib().pt_set_debug_tap(self.h, layer, self._tap.data_ptr()))
+        return self._tap
+
+    def prefill(self, cache: "Cache", x, seq_ids, out=None):
+        """x: torch tensor [T, B, S, H] (or [1, B, S, H] = shared input) in the model dtype."""
+        torch = self.torch
+        assert x.is_cuda and x.dtype == self.tdtype and x.is_contiguous()
+        Tn, B, S, H = x.shape
+        stride = 0 if Tn == 1 and self.cfg.T > 1 else B * S * H
+        if out is None:
+            out = torch.empty((B, S, H), dtype=torch.float32, device=self.device)
+        ws = self.workspace(B * S, B, cache.page_size)
+        ids, pids = _i32arr(seq_ids)
+        assert len(ids) == B
+        with torch.cuda.device(self.device):
+            check(lib().pt_prefill(self.h, cache.h, x.data_ptr(), stride, B, S, pids, out.data_ptr(),
+                                   ws.data_ptr(), ws.numel(), self._stream()))
+        return out
+
+    def decode_step(self, cache: "Cache", x, seq_ids, out=None):
+        """x: torch tensor [T, B, H] (or [1, B, H]) in the model dtype -> fp32 [B, H]."""
+        torch = self.torch
+        assert x.is_cuda and x.dtype == self.tdtype and x.is_contiguous()
+        Tn, B, H = x.shape
+        stride = 0 if Tn == 1 and self.cfg.T > 1 else B * H
+        if out is None:
+            out = torch.empty((B, H), dtype=torch.float32, device=self.device)
+        ws = self.workspace(B, B, cache.page_size)
+        ids, pids = _i32arr(seq_ids)
+        assert len(ids) == B
+        with torch.cuda.device(self.device):
+            check(lib().pt_decode_step(self.h, cache.h, x.data_ptr(), stride, B, pids, out.data_ptr(),
+                                       ws.data_ptr(), ws.numel(), self._stream()))
+        return out
+
+    def device_status(self) -> tuple[int, int]:
+        code, detail = _I32(), _I32()
+        with self.torch.cuda.device(self.device):
+            check(lib().pt_device_status(self.h, self._stream(), C.byref(code), C.byref(detail)))
+        return code.value, detail.value
+
+
+class Cache:
+    """Paged KV cache: torch owns the pool, the library's host allocator owns the page tables."""
+
+    def __init__(self, model: Model, num_pages: int, page_size: int = 16, free_order=None, fill=None):
+        torch = model.torch
+        self.model, self.num_pages, self.page_size = model, num_pages, page_size
+        n = _SZ()
+        check(lib().pt_kv_cache_bytes(model.h, num_pages, page_size, C.byref(n)))
+        self.bytes = n.value
+        self.pool = torch.empty(n.value // (2 if model.dtype == "bf16" else 4), dtype=model.tdtype, device=model.device)
+        self.h = _P()
+        check(lib().pt_kv_cache_alloc(model.h, num_pages, page_size, self.pool.data_ptr(), n.value, C.byref(self.h)))
+        if free_order is not None:
+            a, p = _i32arr(free_order)
+            check(lib().pt_kv_set_free_list(self.h, p, len(a)))
+
+    def close(self):
+        if self.h:
+            lib().pt_kv_cache_free(self.h)
+            self.h = _P()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def reserve(self, seq: int, new_len: int):
+        check(lib().pt_kv_seq_reserve(self.h, seq, new_len))
+
+    def release(self, seq: int):
+        check(lib().pt_kv_seq_release(self.h, seq))
+
+    def truncate(self, seq: int, n: int):
+        check(lib().pt_kv_seq_truncate(self.h, seq, n))
+
+    def length(self, seq: int) -> int:
+        v = _I32()
+        check(lib().pt_kv_seq_len(self.h, seq, C.byref(v)))
+        return v.value
+
+    def block_table(self, seq: int) -> list[int]:
+        n = _I32()
+        check(lib().pt_kv_block_table(self.h, seq, None, 0, C.byref(n)))
+        buf = (_I32 * max(1, n.value))()
+        check(lib().pt_kv_block_table(self.h, seq, buf, n.value, C.byref(n)))
+        return list(buf[: n.value])
+
+    def slot(self, t: int, l: int, seq: int, pos: int, kv: int, head: int) -> int:
+        v = _I64()
+        check(lib().pt_kv_slot(self.h, t, l, seq, pos, kv, head, C.byref(v)))
+        return v.value

@@ -1,0 +1,128 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle on the same seeded inputs:
+final output, every layer's residual stream and deltas (debug tap), and the KV pool."""
+import numpy as np
+import pytest
+
+from oracle import pt_oracle as O
+from paper_2602_07306_b200 import inputs as I
+from tests import helpers as Hp
+
+pytestmark = pytest.mark.gpu
+
+
+def run_case(wl, *, B, S, sync_op="sum", simt=False, shuffle=False, shared=False, gain_jitter=0.0,
+             std=0.02, chunks=None, decode_steps=0, pages=None, check_pool=True):
+    """Prefill (optionally in chunks), then decode steps, on oracle and GPU; compare everything."""
+    import torch
+    ws = I.WeightSource(wl, gain_jitter=gain_jitter, std=std)
+    cfg = Hp.oracle_cfg(wl, sync_op)
+    total = S + decode_steps
+    ps = wl.page_size
+    pages = pages or (B * (-(-total // ps)) + 3)
+    order = I.free_list_permutation(pages, seed=7) if shuffle else None
+    seq_ids = [5 + 3 * b for b in range(B)]
+    model = Hp.make_model(wl, ws, sync_op=sync_op, max_pos=max(64, total), simt=simt)
+    cache = model.new_cache(pages, ps, order)
+    cache.pool.fill_(float("nan"))                       # sentinel: untouched slots must stay NaN
+    ocache = O.PagedKVCache(cfg, pages, ps, order)
+    x = I.prefill_inputs(wl, batch=B, seq=S, shared=shared)
+    chunks = chunks or [S]
+    assert sum(chunks) == S
+    report = []
+    s0 = 0
+    for n in chunks:
+        xs = x[:, :, s0:s0 + n]
+        taps = {}
+        ref = O.pt_prefill(cfg, ws, xs, ocache, seq_ids, taps)
+        tap = model.set_tap(-1, B * n)
+        xin = xs[:1] if shared else xs
+        got = model.prefill(cache, Hp.to_dev(model, xin), seq_ids)
+        torch.cuda.synchronize()
+        assert model.device_status() == (0, 0)
+        report.append(Hp.assert_close(got.cpu().numpy(), ref, wl.dtype, f"prefill chunk at {s0}"))
+        _check_taps(wl, tap.cpu().numpy(), taps, B, n)
+        s0 += n
+    for step in range(decode_steps):
+        xd = I.decode_inputs(wl, batch=B, step=step)
+        taps = {}
+        ref = O.pt_decode_step(cfg, ws, xd, ocache, seq_ids, taps)
+        tap = model.set_tap(-1, B)
+        got = model.decode_step(cache, Hp.to_dev(model, xd), seq_ids)
+        torch.cuda.synchronize()
+        assert model.device_status() == (0, 0)
+        report.append(Hp.assert_close(got.cpu().numpy(), ref, wl.dtype, f"decode step {step}"))
+        _check_taps(wl, tap.cpu().numpy(), taps, B, 1)
+    model.set_tap(None)
+    # page tables and lengths: bit-exact with the oracle's allocator
+    for s in seq_ids:
+        assert cache.block_table(s) == ocache.block_table[s]
+        assert cache.length(s) == ocache.length[s] == total
+    if check_pool:
+        pool = Hp.pool_as_numpy(cache, wl)
+        written = np.zeros(pool.shape, bool)
+        for s in seq_ids:
+            for pos in range(total):
+                page, slot = ocache.locate(s, pos)
+                written[:, :, page, :, :, slot, :] = True
+        assert np.all(np.isnan(pool[~written])), "a slot outside the expected set was written"
+        assert not np.any(np.isnan(pool[written])), "an expected slot was not written"
+        # cached values are single bf16 roundings of fp32 results (mean relative rounding error
+        # about 1.4e-3 by itself); the SIMT cross-check path rounds twice (projection, then RoPE)
+        mx, mean = Hp.rel_errs(pool[written], ocache.pool[written])
+        tmx, tmean = Hp.tol(wl.dtype)
+        if wl.dtype == "bf16":
+            tmean = 4e-3 if simt else 2.5e-3
+        assert mx <= tmx and mean <= tmean, f"KV pool: max-rel {mx:.3e}, mean-rel {mean:.3e}"
+    model.close()
+    return report
+
+
+def _check_taps(wl, tap, taps, B, n):
+    """tap [L, 2, T, B*n, H]: after-attention and after-layer residual streams."""
+    L, T = wl.L, wl.T
+    prev = None
+    for l in range(L):
+        h_end = taps["h"][l].reshape(T, B * n, wl.hidden)
+        Hp.assert_close(tap[l, 1], h_end, wl.dtype, f"layer {l} residual stream")
+        closes = (l + 1) % wl.D == 0
+        for t in range(T):
+            attn = taps["attn_delta"][(t, l)].reshape(B * n, wl.hidden)
+            ffn = taps["ffn_delta"][(t, l)].reshape(B * n, wl.hidden)
+            if prev is not None:                          # deltas on their own scale
+                got_attn = tap[l, 0, t].astype(np.float64) - prev[t]
+                mx, _ = Hp.rel_errs(got_attn, attn)
+                # the difference of two fp32 streams carries their rounding: allow it explicitly
+                slack = 4 * 6e-8 * np.abs(prev[t]).max() / max(np.abs(attn).max(), 1e-30)
+                assert mx <= Hp.tol(wl.dtype)[0] + slack, f"layer {l} track {t} attention delta: {mx:.3e}"
+            if not closes:
+                got_ffn = tap[l, 1, t].astype(np.float64) - tap[l, 0, t].astype(np.float64)
+                mx, _ = Hp.rel_errs(got_ffn, ffn)
+                slack = 4 * 6e-8 * np.abs(tap[l, 0, t]).max() / max(np.abs(ffn).max(), 1e-30)
+                assert mx <= Hp.tol(wl.dtype)[0] + slack, f"layer {l} track {t} ffn delta: {mx:.3e}"
+        prev = tap[l, 1].astype(np.float64)
+
+
+def small(dtype, T=2, L=4, D=2, H=128, nq=4, nkv=4, F=512, name="small"):
+    return I.Workload(name, T=T, L=L, D=D, hidden=H, heads=nq, kv_heads=nkv, ffn=F, dtype=dtype,
+                      mode="prefill", batch=1, seq=64, seed=0)
+
+
+def test_cfg0_fp32_prefill():
+    wl = I.WORKLOADS["cfg0"]
+    run_case(wl, B=wl.batch, S=wl.seq)
+
+
+def test_fp32_ragged_chunks_decode_shuffled_pages():
+    wl = small("f32", T=3, L=4, D=2, H=128, nq=4, nkv=2, F=176)
+    run_case(wl, B=3, S=37, chunks=[1, 15, 16, 5], decode_steps=3, shuffle=True, gain_jitter=0.2, std=0.05)
+
+
+@pytest.mark.parametrize("sync_op", ["sum", "mean"])
+def test_fp32_sync_ops_and_shared_input(sync_op):
+    wl = small("f32", T=4, L=4, D=1, H=64, nq=2, nkv=1, F=48)
+    run_case(wl, B=2, S=20, sync_op=sync_op, shared=True, gain_jitter=0.2, std=0.05)
+
+
+def test_bf16_simt_crosscheck_path():
+    wl = small("bf16", T=2, L=4, D=2, H=128, nq=2, nkv=1, F=176)
+    run_case(wl, B=2, S=33, simt=True, decode_steps=2, sync_op="mean", gain_jitter=0.1, std=0.05)
