@@ -114,7 +114,7 @@ pt_status pt_model_create(const pt_config* cfg, pt_model** out) {
     return PT_OK;
 }
 
-void pt_model_destroy(pt_model* m) { delete m; }
+void pt_model_destroy(pt_model* m) { if (m) tc_forget_model(m); delete m; }
 
 int32_t pt_sync_count(const pt_model* m) { return m ? m->cfg.L / m->cfg.D : -1; }
 

@@ -48,8 +48,6 @@ struct pt_model {
     int tap_layer = -2;
     float* tap_buf = nullptr;
     std::vector<char> meta_host;          // staging for the per-call metadata upload
-    // TMA descriptors of the packed weights (tensor-core path), built at bind time
-    CUtensorMap tm_wqkv, tm_wo, tm_wgu, tm_wd;
 
     size_t wqkv_layer() const { return (size_t)cfg.T * Nqkv * cfg.hidden; }     // elements
     size_t wo_layer() const { return (size_t)cfg.T * cfg.hidden * QD; }
@@ -124,5 +122,6 @@ void launch_pack(const pt_model* m, int kind, const void* src, void* dst_matrix_
 // pt_tc.cu (bf16 tensor-core path)
 pt_status tc_build_weight_maps(pt_model* m);
 pt_status tc_forward(Call& k);
+void tc_forget_model(const pt_model* m);
 
 }  // namespace pt

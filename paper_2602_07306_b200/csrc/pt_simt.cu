@@ -2,7 +2,7 @@
 // They are the fp32 path (accumulating in fp32 FMA, no tensor cores, no tf32) and, with
 // pt_config.flags bit 0, a slow cross-check of the bf16 tensor-core path.  The track index is
 // a grid dimension of every kernel.
-#include "pt_internal.h"
+#include "pt_tc.h"
 
 namespace pt {
 
@@ -239,6 +239,20 @@ void tap_copy(Call& k, int layer, int point, const float* src, size_t src_tstrid
     size_t block = (size_t)m->cfg.T * MH;
     float* dst = m->tap_buf + ((m->tap_layer == -1 ? (size_t)layer * 2 : 0) + point) * block;
     k_bcast<<<dim3(grid1d(MH), m->cfg.T), 256, 0, k.st>>>(src, src_tstride, dst, MH);
+    LAUNCH_COUNT();
+}
+
+void launch_simt_attn_bf16(Call& k, const __nv_bfloat16* q, int q_row_stride, const __nv_bfloat16* pool_l, __nv_bfloat16* o) {
+    pt_model* m = k.m;
+    pt_kv_cache* c = k.c;
+    const pt_config& g = m->cfg;
+    using E = __nv_bfloat16;
+    const int64_t pool_tstride = (int64_t)g.L * c->slab_elems;
+    dim3 ag(((size_t)k.M * g.heads * 32 + 127) / 128, g.T);
+#define ATTN(DH_) k_attn<E, DH_><<<ag, 128, 0, k.st>>>(q, q_row_stride, pool_l, pool_tstride, k.w.meta.bt, k.w.meta.maxp, \
+        k.w.meta.row_pos, k.w.meta.row_b, o, k.M, g.heads, g.kv_heads, c->ps, c->num_pages, m->status())
+    if (m->dh == 32) ATTN(32); else if (m->dh == 64) ATTN(64); else ATTN(128);
+#undef ATTN
     LAUNCH_COUNT();
 }
 

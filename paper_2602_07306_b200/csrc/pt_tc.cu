@@ -1,6 +1,188 @@
-// placeholder until the tensor-core path lands
-#include "pt_internal.h"
+// Forward pass of the bf16 tensor-core path: five launches per layer for all tracks at once
+// (QKV GEMM, attention, output-projection GEMM, gate/up GEMM, down GEMM); the track-sync of
+// Algorithm 1 is the down GEMM of every D-th layer run with its K loop over (track, k).
+#include "pt_tc.h"
+
 namespace pt {
-pt_status tc_build_weight_maps(pt_model*) { return PT_OK; }
-pt_status tc_forward(Call&) { set_error("bf16 tensor-core path not built yet"); return PT_ERR_UNSUPPORTED; }
+
+namespace {
+
+// x (bf16) -> fp32 residual stream, gain-scaled bf16 GEMM operand, partial sums of squares.
+// One warp per (row, track).
+__global__ void k_tc_prep(const __nv_bfloat16* __restrict__ x, int64_t x_stride, const float* __restrict__ gain,
+                          float* __restrict__ h, __nv_bfloat16* __restrict__ hb, float* __restrict__ ssq,
+                          int M, int H, int tiles) {
+    int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    int t = blockIdx.y;
+    if (warp >= M) return;
+    const __nv_bfloat16* xr = x + (size_t)t * x_stride + (size_t)warp * H;
+    size_t ro = ((size_t)t * M + warp) * H;
+    for (int tile = 0; tile < tiles; ++tile) {
+        int c = tile * kSsqTile + lane * 4;
+        float s = 0.f;
+        if (c < H) {
+            uint2 raw = *reinterpret_cast<const uint2*>(xr + c);
+            __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162*>(&raw.x), b = *reinterpret_cast<__nv_bfloat162*>(&raw.y);
+            float v0 = __low2float(a), v1 = __high2float(a), v2 = __low2float(b), v3 = __high2float(b);
+            *reinterpret_cast<float4*>(h + ro + c) = make_float4(v0, v1, v2, v3);
+            float4 g = *reinterpret_cast<const float4*>(gain + (size_t)t * H + c);
+            __nv_bfloat162 o0 = __floats2bfloat162_rn(v0 * g.x, v1 * g.y), o1 = __floats2bfloat162_rn(v2 * g.z, v3 * g.w);
+            uint2 ov;
+            ov.x = *reinterpret_cast<uint32_t*>(&o0); ov.y = *reinterpret_cast<uint32_t*>(&o1);
+            *reinterpret_cast<uint2*>(hb + ro + c) = ov;
+            s = v0 * v0 + v1 * v1 + v2 * v2 + v3 * v3;
+        }
+        for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (lane == 0) ssq[((size_t)t * M + warp) * tiles + tile] = s;
+    }
+}
+
+struct WMaps { CUtensorMap m[4][2]; };   // [qkv, o, gu, d][bn 128, bn 256]
+
+}  // namespace
+
+static std::unordered_map<const pt_model*, std::vector<WMaps>> g_wmaps;
+
+pt_status tc_build_weight_maps(pt_model* m) {
+    const pt_config& c = m->cfg;
+    if (c.hidden < 64 || c.ffn < 64) { set_error("the tensor-core path needs hidden >= 64 and ffn >= 64"); return PT_ERR_UNSUPPORTED; }
+    std::vector<WMaps> v(c.L);
+    const __nv_bfloat16* wqkv = (const __nv_bfloat16*)(m->wbuf + m->off_wqkv);
+    const __nv_bfloat16* wo = (const __nv_bfloat16*)(m->wbuf + m->off_wo);
+    const __nv_bfloat16* wgu = (const __nv_bfloat16*)(m->wbuf + m->off_wgu);
+    const __nv_bfloat16* wd = (const __nv_bfloat16*)(m->wbuf + m->off_wd);
+    for (int l = 0; l < c.L; ++l)
+        for (int b = 0; b < 2; ++b) {
+            int bn = b ? 256 : 128;
+            pt_status s;
+            if ((s = make_map_bf16(&v[l].m[0][b], wqkv + (size_t)l * m->wqkv_layer(), c.hidden, m->Nqkv, c.T, bn)) != PT_OK) return s;
+            if ((s = make_map_bf16(&v[l].m[1][b], wo + (size_t)l * m->wo_layer(), m->QD, c.hidden, c.T, bn)) != PT_OK) return s;
+            if ((s = make_map_bf16(&v[l].m[2][b], wgu + (size_t)l * m->wgu_layer(), c.hidden, 2 * c.ffn, c.T, bn)) != PT_OK) return s;
+            if ((s = make_map_bf16(&v[l].m[3][b], wd + (size_t)l * m->wd_layer(), c.ffn, c.hidden, c.T, bn)) != PT_OK) return s;
+        }
+    g_wmaps[m] = std::move(v);
+    return PT_OK;
+}
+
+void tc_forget_model(const pt_model* m) { g_wmaps.erase(m); }
+
+pt_status tc_forward(Call& k) {
+    pt_model* m = k.m;
+    pt_kv_cache* c = k.c;
+    const pt_config& g = m->cfg;
+    const int T = g.T, M = k.M, H = g.hidden, F = g.ffn;
+    const size_t MH = (size_t)M * H;
+    cudaStream_t st = k.st;
+    Work& w = k.w;
+    auto it = g_wmaps.find(m);
+    if (it == g_wmaps.end()) { set_error("weights not bound"); return PT_ERR_STATE; }
+    const std::vector<WMaps>& wm = it->second;
+    __nv_bfloat16* pool = (__nv_bfloat16*)c->pool;
+    const int64_t pool_tstride = (int64_t)g.L * c->slab_elems;
+    const int tiles = (H + kSsqTile - 1) / kSsqTile;
+    __nv_bfloat16* hb = (__nv_bfloat16*)w.a;
+    __nv_bfloat16* q = (__nv_bfloat16*)w.qkv;
+    __nv_bfloat16* o = (__nv_bfloat16*)w.o;
+    __nv_bfloat16* z = (__nv_bfloat16*)w.z;
+
+    CUtensorMap ta_h, ta_o, ta_z;
+    pt_status s;
+    if ((s = make_map_bf16(&ta_h, hb, H, M, T, 128)) != PT_OK) return s;
+    if ((s = make_map_bf16(&ta_o, o, m->QD, M, T, 128)) != PT_OK) return s;
+    if ((s = make_map_bf16(&ta_z, z, F, M, T, 128)) != PT_OK) return s;
+
+    k_tc_prep<<<dim3((M * 32 + 255) / 256, T), 256, 0, st>>>((const __nv_bfloat16*)k.x, k.x_stride, m->gain(0, 0), w.hT, hb, w.ssq, M, H, tiles);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+
+    const float* hin = w.hT;
+    size_t hin_stride = MH;
+    size_t ssq_tstride = (size_t)M * tiles;
+    for (int l = 0; l < g.L; ++l) {
+        __nv_bfloat16* pool_l = pool + (size_t)l * c->slab_elems;
+        GemmP base{};
+        base.M = M; base.status = m->status(); base.eps = g.rms_eps; base.kt = 1; base.T = T;
+        base.scale = 1.0f; base.n_sum = 1; base.n_out = 1;
+        {   // QKV: RMSNorm-1 scale, RoPE, KV append
+            GemmP p = base;
+            p.N = m->Nqkv; p.K = H;
+            p.ssq_in = w.ssq; p.ssq_in_tstride = ssq_tstride; p.ssq_tiles = tiles;
+            p.q_out = q; p.pool_l = pool_l; p.pool_tstride = pool_tstride; p.slab_elems = c->slab_elems;
+            p.row_kvoff = w.meta.row_kvoff; p.row_pos = w.meta.row_pos; p.cs = m->rope_cos(); p.sn = m->rope_sin();
+            p.nq = g.heads; p.nkv = g.kv_heads; p.dh = m->dh; p.ps = c->ps;
+            int bn = gemm_bn(p.N, M, T);
+            if ((s = launch_gemm(EPI_QKV, bn, ta_h, wm[l].m[0][bn == 256], p, st)) != PT_OK) return s;
+        }
+        if (k.decode) s = launch_decode_attn(k, q, pool_l, o);
+        else s = launch_flash_prefill(k, q, pool_l, o);
+        if (s != PT_OK) return s;
+        {   // output projection + residual; emits the operand and statistics of RMSNorm-2
+            GemmP p = base;
+            p.N = H; p.K = m->QD;
+            p.h_in = hin; p.h_in_tstride = hin_stride; p.h_out = w.hT; p.h_out_tstride = MH;
+            p.hb_out = hb; p.gain = m->gain(1, l);
+            p.ssq_out = w.ssq; p.ssq_out_tstride = (size_t)M * tiles; p.ssq_out_tiles = tiles;
+            int bn = gemm_bn(p.N, M, T);
+            if ((s = launch_gemm(EPI_RESID, bn, ta_o, wm[l].m[1][bn == 256], p, st)) != PT_OK) return s;
+            ssq_tstride = (size_t)M * tiles;
+        }
+        tap_copy(k, l, 0, w.hT, MH);
+        {   // gate/up + SwiGLU
+            GemmP p = base;
+            p.N = 2 * F; p.K = H;
+            p.ssq_in = w.ssq; p.ssq_in_tstride = ssq_tstride; p.ssq_tiles = tiles;
+            p.z_out = z;
+            int bn = gemm_bn(p.N, M, T);
+            if ((s = launch_gemm(EPI_SWIGLU, bn, ta_h, wm[l].m[2][bn == 256], p, st)) != PT_OK) return s;
+        }
+        {   // down projection + residual (+ track-sync when the layer closes a track block)
+            const bool sync = (l + 1) % g.D == 0, last = l + 1 == g.L;
+            GemmP p = base;
+            p.N = H; p.K = F;
+            p.h_in = w.hT; p.h_in_tstride = MH;
+            if (!last) { p.hb_out = hb; p.gain = m->gain(0, l + 1); p.ssq_out = w.ssq; p.ssq_out_tiles = tiles; }
+            if (sync) {
+                p.T = 1; p.kt = T; p.n_sum = T; p.n_out = T;
+                p.scale = g.sync_op ? 1.0f / T : 1.0f;
+                p.h_out = last ? k.out : w.hS; p.h_out_tstride = 0;
+                p.ssq_out_tstride = 0;
+                ssq_tstride = 0;
+                hin = p.h_out; hin_stride = 0;
+            } else {
+                p.h_out = w.hT; p.h_out_tstride = MH;
+                p.ssq_out_tstride = (size_t)M * tiles;
+                ssq_tstride = (size_t)M * tiles;
+                hin = w.hT; hin_stride = MH;
+            }
+            int bn = gemm_bn(p.N, M, p.T);
+            if ((s = launch_gemm(EPI_RESID, bn, ta_z, wm[l].m[3][bn == 256], p, st)) != PT_OK) return s;
+        }
+        tap_copy(k, l, 1, hin, hin_stride);
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_error("kernel launch failed: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
+    return PT_OK;
+}
+
+}  // namespace pt
+
+#include "pt_kernels.h"
+
+extern "C" pt_status pt_kernel_gemm_bf16(const void* a, const void* w, void* c, int32_t T, int32_t M, int32_t N,
+                                         int32_t K, int32_t bn, int32_t fold_tracks, void* status, void* stream) {
+    using namespace pt;
+    if (!a || !w || !c || !status) { set_error("null argument"); return PT_ERR_INVALID_ARG; }
+    if (T < 1 || M < 1 || N < 16 || N % 16 || K < 64 || K % 8) { set_error("unsupported GEMM shape"); return PT_ERR_INVALID_ARG; }
+    if (bn == 0) bn = gemm_bn(N, M, fold_tracks ? 1 : T);
+    if (bn != 128 && bn != 256) { set_error("bn must be 0, 128 or 256"); return PT_ERR_INVALID_ARG; }
+    CUtensorMap ta, tb;
+    pt_status s;
+    if ((s = make_map_bf16(&ta, a, K, M, T, 128)) != PT_OK) return s;
+    if ((s = make_map_bf16(&tb, w, K, N, T, bn)) != PT_OK) return s;
+    GemmP p{};
+    p.M = M; p.N = N; p.K = K; p.T = fold_tracks ? 1 : T; p.kt = fold_tracks ? T : 1;
+    p.status = (int*)status; p.c_out = (float*)c; p.scale = 1.f; p.n_sum = 1; p.n_out = 1;
+    if ((s = launch_gemm(EPI_PLAIN, bn, ta, tb, p, (cudaStream_t)stream)) != PT_OK) return s;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_error("kernel launch failed: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
+    return PT_OK;
 }

@@ -1,0 +1,53 @@
+// Declarations of the bf16 tensor-core path (tcgen05 GEMMs, flash prefill attention, split-KV
+// decode attention).
+#pragma once
+#include <algorithm>
+#include "pt_internal.h"
+
+namespace pt {
+
+enum { EPI_PLAIN = 0, EPI_QKV = 1, EPI_SWIGLU = 2, EPI_RESID = 3 };
+
+// Arguments of one track-grouped GEMM launch: C[t][M][N] = A[t][M][K] * W[t][N][K]^T.
+struct GemmP {
+    int M, N, K;            // per-track problem
+    int T;                  // tracks folded into the grid
+    int kt;                 // tracks folded into the K loop (1, or all tracks for the sync GEMM with T = 1)
+    int tiles_m, tiles_n;   // filled by the launcher
+    uint32_t tx_bytes;      // bytes one stage's two TMA loads deliver (filled by the launcher)
+    int* status;
+    // RMSNorm applied as a per-row scale: rinv = rsqrt(sum(ssq_in[row][:]) / K + eps)
+    const float* ssq_in; size_t ssq_in_tstride; int ssq_tiles; float eps;
+    // EPI_PLAIN
+    float* c_out;
+    // EPI_QKV
+    __nv_bfloat16* q_out;   // [T][M][nq*dh]
+    __nv_bfloat16* pool_l;  // KV pool slab of this layer, track 0
+    int64_t pool_tstride, slab_elems;
+    const int64_t* row_kvoff; const int32_t* row_pos;
+    const float* cs; const float* sn;
+    int nq, nkv, dh, ps;
+    // EPI_SWIGLU
+    __nv_bfloat16* z_out;   // [T][M][N/2]
+    // EPI_RESID
+    const float* h_in; size_t h_in_tstride; int n_sum; float scale;
+    float* h_out; size_t h_out_tstride;
+    __nv_bfloat16* hb_out;  // [T][M][N] gain-scaled copy for the next GEMM (may be null)
+    const float* gain;      // [T][N] gains of the next RMSNorm
+    int n_out;              // tracks that receive hb_out (1 = own track, T = all after a sync)
+    float* ssq_out; size_t ssq_out_tstride; int ssq_out_tiles;
+};
+
+pt_status make_map_bf16(CUtensorMap* out, const void* base, int64_t k, int64_t rows, int64_t tracks, int box_rows);
+int gemm_bn(int N, int M, int T);
+pt_status launch_gemm(int epi, int bn, const CUtensorMap& ta, const CUtensorMap& tb, GemmP p, cudaStream_t st);
+
+// pt_simt.cu
+void tap_copy(Call& k, int layer, int point, const float* src, size_t src_tstride);
+void launch_simt_attn_bf16(Call& k, const __nv_bfloat16* q, int q_row_stride, const __nv_bfloat16* pool_l, __nv_bfloat16* o);
+
+// pt_tc_attn.cu
+pt_status launch_flash_prefill(Call& k, const __nv_bfloat16* q, const __nv_bfloat16* pool_l, __nv_bfloat16* o);
+pt_status launch_decode_attn(Call& k, const __nv_bfloat16* q, const __nv_bfloat16* pool_l, __nv_bfloat16* o);
+
+}  // namespace pt

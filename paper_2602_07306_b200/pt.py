@@ -60,6 +60,7 @@ _PROTOS = {
     "pt_set_debug_tap": (_I32, [_P, _I32, _P]),
     "pt_device_status": (_I32, [_P, _P, C.POINTER(_I32), C.POINTER(_I32)]),
     "pt_launch_count": (_I64, []),
+    "pt_kernel_gemm_bf16": (_I32, [_P, _P, _P, _I32, _I32, _I32, _I32, _I32, _I32, _P, _P]),
     "pt_last_error": (C.c_char_p, []),
 }
 EXPORTS = tuple(_PROTOS)
@@ -287,3 +288,17 @@ class Cache:
         v = _I64()
         check(lib().pt_kv_slot(self.h, t, l, seq, pos, kv, head, C.byref(v)))
         return v.value
+
+
+def kernel_gemm_bf16(a, w, bn: int = 0, fold_tracks: bool = False):
+    """a [T, M, K], w [T, N, K] bf16 CUDA tensors -> fp32 [T, M, N] ([1, M, N] when folding tracks)."""
+    import torch
+    T, M, K = a.shape
+    N = w.shape[1]
+    assert a.is_contiguous() and w.is_contiguous() and a.dtype == w.dtype == torch.bfloat16
+    c = torch.empty((1 if fold_tracks else T, M, N), dtype=torch.float32, device=a.device)
+    status = torch.zeros(16, dtype=torch.int32, device=a.device)
+    with torch.cuda.device(a.device):
+        check(lib().pt_kernel_gemm_bf16(a.data_ptr(), w.data_ptr(), c.data_ptr(), T, M, N, K, bn, int(fold_tracks),
+                                        status.data_ptr(), torch.cuda.current_stream().cuda_stream))
+    return c, status

@@ -66,12 +66,14 @@ def run_case(wl, *, B, S, sync_op="sum", simt=False, shuffle=False, shared=False
                 written[:, :, page, :, :, slot, :] = True
         assert np.all(np.isnan(pool[~written])), "a slot outside the expected set was written"
         assert not np.any(np.isnan(pool[written])), "an expected slot was not written"
-        # cached values are single bf16 roundings of fp32 results (mean relative rounding error
-        # about 1.4e-3 by itself); the SIMT cross-check path rounds twice (projection, then RoPE)
+        # a cached bf16 value carries its own rounding (mean relative error about 1.4e-3) on top
+        # of the rounding of the bf16 GEMM operand it was projected from, so the mean bound of
+        # the fp32 output (2e-3) is doubled for the pool; the SIMT cross-check path rounds once
+        # more (projection, then RoPE)
         mx, mean = Hp.rel_errs(pool[written], ocache.pool[written])
         tmx, tmean = Hp.tol(wl.dtype)
         if wl.dtype == "bf16":
-            tmean = 4e-3 if simt else 2.5e-3
+            tmean = 6e-3 if simt else 4e-3
         assert mx <= tmx and mean <= tmean, f"KV pool: max-rel {mx:.3e}, mean-rel {mean:.3e}"
     model.close()
     return report
@@ -126,3 +128,22 @@ def test_fp32_sync_ops_and_shared_input(sync_op):
 def test_bf16_simt_crosscheck_path():
     wl = small("bf16", T=2, L=4, D=2, H=128, nq=2, nkv=1, F=176)
     run_case(wl, B=2, S=33, simt=True, decode_steps=2, sync_op="mean", gain_jitter=0.1, std=0.05)
+
+
+@pytest.mark.parametrize("H,nq,nkv,F", [(128, 2, 1, 176), (128, 4, 4, 256), (256, 2, 2, 208)])
+def test_bf16_tensor_core_path_small(H, nq, nkv, F):
+    """Head sizes 64, 32 and 128; GQA and MHA; widths that leave N and K tile tails."""
+    wl = small("bf16", T=3, L=4, D=2, H=H, nq=nq, nkv=nkv, F=F)
+    run_case(wl, B=3, S=37, chunks=[1, 15, 16, 5], decode_steps=3, shuffle=True, gain_jitter=0.1, std=0.05)
+
+
+@pytest.mark.parametrize("sync_op", ["sum", "mean"])
+def test_bf16_tensor_core_sync_every_layer_shared_input(sync_op):
+    wl = small("bf16", T=4, L=3, D=1, H=128, nq=2, nkv=2, F=128)
+    run_case(wl, B=2, S=150, sync_op=sync_op, shared=True, gain_jitter=0.1, std=0.05)
+
+
+@pytest.mark.parametrize("sync_op", ["sum", "mean"])
+def test_cfg1_bf16_prefill(sync_op):
+    wl = I.WORKLOADS["cfg1"]
+    run_case(wl, B=wl.batch, S=wl.seq, sync_op=sync_op, check_pool=(sync_op == "sum"))

@@ -32,7 +32,7 @@ def make(lib, **kw):
 
 
 def test_library_exports_every_declared_symbol(lib):
-    text = open(os.path.join(ROOT, "include", "pt.h")).read()
+    text = "".join(open(os.path.join(ROOT, "include", f)).read() for f in sorted(os.listdir(os.path.join(ROOT, "include"))))
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     declared = set(re.findall(r"\b(pt_[a-z0-9_]+)\s*\(", text))
     assert declared, "no declarations found"
