@@ -147,3 +147,11 @@ def test_bf16_tensor_core_sync_every_layer_shared_input(sync_op):
 def test_cfg1_bf16_prefill(sync_op):
     wl = I.WORKLOADS["cfg1"]
     run_case(wl, B=wl.batch, S=wl.seq, sync_op=sync_op, check_pool=(sync_op == "sum"))
+
+
+@pytest.mark.parametrize("H,nq,nkv", [(256, 2, 1), (256, 4, 4), (128, 4, 2)])
+def test_bf16_decode_split_kv_long_context(H, nq, nkv):
+    """KV long enough for several key ranges per sequence (split-KV + combine), ragged lengths
+    via an extra prefill chunk on one sequence only is covered by the decode steps below."""
+    wl = small("bf16", T=2, L=2, D=1, H=H, nq=nq, nkv=nkv, F=128)
+    run_case(wl, B=2, S=700, decode_steps=2, shuffle=True, std=0.05, gain_jitter=0.1)
