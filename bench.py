@@ -1,0 +1,469 @@
+#!/usr/bin/env python
+"""Benchmark of the Parallel Track (PT) forward pass on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg3|cfg1|cfg4]
+                    [--extra cfg3,cfg1] [--impl ours|reference]
+
+One JSON line on stdout.  A "step" is one pass of the whole hot path over one batch: one
+decode step (cfg2, cfg4) or one prefill (cfg1, cfg3) through every layer and track-sync.
+`value` is tokens/s with inputs resident in HBM; `e2e` is the same call made from pinned host
+buffers with the host<->device copies inside the timed region.  With N > 1 (torchrun) every
+rank runs the same workload on its own batch (weak scaling, no data-path collective: batch
+rows are independent) and rank 0 reports the aggregate over the slowest rank.
+
+`--impl reference` times the CPU oracle (float64 NumPy, as it stands) on a bounded sample of
+the same workload on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2602_07306_b200 import inputs as I  # noqa: E402
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ------------------------------------------------------------------------------ clocks
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, dev):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID("GPU-" + str(torch.cuda.get_device_properties(dev).uuid))
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(dev.index or 0)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "sw_thermal_slowdown": 0x20,
+                 "hw_thermal_slowdown": 0x40, "hw_power_brake": 0x80}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(0.05)
+
+    def __enter__(self):
+        if self.nv:
+            self._thr = threading.Thread(target=self._loop, daemon=True)
+            self._thr.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thr:
+            self._thr.join()
+
+    def summary(self):
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------------------ workloads
+
+def algorithmic(wl, B, lens=None, S=None):
+    """Algorithmic work of one step (no padding, no re-reads, causal triangle only)."""
+    P = wl.params_per_track_layer()
+    dh = wl.head_dim
+    if wl.mode == "decode":
+        keys = int(np.sum(np.asarray(lens, np.int64) + 1))
+        kv_read = wl.T * wl.L * 2 * wl.kv_heads * dh * 2 * keys
+        kv_write = wl.T * wl.L * 2 * wl.kv_heads * dh * 2 * B
+        weights = wl.T * wl.L * P * 2
+        return {"bytes": kv_read + kv_write + weights, "kv_read_bytes": kv_read, "weight_bytes": weights,
+                "attn_bytes_per_layer": kv_read // wl.L}
+    tokens = B * S
+    gemm = 2 * wl.T * wl.L * P * tokens
+    attn = wl.T * wl.L * B * 4 * wl.heads * dh * S * (S + 1) // 2
+    return {"flops": gemm + attn, "gemm_flops": gemm, "attn_flops": attn}
+
+
+def make_model(wl, dev, max_pos):
+    from paper_2602_07306_b200 import pt
+    m = pt.Model(T=wl.T, D=wl.D, L=wl.L, hidden=wl.hidden, heads=wl.heads, kv_heads=wl.kv_heads, ffn=wl.ffn,
+                 dtype=wl.dtype, rope_base=wl.rope_base, rms_eps=wl.rms_eps, max_pos=max_pos, device=dev)
+    m.init_random(seed=wl.seed)
+    return m
+
+
+def timed_steps(torch, fn, steps, warmup):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(steps):
+        fn()
+    ev1.record()
+    torch.cuda.synchronize()
+    return ev0.elapsed_time(ev1) / steps
+
+
+def run_decode(wl, dev, steps, warmup, barrier, rank):
+    import torch
+    from paper_2602_07306_b200 import pt
+    pk, pk_kind = peaks()
+    lens_all = I.kv_lengths(wl)
+    ps = wl.page_size
+    model = make_model(wl, dev, max_pos=int(lens_all.max()) + 16)
+    # choose the batch: everything, or the largest prefix (multiple of 16) whose pages fit
+    free, _ = torch.cuda.mem_get_info(dev)
+    page_bytes = wl.T * wl.L * 2 * wl.kv_heads * ps * wl.head_dim * 2
+    pages_of = (lens_all.astype(np.int64) + 1 + ps - 1) // ps
+    budget = free - (6 << 30)
+    B = wl.batch
+    while B > 16 and int(pages_of[:B].sum()) * page_bytes > budget:
+        B -= 16
+    lens = lens_all[:B]
+    num_pages = int(pages_of[:B].sum())
+    cache = model.new_cache(num_pages, ps)
+    seq_ids = list(range(B))
+    # fill the cache by real prefills of N(0,1) inputs, grouped by length, in bounded sub-batches
+    g = torch.Generator(device=dev).manual_seed(wl.seed + 1)
+    t_fill = time.time()
+    order = np.argsort(-lens, kind="stable")
+    i = 0
+    while i < B:
+        n = int(lens[order[i]])
+        j = i
+        while j < B and int(lens[order[j]]) == n and (j - i + 1) * n <= 16384:
+            j += 1
+        ids = [int(s) for s in order[i:j]]
+        x = torch.randn((wl.T, len(ids), n, wl.hidden), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        model.prefill(cache, x, ids)
+        i = j
+    torch.cuda.synchronize()
+    t_fill = time.time() - t_fill
+    code = model.device_status()
+    assert code == (0, 0), f"device status after cache fill: {code}"
+    xd = torch.randn((wl.T, B, wl.hidden), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    out = torch.empty((B, wl.hidden), dtype=torch.float32, device=dev)
+
+    def step():
+        model.decode_step(cache, xd, seq_ids, out)
+        for s in seq_ids:                     # same KV lengths every step
+            cache.truncate(s, int(lens[s]))
+
+    alg = algorithmic(wl, B, lens=lens)
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    barrier()
+    model.profile(True)
+    l0 = pt.lib().pt_launch_count()
+    with ClockSampler(dev) as clk:
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for _ in range(steps):
+            step()
+        ev1.record()
+        torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1) / steps
+    launches = pt.lib().pt_launch_count() - l0
+    prof = model.profile_read()
+    model.profile(False)
+    assert model.device_status() == (0, 0)
+    attn_ms, attn_n = prof["attention"]
+    attn_avg_ms = attn_ms / max(attn_n, 1)
+    achieved = alg["attn_bytes_per_layer"] / (attn_avg_ms * 1e-3) / 1e9
+    roof = {"bound": "hbm", "kernel": "k_decode_attn", "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s",
+            "frac": achieved / pk["hbm_gbs"], "traffic": None, "peak_kind": f"of {pk_kind}",
+            "avg_launch_ms": attn_avg_ms, "launches": attn_n,
+            "step_hbm_gbs": alg["bytes"] / (ms * 1e-3) / 1e9, "step_frac": alg["bytes"] / (ms * 1e-3) / 1e9 / pk["hbm_gbs"],
+            "step_frac_of_nominal_8tbs": alg["bytes"] / (ms * 1e-3) / 8e12}
+    # end to end from pinned host buffers
+    xh = xd.cpu().pin_memory()
+    oh = torch.empty((B, wl.hidden), dtype=torch.float32).pin_memory()
+    xdev = torch.empty_like(xd)
+
+    def e2e_step():
+        xdev.copy_(xh, non_blocking=True)
+        model.decode_step(cache, xdev, seq_ids, out)
+        oh.copy_(out, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        for s in seq_ids:
+            cache.truncate(s, int(lens[s]))
+
+    for _ in range(2):
+        e2e_step()
+    t0 = time.perf_counter()
+    n_e2e = max(3, steps // 2)
+    for _ in range(n_e2e):
+        e2e_step()
+    e2e_ms = (time.perf_counter() - t0) / n_e2e * 1e3
+    res = {"ms": ms, "tokens": B, "alg": alg, "roofline": roof, "launches": launches, "clocks": clk.summary(),
+           "kernels_ms_per_step": {k: round(v[0] / steps, 4) for k, v in prof.items()},
+           "e2e": {"value": B / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": xh.numel() * 2,
+                   "d2h_bytes_per_step": oh.numel() * 4},
+           "config": {"workload": f"{wl.name}: decode T={wl.T} L={wl.L} D={wl.D} H={wl.hidden} heads={wl.heads}/{wl.kv_heads} "
+                                  f"F={wl.ffn} batch={B} kv_len={'U[%d,%d]' % wl.ragged if wl.ragged else wl.seq} page={ps}",
+                      "batch": B, "batch_requested": wl.batch, "kv_tokens": int(lens.sum()), "cache_fill_s": round(t_fill, 2),
+                      "l2": "working set (KV cache + weights) far larger than L2; no flush needed"}}
+    cache.close()
+    model.close()
+    del cache, model
+    torch.cuda.empty_cache()
+    return res
+
+
+def run_prefill(wl, dev, steps, warmup, barrier, rank):
+    import torch
+    from paper_2602_07306_b200 import pt
+    pk, pk_kind = peaks()
+    B, S, ps = wl.batch, wl.seq, wl.page_size
+    model = make_model(wl, dev, max_pos=S)
+    pages = B * ((S + ps - 1) // ps)
+    cache = model.new_cache(pages, ps)
+    seq_ids = list(range(B))
+    g = torch.Generator(device=dev).manual_seed(wl.seed + 1)
+    x = torch.randn((wl.T, B, S, wl.hidden), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    out = torch.empty((B, S, wl.hidden), dtype=torch.float32, device=dev)
+
+    def step():
+        model.prefill(cache, x, seq_ids, out)
+        for s in seq_ids:
+            cache.truncate(s, 0)
+
+    alg = algorithmic(wl, B, S=S)
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    barrier()
+    model.profile(True)
+    l0 = pt.lib().pt_launch_count()
+    with ClockSampler(dev) as clk:
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for _ in range(steps):
+            step()
+        ev1.record()
+        torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1) / steps
+    launches = pt.lib().pt_launch_count() - l0
+    prof = model.profile_read()
+    model.profile(False)
+    assert model.device_status() == (0, 0)
+    gemm_ms = sum(prof[k][0] for k in ("gemm_qkv", "gemm_out", "gemm_gate_up", "gemm_down", "gemm_down_sync")) / steps
+    gemm_n = sum(prof[k][1] for k in ("gemm_qkv", "gemm_out", "gemm_gate_up", "gemm_down", "gemm_down_sync"))
+    attn_ms = prof["attention"][0] / steps
+    gemm_tf = alg["gemm_flops"] / (gemm_ms * 1e-3) / 1e12
+    attn_tf = alg["attn_flops"] / (attn_ms * 1e-3) / 1e12
+    peak = pk["bf16_tflops_sustained"] if ms * steps > 1000 else pk["bf16_tflops"]
+    roof = {"bound": "tensor", "kernel": "gemm_tc (QKV, out, gate/up, down, down+sync)", "achieved": gemm_tf, "peak": peak,
+            "unit": "TFLOP/s", "frac": gemm_tf / peak, "traffic": None, "peak_kind": f"of {pk_kind}",
+            "avg_launch_ms": gemm_ms * steps / max(gemm_n, 1), "launches": gemm_n,
+            "frac_of_nominal_2250": gemm_tf / 2250.0, "attention_tflops": attn_tf,
+            "step_tflops": alg["flops"] / (ms * 1e-3) / 1e12}
+    xh = x.cpu().pin_memory()
+    oh = torch.empty((B, S, wl.hidden), dtype=torch.float32).pin_memory()
+    xdev = torch.empty_like(x)
+
+    def e2e_step():
+        xdev.copy_(xh, non_blocking=True)
+        model.prefill(cache, xdev, seq_ids, out)
+        oh.copy_(out, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        for s in seq_ids:
+            cache.truncate(s, 0)
+
+    e2e_step()
+    t0 = time.perf_counter()
+    n_e2e = max(2, steps // 2)
+    for _ in range(n_e2e):
+        e2e_step()
+    e2e_ms = (time.perf_counter() - t0) / n_e2e * 1e3
+    res = {"ms": ms, "tokens": B * S, "alg": alg, "roofline": roof, "launches": launches, "clocks": clk.summary(),
+           "kernels_ms_per_step": {k: round(v[0] / steps, 4) for k, v in prof.items()},
+           "e2e": {"value": B * S / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": xh.numel() * 2,
+                   "d2h_bytes_per_step": oh.numel() * 4},
+           "config": {"workload": f"{wl.name}: prefill T={wl.T} L={wl.L} D={wl.D} H={wl.hidden} heads={wl.heads}/{wl.kv_heads} "
+                                  f"F={wl.ffn} batch={B} seq={S} page={ps}", "batch": B, "seq_len": S,
+                      "l2": "activations + weights per step larger than L2" if wl.T * B * S * wl.hidden * 4 > 126e6
+                            else "inputs smaller than L2: weights partly L2-resident between steps (launch-bound workload)"}}
+    cache.close()
+    model.close()
+    del cache, model
+    torch.cuda.empty_cache()
+    return res
+
+
+# ------------------------------------------------------------------------------ CPU oracle arm
+
+class _Cached:
+    def __init__(self, src, T, L):
+        self.w = {(t, l): src.get(t, l) for l in range(L) for t in range(T)}
+
+    def get(self, t, l):
+        return self.w[(t, l)]
+
+
+def oracle_sample(wl, budget_s=20.0):
+    """Time the CPU oracle, as it stands, on a bounded sample of the workload: the first track
+    block (D of the L layers, all T tracks) on a few rows / a shorter prompt; tokens/s is scaled by
+    D/L to the full depth (layers cost the same).  Returns (tokens_per_s, description, seconds)."""
+    from oracle import pt_oracle as O
+    import dataclasses
+    cores = len(os.sched_getaffinity(0))
+    sub = dataclasses.replace(wl, L=wl.D)
+    cfg = O.PTConfig(T=sub.T, D=sub.D, L=sub.L, hidden=sub.hidden, heads=sub.heads, kv_heads=sub.kv_heads, ffn=sub.ffn)
+    ws = _Cached(I.WeightSource(sub), sub.T, sub.L)
+    scale = wl.D / wl.L
+    if wl.mode == "decode":
+        rows = 2
+        lens = I.kv_lengths(wl, batch=rows)
+        pages = int(sum((int(n) + 1 + 15) // 16 for n in lens))
+        cache = O.PagedKVCache(cfg, pages, 16)
+        rng = np.random.default_rng(0)
+        for b in range(rows):                     # synthetic cache contents: timing does not depend on them
+            cache.reserve(b, int(lens[b]))
+            cache.length[b] = int(lens[b])
+        cache.pool[...] = rng.standard_normal(cache.pool.shape)
+        x = I.decode_inputs(sub, batch=rows)
+        t0 = time.perf_counter()
+        O.pt_decode_step(cfg, ws, x, cache, list(range(rows)))
+        dt = time.perf_counter() - t0
+        return rows / dt * scale, (f"{rows} sequences (KV {lens.tolist()}), first track block ({wl.D} of {wl.L} layers, "
+                                   f"all {wl.T} tracks), cache pre-filled with N(0,1); tokens/s scaled by {wl.D}/{wl.L}"), dt, cores
+    S = min(wl.seq, 256)
+    x = I.prefill_inputs(sub, batch=1, seq=S)
+    cache = O.PagedKVCache(cfg, (S + 15) // 16, 16)
+    t0 = time.perf_counter()
+    O.pt_prefill(cfg, ws, x, cache, [0])
+    dt = time.perf_counter() - t0
+    return S / dt * scale, (f"1 sequence x {S} tokens, first track block ({wl.D} of {wl.L} layers, all {wl.T} tracks); "
+                            f"tokens/s scaled by {wl.D}/{wl.L}"), dt, cores
+
+
+# ------------------------------------------------------------------------------ main
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--extra", default="cfg3", help="comma-separated workloads reported under 'extra' (N=1 only); '' for none")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    a = ap.parse_args()
+    a.warmup = max(a.warmup, 3) if a.impl == "ours" else a.warmup
+    wl = I.WORKLOADS[a.workload]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    metric = "decode tokens/s" if wl.mode == "decode" else "prefill tokens/s"
+
+    if a.impl == "reference":
+        if rank != 0:
+            return
+        vals = []
+        for _ in range(max(1, a.warmup)):
+            oracle_sample(wl)
+        t0 = time.perf_counter()
+        for _ in range(a.steps):
+            v, sample, dt, cores = oracle_sample(wl)
+            vals.append(v)
+        ms = (time.perf_counter() - t0) / a.steps * 1e3
+        v = float(np.mean(vals))
+        print(json.dumps({"impl": "reference", "metric": f"PT {metric} (CPU oracle, bounded sample)", "value": v, "unit": "tokens/s",
+                          "n_gpus": a.gpus, "steps": a.steps, "warmup": a.warmup, "ms_per_step": ms, "higher_is_better": True,
+                          "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                          "config": {"workload": f"{wl.name} ({wl.mode})"},
+                          "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+                          "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+        return
+
+    import torch
+    import torch.distributed as dist
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    run = run_decode if wl.mode == "decode" else run_prefill
+    r = run(wl, dev, a.steps, a.warmup, barrier, rank)
+    ms = r["ms"]
+    if world > 1:
+        tmax = torch.tensor([ms], device=dev)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        ms = float(tmax.item())
+        toks = torch.tensor([float(r["tokens"])], device=dev)
+        dist.all_reduce(toks, op=dist.ReduceOp.SUM)
+        total_tokens = float(toks.item())
+        e2e_t = torch.tensor([r["tokens"] / r["e2e"]["value"]], device=dev)
+        dist.all_reduce(e2e_t, op=dist.ReduceOp.MAX)
+        r["e2e"]["value"] = total_tokens / float(e2e_t.item())
+    else:
+        total_tokens = float(r["tokens"])
+    extra = {}
+    if world == 1 and a.extra:
+        for name in [n for n in a.extra.split(",") if n and n != a.workload]:
+            w2 = I.WORKLOADS[name]
+            try:
+                r2 = (run_decode if w2.mode == "decode" else run_prefill)(w2, dev, max(3, a.steps // 4), 3, barrier, rank)
+                extra[name] = {"metric": "decode tokens/s" if w2.mode == "decode" else "prefill tokens/s",
+                               "value": r2["tokens"] / (r2["ms"] * 1e-3), "ms_per_step": r2["ms"], "roofline": r2["roofline"],
+                               "kernels_ms_per_step": r2["kernels_ms_per_step"], "config": r2["config"], "clocks": r2["clocks"],
+                               "e2e": r2["e2e"]}
+            except Exception as e:  # an extra must never take the headline down
+                extra[name] = {"error": repr(e)[:300]}
+    cpu = None
+    if rank == 0 and world == 1 and not a.no_cpu_baseline:
+        v, sample, dt, cores = oracle_sample(wl)
+        cpu = {"value": v, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample, "seconds": round(dt, 2)}
+    if rank == 0:
+        line = {"metric": f"PT {metric} on B200", "value": total_tokens / (ms * 1e-3), "unit": "tokens/s", "n_gpus": world,
+                "steps": a.steps, "warmup": a.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
+                "config": r["config"], "clocks": r["clocks"], "e2e": r["e2e"], "gpu_launches": int(r["launches"]),
+                "roofline": r["roofline"], "cpu_baseline": cpu, "kernels_ms_per_step": r["kernels_ms_per_step"],
+                "algorithmic": r["alg"], "extra": extra}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

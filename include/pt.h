@@ -187,6 +187,15 @@ pt_status pt_set_debug_tap(pt_model* m, int32_t layer, void* dev_buf);
  * location code. */
 pt_status pt_device_status(pt_model* m, void* stream, int32_t* code, int32_t* detail);
 
+/* Kernel timing for benchmarks.  With timing on, the bf16 forward calls bracket every kernel
+ * with CUDA events on the call's stream.  pt_profile_read waits for those events, ADDS device
+ * milliseconds and launch counts per category into ms[] and launches[] (host, PT_PROF_CATEGORIES
+ * entries each) and forgets the events.  Categories: 0 attention, 1 QKV GEMM, 2 output-projection
+ * GEMM, 3 gate/up GEMM, 4 down GEMM, 5 down GEMM with track-sync, 6 everything else. */
+#define PT_PROF_CATEGORIES 7
+pt_status pt_profile_enable(pt_model* m, int32_t on);
+pt_status pt_profile_read(pt_model* m, float* ms, int64_t* launches);
+
 /* Kernels launched by this library since the process started (all models). */
 int64_t pt_launch_count(void);
 

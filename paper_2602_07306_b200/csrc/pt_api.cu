@@ -114,7 +114,32 @@ pt_status pt_model_create(const pt_config* cfg, pt_model** out) {
     return PT_OK;
 }
 
-void pt_model_destroy(pt_model* m) { if (m) tc_forget_model(m); delete m; }
+void pt_model_destroy(pt_model* m) {
+    if (!m) return;
+    tc_forget_model(m);
+    for (auto& e : m->prof_ev) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
+    delete m;
+}
+
+pt_status pt_profile_enable(pt_model* m, int32_t on) {
+    if (!m) PT_FAIL(PT_ERR_INVALID_ARG, "null argument");
+    m->prof_on = on != 0;
+    if (!on) m->prof_used = 0;
+    return PT_OK;
+}
+
+pt_status pt_profile_read(pt_model* m, float* ms, int64_t* launches) {
+    if (!m || !ms || !launches) PT_FAIL(PT_ERR_INVALID_ARG, "null argument");
+    for (size_t i = 0; i < m->prof_used; ++i) {
+        auto& e = m->prof_ev[i];
+        PT_CUDA(cudaEventSynchronize(e.b));
+        float t = 0.f;
+        PT_CUDA(cudaEventElapsedTime(&t, e.a, e.b));
+        if (e.cat >= 0 && e.cat < PT_PROF_CATEGORIES) { ms[e.cat] += t; launches[e.cat] += 1; }
+    }
+    m->prof_used = 0;
+    return PT_OK;
+}
 
 int32_t pt_sync_count(const pt_model* m) { return m ? m->cfg.L / m->cfg.D : -1; }
 

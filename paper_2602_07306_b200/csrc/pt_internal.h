@@ -48,6 +48,11 @@ struct pt_model {
     int tap_layer = -2;
     float* tap_buf = nullptr;
     std::vector<char> meta_host;          // staging for the per-call metadata upload
+    // optional per-kernel timing (pt_profile_enable)
+    struct ProfEv { cudaEvent_t a, b; int cat; };
+    bool prof_on = false;
+    std::vector<ProfEv> prof_ev;
+    size_t prof_used = 0;
 
     size_t wqkv_layer() const { return (size_t)cfg.T * Nqkv * cfg.hidden; }     // elements
     size_t wo_layer() const { return (size_t)cfg.T * cfg.hidden * QD; }
@@ -113,6 +118,23 @@ struct Call {
     int n_items, max_splits;
     const int32_t* items;     // device [n_items][4]: b, start, count, split index
     const int32_t* nsplit;    // device [B]
+};
+
+// Brackets one kernel launch with events when timing is on.
+struct ProfScope {
+    pt_model* m; cudaStream_t st; int idx = -1;
+    ProfScope(pt_model* m_, cudaStream_t st_, int cat) : m(m_), st(st_) {
+        if (!m->prof_on) return;
+        if (m->prof_used == m->prof_ev.size()) {
+            pt_model::ProfEv e{};
+            if (cudaEventCreate(&e.a) != cudaSuccess || cudaEventCreate(&e.b) != cudaSuccess) return;
+            m->prof_ev.push_back(e);
+        }
+        idx = (int)m->prof_used++;
+        m->prof_ev[idx].cat = cat;
+        cudaEventRecord(m->prof_ev[idx].a, st);
+    }
+    ~ProfScope() { if (idx >= 0) cudaEventRecord(m->prof_ev[idx].b, st); }
 };
 
 // pt_simt.cu

@@ -91,8 +91,9 @@ pt_status tc_forward(Call& k) {
     if ((s = make_map_bf16(&ta_o, o, m->QD, M, T, 128)) != PT_OK) return s;
     if ((s = make_map_bf16(&ta_z, z, F, M, T, 128)) != PT_OK) return s;
 
+    { ProfScope ps(m, st, 6);
     k_tc_prep<<<dim3((M * 32 + 255) / 256, T), 256, 0, st>>>((const __nv_bfloat16*)k.x, k.x_stride, m->gain(0, 0), w.hT, hb, w.ssq, M, H, tiles);
-    g_launches.fetch_add(1, std::memory_order_relaxed);
+    g_launches.fetch_add(1, std::memory_order_relaxed); }
 
     const float* hin = w.hT;
     size_t hin_stride = MH;
@@ -110,10 +111,14 @@ pt_status tc_forward(Call& k) {
             p.row_kvoff = w.meta.row_kvoff; p.row_pos = w.meta.row_pos; p.cs = m->rope_cos(); p.sn = m->rope_sin();
             p.nq = g.heads; p.nkv = g.kv_heads; p.dh = m->dh; p.ps = c->ps;
             int bn = gemm_bn(p.N, M, T);
+            ProfScope ps(m, st, 1);
             if ((s = launch_gemm(EPI_QKV, bn, ta_h, wm[l].m[0][bn == 256], p, st)) != PT_OK) return s;
         }
-        if (k.decode) s = launch_decode_attn(k, q, pool_l, o);
-        else s = launch_flash_prefill(k, q, pool_l, o);
+        {
+            ProfScope ps(m, st, 0);
+            if (k.decode) s = launch_decode_attn(k, q, pool_l, o);
+            else s = launch_flash_prefill(k, q, pool_l, o);
+        }
         if (s != PT_OK) return s;
         {   // output projection + residual; emits the operand and statistics of RMSNorm-2
             GemmP p = base;
@@ -122,6 +127,7 @@ pt_status tc_forward(Call& k) {
             p.hb_out = hb; p.gain = m->gain(1, l);
             p.ssq_out = w.ssq; p.ssq_out_tstride = (size_t)M * tiles; p.ssq_out_tiles = tiles;
             int bn = gemm_bn(p.N, M, T);
+            ProfScope ps(m, st, 2);
             if ((s = launch_gemm(EPI_RESID, bn, ta_o, wm[l].m[1][bn == 256], p, st)) != PT_OK) return s;
             ssq_tstride = (size_t)M * tiles;
         }
@@ -132,6 +138,7 @@ pt_status tc_forward(Call& k) {
             p.ssq_in = w.ssq; p.ssq_in_tstride = ssq_tstride; p.ssq_tiles = tiles;
             p.z_out = z;
             int bn = gemm_bn(p.N, M, T);
+            ProfScope ps(m, st, 3);
             if ((s = launch_gemm(EPI_SWIGLU, bn, ta_h, wm[l].m[2][bn == 256], p, st)) != PT_OK) return s;
         }
         {   // down projection + residual (+ track-sync when the layer closes a track block)
@@ -154,6 +161,7 @@ pt_status tc_forward(Call& k) {
                 hin = w.hT; hin_stride = MH;
             }
             int bn = gemm_bn(p.N, M, p.T);
+            ProfScope ps(m, st, sync ? 5 : 4);
             if ((s = launch_gemm(EPI_RESID, bn, ta_z, wm[l].m[3][bn == 256], p, st)) != PT_OK) return s;
         }
         tap_copy(k, l, 1, hin, hin_stride);

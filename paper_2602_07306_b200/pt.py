@@ -59,6 +59,8 @@ _PROTOS = {
     "pt_decode_step": (_I32, [_P, _P, _P, _I64, _I32, C.POINTER(_I32), _P, _P, _SZ, _P]),
     "pt_set_debug_tap": (_I32, [_P, _I32, _P]),
     "pt_device_status": (_I32, [_P, _P, C.POINTER(_I32), C.POINTER(_I32)]),
+    "pt_profile_enable": (_I32, [_P, _I32]),
+    "pt_profile_read": (_I32, [_P, C.POINTER(C.c_float), C.POINTER(_I64)]),
     "pt_launch_count": (_I64, []),
     "pt_kernel_gemm_bf16": (_I32, [_P, _P, _P, _I32, _I32, _I32, _I32, _I32, _I32, _P, _P]),
     "pt_last_error": (C.c_char_p, []),
@@ -228,6 +230,19 @@ class Model:
             check(lib().pt_decode_step(self.h, cache.h, x.data_ptr(), stride, B, pids, out.data_ptr(),
                                        ws.data_ptr(), ws.numel(), self._stream()))
         return out
+
+    PROF_NAMES = ("attention", "gemm_qkv", "gemm_out", "gemm_gate_up", "gemm_down", "gemm_down_sync", "other")
+
+    def profile(self, on: bool) -> None:
+        check(lib().pt_profile_enable(self.h, int(on)))
+
+    def profile_read(self) -> dict:
+        """Device milliseconds and launches per kernel category since the last read."""
+        ms = (C.c_float * 7)()
+        n = (_I64 * 7)()
+        with self.torch.cuda.device(self.device):
+            check(lib().pt_profile_read(self.h, ms, n))
+        return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(self.PROF_NAMES)}
 
     def device_status(self) -> tuple[int, int]:
         code, detail = _I32(), _I32()
