@@ -24,6 +24,28 @@ extern "C" {
 pt_status pt_kernel_gemm_bf16(const void* a, const void* w, void* c, int32_t T, int32_t M, int32_t N,
                               int32_t K, int32_t bn, int32_t fold_tracks, void* status, void* stream);
 
+/* Split-KV decode attention over the paged per-track KV cache (one new token per sequence, the
+ * attention of a track layer during decode: every query head of every track attends to its KV
+ * head's cached keys, tracks never read each other's cache between syncs - Section 2.2):
+ *   out[t][b][h] = softmax_j( q[t][b][h] . K[t][b][h / G][j] / sqrt(dh) ) V[t][b][h / G][j],
+ *   j < kv_len[b], G = nq / nkv.
+ *   q, out        device bf16 [T][B][nq*dh]
+ *   pool_l        device bf16: one layer's slabs, track t at pool_l + t*pool_track_stride elements,
+ *                 each [num_pages][K|V][nkv][ps][dh]
+ *   block_table   device int32 [B][maxp]: page of positions i*ps .. of sequence b
+ *   kv_len        host int32 [B] (>= 1): keys to attend to
+ *   scratch       device, 256-byte aligned, >= pt_kernel_decode_attn_scratch_bytes: holds the
+ *                 split plan and the per-range partial results; contents need not be kept
+ *   status        device int32[16], zeroed by the caller; PT_ERR_DEVICE_BOUNDS is recorded there
+ *                 when a page id is outside [0, num_pages)
+ * dh in {32, 64, 128}, nq/nkv <= 8.  Asynchronous on `stream`; kv_len is consumed before return. */
+pt_status pt_kernel_decode_attn_scratch_bytes(int32_t T, int32_t B, int32_t nq, int32_t dh, size_t* bytes);
+pt_status pt_kernel_decode_attn(const void* q, const void* pool_l, int64_t pool_track_stride,
+                                const int32_t* block_table, int32_t maxp, const int32_t* kv_len,
+                                int32_t T, int32_t B, int32_t nq, int32_t nkv, int32_t dh, int32_t ps,
+                                int32_t num_pages, void* out, void* scratch, size_t scratch_bytes,
+                                void* status, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

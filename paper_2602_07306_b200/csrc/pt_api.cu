@@ -25,7 +25,6 @@ void set_error(const char* fmt, ...) {
 #define PT_CUDA(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) { \
     pt::set_error("%s failed: %s", #call, cudaGetErrorString(e_)); return PT_ERR_CUDA; } } while (0)
 
-constexpr int kMaxSplits = 16;            // upper bound of KV splits per sequence in decode
 
 static size_t meta_bytes(int64_t M, int B, int maxp) {
     size_t b = 0;
@@ -59,6 +58,37 @@ static size_t carve(const pt_model* m, int64_t M, int B, int maxp, char* base, W
         (void)meta;
     }
     return off;
+}
+
+void plan_decode_splits(const int32_t* lens, int B, int ps, int64_t units, int32_t* items, int32_t* nsplit,
+                        int* n_items_out, int* max_splits_out) {
+    int n_items = 0, max_splits = 1;
+    int64_t total_keys = 0;
+    for (int b = 0; b < B; ++b) total_keys += lens[b];
+    // aim for >= 4 key ranges per SM over (tracks, kv heads, ranges); never split below 256 keys
+    int64_t want_items = std::max<int64_t>(B, (148 * 4 + units - 1) / units);
+    int64_t chunk = std::max<int64_t>(256, (total_keys + want_items - 1) / want_items);
+    chunk = (chunk + ps - 1) / ps * ps;
+    std::vector<int> order(B);
+    for (int b = 0; b < B; ++b) order[b] = b;
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b2) { return lens[a] > lens[b2]; });
+    for (int b : order) {
+        int ns = (int)std::min<int64_t>(kMaxSplits, (lens[b] + chunk - 1) / chunk);
+        ns = std::max(ns, 1);
+        int64_t per = ((lens[b] + ns - 1) / ns + ps - 1) / ps * ps;
+        per = std::max<int64_t>(per, ps);
+        ns = (int)std::max<int64_t>(1, (lens[b] + per - 1) / per);
+        nsplit[b] = ns;
+        max_splits = std::max(max_splits, ns);
+        for (int s2 = 0; s2 < ns; ++s2) {
+            int32_t* it = items + (size_t)n_items * 4;
+            it[0] = b; it[1] = (int32_t)(s2 * per);
+            it[2] = (int32_t)std::min<int64_t>(per, lens[b] - s2 * per); it[3] = s2;
+            ++n_items;
+        }
+    }
+    *n_items_out = n_items;
+    *max_splits_out = max_splits;
 }
 
 }  // namespace pt
@@ -394,34 +424,8 @@ static pt_status forward(pt_model* m, pt_kv_cache* c, const void* x, int64_t x_s
             h_kvoff[r] = slab_offset(c, s.pages[pos / c->ps], 0, 0, pos % c->ps);
         }
     }
-    // decode split plan: key ranges are whole pages; longest sequences first so the tail of
-    // the grid is made of short items
     int n_items = 0, max_splits = 1;
-    if (decode) {
-        int64_t total_keys = 0;
-        for (int b = 0; b < B; ++b) total_keys += h_len[b];
-        // aim for >= 4 items per SM over (T, kv_heads, items); never split below 256 keys
-        int64_t units = (int64_t)g.T * g.kv_heads;
-        int64_t want_items = std::max<int64_t>(B, (148 * 4 + units - 1) / units);
-        int64_t chunk = std::max<int64_t>(256, (total_keys + want_items - 1) / want_items);
-        chunk = (chunk + c->ps - 1) / c->ps * c->ps;
-        std::vector<int> order(B);
-        for (int b = 0; b < B; ++b) order[b] = b;
-        std::stable_sort(order.begin(), order.end(), [&](int a, int b2) { return h_len[a] > h_len[b2]; });
-        for (int b : order) {
-            int ns = (int)std::min<int64_t>(kMaxSplits, (h_len[b] + chunk - 1) / chunk);
-            int64_t per = ((h_len[b] + ns - 1) / ns + c->ps - 1) / c->ps * c->ps;
-            ns = (int)((h_len[b] + per - 1) / per);
-            h_nsp[b] = ns;
-            max_splits = std::max(max_splits, ns);
-            for (int s2 = 0; s2 < ns; ++s2) {
-                int32_t* it = h_items + (size_t)n_items * 4;
-                it[0] = b; it[1] = (int32_t)(s2 * per);
-                it[2] = (int32_t)std::min<int64_t>(per, h_len[b] - s2 * per); it[3] = s2;
-                ++n_items;
-            }
-        }
-    }
+    if (decode) plan_decode_splits(h_len, B, c->ps, (int64_t)g.T * g.kv_heads, h_items, h_nsp, &n_items, &max_splits);
     cudaStream_t st = (cudaStream_t)stream;
     PT_CUDA(cudaMemcpyAsync(db, hb, mb, cudaMemcpyHostToDevice, st));
     k.w.meta.row_kvoff = (const int64_t*)(db + o_kvoff);

@@ -17,6 +17,7 @@ namespace pt {
 
 constexpr int kStatusWords = 16;          // device status word block (int32 each)
 constexpr int kSsqTile = 128;             // columns covered by one partial sum of squares
+constexpr int kMaxSplits = 16;            // upper bound of KV key ranges per sequence in decode
 
 // Location codes written next to PT_ERR_DEVICE_* in the status block.
 enum : int {
@@ -136,6 +137,11 @@ struct ProfScope {
     }
     ~ProfScope() { if (idx >= 0) cudaEventRecord(m->prof_ev[idx].b, st); }
 };
+
+// Split-KV plan of a decode step (host): key ranges are whole pages, longest sequences first.
+// items gets 4 ints per range (batch row, first key, key count, range index); nsplit one per row.
+void plan_decode_splits(const int32_t* lens, int B, int ps, int64_t units, int32_t* items, int32_t* nsplit,
+                        int* n_items, int* max_splits);
 
 // pt_simt.cu
 pt_status simt_forward(Call& k);

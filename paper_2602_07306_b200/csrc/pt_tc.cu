@@ -194,3 +194,86 @@ extern "C" pt_status pt_kernel_gemm_bf16(const void* a, const void* w, void* c, 
     if (e != cudaSuccess) { set_error("kernel launch failed: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
     return PT_OK;
 }
+
+namespace pt {
+
+// Scratch layout of the kernel-level decode attention: plan first, partials after.
+struct DecodeScratch { size_t o_items, o_nsplit, o_len, o_part, total; };
+static DecodeScratch decode_scratch_layout(int T, int B, int nq, int dh) {
+    DecodeScratch d{};
+    size_t off = 0;
+    auto take = [&](size_t b) { size_t o = off; off += align_up(b, 256); return o; };
+    d.o_items = take((size_t)B * kMaxSplits * 16);
+    d.o_nsplit = take((size_t)B * 4);
+    d.o_len = take((size_t)B * 4);
+    d.o_part = take((size_t)T * B * kMaxSplits * nq * (dh + 2) * 4);
+    d.total = off;
+    return d;
+}
+
+// Shared by the caller-scratch and the static-scratch entry points.
+pt_status decode_attn_with_scratch(const void* q, const void* pool_l, int64_t pool_track_stride,
+                                   const int32_t* block_table, int32_t maxp, const int32_t* kv_len,
+                                   int32_t T, int32_t B, int32_t nq, int32_t nkv, int32_t dh, int32_t ps,
+                                   int32_t num_pages, void* out, char* scratch, void* status, cudaStream_t st) {
+    DecodeScratch d = decode_scratch_layout(T, B, nq, dh);
+    std::vector<int32_t> host((d.o_part) / 4, 0);
+    int32_t* items = host.data() + d.o_items / 4;
+    int32_t* nsplit = host.data() + d.o_nsplit / 4;
+    int32_t* lens = host.data() + d.o_len / 4;
+    for (int b = 0; b < B; ++b) lens[b] = kv_len[b];
+    int n_items = 0, max_splits = 1;
+    plan_decode_splits(lens, B, ps, (int64_t)T * nkv, items, nsplit, &n_items, &max_splits);
+    cudaError_t e = cudaMemcpyAsync(scratch, host.data(), d.o_part, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) { set_error("cudaMemcpyAsync: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
+    AttnP p{};
+    p.q = (const __nv_bfloat16*)q; p.pool_l = (const __nv_bfloat16*)pool_l; p.pool_tstride = pool_track_stride;
+    p.o = (__nv_bfloat16*)out; p.bt = block_table; p.maxp = maxp; p.kvlen = (const int32_t*)(scratch + d.o_len);
+    p.B = B; p.S = 1; p.M = B; p.nq = nq; p.nkv = nkv; p.ps = ps; p.num_pages = num_pages;
+    p.scale_log2 = 1.4426950408889634f / sqrtf((float)dh);
+    p.status = (int*)status;
+    p.items = (const int32_t*)(scratch + d.o_items); p.nsplit = (const int32_t*)(scratch + d.o_nsplit);
+    p.part = (float*)(scratch + d.o_part); p.max_splits = kMaxSplits;
+    pt_status s = launch_decode_attn_p(p, T, dh, n_items, max_splits, st);
+    if (s != PT_OK) return s;
+    e = cudaGetLastError();
+    if (e != cudaSuccess) { set_error("kernel launch failed: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
+    return PT_OK;
+}
+
+pt_status decode_attn_check_args(const void* q, const void* pool_l, const int32_t* block_table, int32_t maxp,
+                                 const int32_t* kv_len, int32_t T, int32_t B, int32_t nq, int32_t nkv, int32_t dh,
+                                 int32_t ps, int32_t num_pages, const void* out, const void* status) {
+    if (!q || !pool_l || !block_table || !kv_len || !out || !status) { set_error("null argument"); return PT_ERR_INVALID_ARG; }
+    if (T < 1 || B < 1 || nq < 1 || nkv < 1 || nq % nkv || nq / nkv > 8 || maxp < 1 || num_pages < 1) { set_error("bad sizes"); return PT_ERR_INVALID_ARG; }
+    if (dh != 32 && dh != 64 && dh != 128) { set_error("head_dim %d not in {32, 64, 128}", dh); return PT_ERR_UNSUPPORTED; }
+    if (ps < 8 || ps > 64 || ps % 8) { set_error("page size must be a multiple of 8 in [8, 64]"); return PT_ERR_INVALID_ARG; }
+    for (int b = 0; b < B; ++b)
+        if (kv_len[b] < 1 || (int64_t)kv_len[b] > (int64_t)maxp * ps) { set_error("kv_len[%d] = %d outside [1, maxp*ps]", b, kv_len[b]); return PT_ERR_INVALID_ARG; }
+    return PT_OK;
+}
+
+}  // namespace pt
+
+extern "C" pt_status pt_kernel_decode_attn_scratch_bytes(int32_t T, int32_t B, int32_t nq, int32_t dh, size_t* bytes) {
+    using namespace pt;
+    if (!bytes || T < 1 || B < 1 || nq < 1 || dh < 1) { set_error("bad argument"); return PT_ERR_INVALID_ARG; }
+    *bytes = decode_scratch_layout(T, B, nq, dh).total;
+    return PT_OK;
+}
+
+extern "C" pt_status pt_kernel_decode_attn(const void* q, const void* pool_l, int64_t pool_track_stride,
+                                           const int32_t* block_table, int32_t maxp, const int32_t* kv_len,
+                                           int32_t T, int32_t B, int32_t nq, int32_t nkv, int32_t dh, int32_t ps,
+                                           int32_t num_pages, void* out, void* scratch, size_t scratch_bytes,
+                                           void* status, void* stream) {
+    using namespace pt;
+    pt_status s = decode_attn_check_args(q, pool_l, block_table, maxp, kv_len, T, B, nq, nkv, dh, ps, num_pages, out, status);
+    if (s != PT_OK) return s;
+    if (!scratch) { set_error("null scratch"); return PT_ERR_INVALID_ARG; }
+    if ((uintptr_t)scratch % 256) { set_error("scratch must be 256-byte aligned"); return PT_ERR_MISALIGNED; }
+    size_t need = decode_scratch_layout(T, B, nq, dh).total;
+    if (scratch_bytes < need) { set_error("scratch: %zu < %zu bytes", scratch_bytes, need); return PT_ERR_BUFFER_TOO_SMALL; }
+    return decode_attn_with_scratch(q, pool_l, pool_track_stride, block_table, maxp, kv_len, T, B, nq, nkv, dh, ps,
+                                    num_pages, out, (char*)scratch, status, (cudaStream_t)stream);
+}

@@ -38,6 +38,23 @@ struct GemmP {
     float* ssq_out; size_t ssq_out_tstride; int ssq_out_tiles;
 };
 
+// Arguments shared by the attention kernels.
+struct AttnP {
+    const __nv_bfloat16* q;        // [T][M][nq*dh]
+    const __nv_bfloat16* pool_l;   // KV slab of this layer, track 0
+    int64_t pool_tstride;
+    __nv_bfloat16* o;              // [T][M][nq*dh]
+    const int32_t* bt; int maxp;
+    const int32_t* kvlen;          // [B] keys cached per sequence, this call's tokens included
+    int B, S, M, nq, nkv, ps, num_pages;
+    float scale_log2;              // log2(e) / sqrt(dh)
+    int* status;
+    // decode
+    const int32_t* items; const int32_t* nsplit; float* part; int max_splits;
+};
+
+pt_status launch_decode_attn_p(const AttnP& p, int T, int dh, int n_items, int max_splits, cudaStream_t st);
+
 pt_status make_map_bf16(CUtensorMap* out, const void* base, int64_t k, int64_t rows, int64_t tracks, int box_rows);
 int gemm_bn(int N, int M, int T);
 pt_status launch_gemm(int epi, int bn, const CUtensorMap& ta, const CUtensorMap& tb, GemmP p, cudaStream_t st);

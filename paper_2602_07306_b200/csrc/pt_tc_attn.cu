@@ -55,19 +55,6 @@ template <int DH> __device__ __forceinline__ uint32_t tile_off(int row, int chun
     return (uint32_t)(row * (DH * 2) + ((chunk ^ sw) << 4));
 }
 
-struct AttnP {
-    const __nv_bfloat16* q;        // [T][M][nq*dh]
-    const __nv_bfloat16* pool_l;   // KV slab of this layer, track 0
-    int64_t pool_tstride;
-    __nv_bfloat16* o;              // [T][M][nq*dh]
-    const int32_t* bt; int maxp;
-    const int32_t* kvlen;          // [B] keys cached per sequence, this call's tokens included
-    int B, S, M, nq, nkv, ps, num_pages;
-    float scale_log2;              // log2(e) / sqrt(dh)
-    int* status;
-    // decode
-    const int32_t* items; const int32_t* nsplit; float* part; int max_splits;
-};
 
 // Stage `rows` keys starting at key `key0` of sequence b (K and V of one KV head) into a tile.
 // Keys at or beyond `key_end` are zero-filled.
@@ -406,7 +393,7 @@ AttnP make_params(Call& k, const __nv_bfloat16* q, const __nv_bfloat16* pool_l, 
     p.B = k.B; p.S = k.S; p.M = k.M; p.nq = g.heads; p.nkv = g.kv_heads; p.ps = k.c->ps; p.num_pages = k.c->num_pages;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)k.m->dh);
     p.status = k.m->status();
-    p.items = k.items; p.nsplit = k.nsplit; p.part = k.w.part; p.max_splits = 16;
+    p.items = k.items; p.nsplit = k.nsplit; p.part = k.w.part; p.max_splits = kMaxSplits;
     return p;
 }
 
@@ -433,19 +420,22 @@ pt_status launch_flash_prefill(Call& k, const __nv_bfloat16* q, const __nv_bfloa
     return PT_OK;
 }
 
-pt_status launch_decode_attn(Call& k, const __nv_bfloat16* q, const __nv_bfloat16* pool_l, __nv_bfloat16* o) {
-    AttnP p = make_params(k, q, pool_l, o);
-    const int dh = k.m->dh;
-    dim3 grid(k.n_items, p.nkv, k.m->cfg.T);
+pt_status launch_decode_attn_p(const AttnP& p, int T, int dh, int n_items, int max_splits, cudaStream_t st) {
+    dim3 grid(n_items, p.nkv, T);
     const int smem = std::max(3 * 2 * kTileKeys * dh * 2, 4 * 8 * (dh + 2) * 4);
     pt_status s = PT_OK;
 #define GO(DH_) { static bool done = false; if (!done) { if ((s = set_smem(k_decode_attn<DH_>, smem)) != PT_OK) return s; done = true; } \
-                  k_decode_attn<DH_><<<grid, kThreads, smem, k.st>>>(p); \
-                  if (k.max_splits > 1) { k_decode_combine<DH_><<<dim3((k.B * p.nq * 32 + 127) / 128, k.m->cfg.T), 128, 0, k.st>>>(p); g_launches.fetch_add(1, std::memory_order_relaxed); } }
+                  k_decode_attn<DH_><<<grid, kThreads, smem, st>>>(p); \
+                  if (max_splits > 1) { k_decode_combine<DH_><<<dim3((p.B * p.nq * 32 + 127) / 128, T), 128, 0, st>>>(p); g_launches.fetch_add(1, std::memory_order_relaxed); } }
     if (dh == 32) GO(32) else if (dh == 64) GO(64) else GO(128)
 #undef GO
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return PT_OK;
+}
+
+pt_status launch_decode_attn(Call& k, const __nv_bfloat16* q, const __nv_bfloat16* pool_l, __nv_bfloat16* o) {
+    AttnP p = make_params(k, q, pool_l, o);
+    return launch_decode_attn_p(p, k.m->cfg.T, k.m->dh, k.n_items, k.max_splits, k.st);
 }
 
 }  // namespace pt

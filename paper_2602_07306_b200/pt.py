@@ -63,6 +63,9 @@ _PROTOS = {
     "pt_profile_read": (_I32, [_P, C.POINTER(C.c_float), C.POINTER(_I64)]),
     "pt_launch_count": (_I64, []),
     "pt_kernel_gemm_bf16": (_I32, [_P, _P, _P, _I32, _I32, _I32, _I32, _I32, _I32, _P, _P]),
+    "pt_kernel_decode_attn_scratch_bytes": (_I32, [_I32, _I32, _I32, _I32, C.POINTER(_SZ)]),
+    "pt_kernel_decode_attn": (_I32, [_P, _P, _I64, _P, _I32, C.POINTER(_I32), _I32, _I32, _I32, _I32, _I32, _I32, _I32,
+                                     _P, _P, _SZ, _P, _P]),
     "pt_last_error": (C.c_char_p, []),
 }
 EXPORTS = tuple(_PROTOS)
@@ -317,3 +320,26 @@ def kernel_gemm_bf16(a, w, bn: int = 0, fold_tracks: bool = False):
         check(lib().pt_kernel_gemm_bf16(a.data_ptr(), w.data_ptr(), c.data_ptr(), T, M, N, K, bn, int(fold_tracks),
                                         status.data_ptr(), torch.cuda.current_stream().cuda_stream))
     return c, status
+
+
+def kernel_decode_attn(q, pool_l, block_table, kv_len, *, nq, nkv, dh, ps, scratch=None):
+    """q bf16 [T, B, nq*dh]; pool_l bf16 [T, pages, 2, nkv, ps, dh]; block_table int32 [B, maxp] (CUDA);
+    kv_len: host ints [B].  Returns (out bf16 [T, B, nq*dh], status int32[16])."""
+    import torch
+    T, B, _ = q.shape
+    pages = pool_l.shape[1]
+    assert q.is_contiguous() and pool_l.is_contiguous() and block_table.is_contiguous()
+    assert q.dtype == pool_l.dtype == torch.bfloat16 and block_table.dtype == torch.int32
+    out = torch.empty_like(q)
+    status = torch.zeros(16, dtype=torch.int32, device=q.device)
+    n = _SZ()
+    check(lib().pt_kernel_decode_attn_scratch_bytes(T, B, nq, dh, C.byref(n)))
+    if scratch is None:
+        scratch = torch.empty(n.value, dtype=torch.uint8, device=q.device)
+    lens, plens = _i32arr(kv_len)
+    with torch.cuda.device(q.device):
+        check(lib().pt_kernel_decode_attn(q.data_ptr(), pool_l.data_ptr(), pool_l.stride(0), block_table.data_ptr(),
+                                          block_table.shape[1], plens, T, B, nq, nkv, dh, ps, pages, out.data_ptr(),
+                                          scratch.data_ptr(), scratch.numel(), status.data_ptr(),
+                                          torch.cuda.current_stream().cuda_stream))
+    return out, status

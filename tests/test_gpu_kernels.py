@@ -39,3 +39,63 @@ def test_gemm_bf16_matches_definition(T, M, N, K, bn, fold):
     got = c.cpu().numpy().astype(np.float64)
     err = np.abs(got - ref).max() / np.abs(ref).max()
     assert err <= 2e-6 * np.sqrt(K * (T if fold else 1)), f"max-rel {err:.3e}"     # fp32 accumulation of exact bf16 products
+
+
+def decode_case(T, B, nq, nkv, dh, ps, lens, seed):
+    """Random paged cache + queries; returns torch inputs and the float64 oracle result
+    (oracle.attention on the gathered keys, one sequence and track at a time)."""
+    import torch
+    from oracle import pt_oracle as O
+    rng = np.random.default_rng(seed)
+    maxp = max(-(-int(n) // ps) for n in lens)
+    pages = sum(-(-int(n) // ps) for n in lens) + 2
+    perm = I.free_list_permutation(pages, seed=seed)
+    bt = np.zeros((B, maxp), np.int32)
+    nxt = 0
+    for b, n in enumerate(lens):
+        k = -(-int(n) // ps)
+        bt[b, :k] = perm[nxt:nxt + k]
+        nxt += k
+    pool = I.round_to_bf16(rng.standard_normal((T, pages, 2, nkv, ps, dh), dtype=np.float32))
+    q = I.round_to_bf16(rng.standard_normal((T, B, nq * dh), dtype=np.float32))
+    ref = np.zeros((T, B, nq * dh))
+    for t in range(T):
+        for b, n in enumerate(lens):
+            pos = np.arange(int(n))
+            k = pool[t, bt[b, pos // ps], 0, :, pos % ps, :].astype(np.float64)       # [n, nkv, dh]
+            v = pool[t, bt[b, pos // ps], 1, :, pos % ps, :].astype(np.float64)
+            o = O.attention(q[t, b].reshape(1, nq, dh).astype(np.float64), k, v, np.array([int(n) - 1]))
+            ref[t, b] = o.reshape(-1)
+    dev = lambda a, dt: torch.from_numpy(a).cuda().to(dt).contiguous()
+    return dev(q, torch.bfloat16), dev(pool, torch.bfloat16), dev(bt, torch.int32), ref
+
+
+@pytest.mark.parametrize("T,B,nq,nkv,dh,ps,lens", [
+    (2, 3, 2, 2, 128, 16, [1, 17, 64]),                 # single token, page tails, exactly one tile
+    (1, 2, 8, 2, 64, 16, [300, 1023]),                  # GQA 4:1, several key ranges per sequence
+    (2, 4, 4, 1, 128, 16, [513, 4097, 2048, 15]),       # ragged, long, GQA 4:1
+    (1, 2, 4, 4, 32, 8, [100, 37]),                     # small heads, 8-token pages
+    (3, 2, 16, 2, 128, 32, [700, 90]),                  # GQA 8:1, 32-token pages
+])
+def test_decode_attention_kernel_matches_oracle(T, B, nq, nkv, dh, ps, lens):
+    import torch
+    from paper_2602_07306_b200 import pt
+    q, pool, bt, ref = decode_case(T, B, nq, nkv, dh, ps, lens, seed=sum(lens))
+    out, status = pt.kernel_decode_attn(q, pool, bt, lens, nq=nq, nkv=nkv, dh=dh, ps=ps)
+    torch.cuda.synchronize()
+    assert status[:2].tolist() == [0, 0]
+    got = out.float().cpu().numpy().astype(np.float64)
+    d = np.abs(got - ref)
+    assert d.max() <= 2e-2 * np.abs(ref).max() and d.mean() <= 4e-3 * np.abs(ref).mean(), (d.max() / np.abs(ref).max(), d.mean() / np.abs(ref).mean())
+
+
+def test_decode_attention_kernel_reports_bad_page():
+    """A page id outside the pool is skipped and reported through the status word (no fault)."""
+    import torch
+    from paper_2602_07306_b200 import pt
+    q, pool, bt, _ = decode_case(1, 2, 2, 2, 64, 16, [40, 20], seed=3)
+    bt[1, 0] = pool.shape[1] + 5
+    out, status = pt.kernel_decode_attn(q, pool, bt, [40, 20], nq=2, nkv=2, dh=64, ps=16)
+    torch.cuda.synchronize()
+    assert status[0].item() == 8 and status[1].item() == 7
+    assert torch.isfinite(out.float()).all()
