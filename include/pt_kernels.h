@@ -46,6 +46,34 @@ pt_status pt_kernel_decode_attn(const void* q, const void* pool_l, int64_t pool_
                                 int32_t num_pages, void* out, void* scratch, size_t scratch_bytes,
                                 void* status, void* stream);
 
+/* The same decode attention for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of pt_kernel_decode_attn.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a region that is being
+ * captured into a CUDA graph, in a real-time or serving loop that must not touch the allocator
+ * after start-up, or in a host program that handed all device memory to another component and
+ * has no pool of its own to carve a scratch buffer from.  Such a caller passes only inputs and
+ * outputs; the split plan and the per-range partial results live in a fixed array inside the
+ * library image (PT_STATIC_SCRATCH_BYTES, 8 MiB, resident on every GPU that loads the library
+ * until the process exits).
+ *
+ *  - Arguments are those of pt_kernel_decode_attn without scratch / scratch_bytes; results are
+ *    identical to it.
+ *  - Problems whose scratch need (pt_kernel_decode_attn_scratch_bytes) exceeds
+ *    PT_STATIC_SCRATCH_BYTES are refused with PT_ERR_BUFFER_TOO_SMALL and nothing is launched.
+ *  - The first call on each device looks up the array's device address (no allocation, but a
+ *    driver query): make that first call before any stream capture begins.
+ *  - The entry point calls no cudaMalloc, cudaFree or any allocating library routine.
+ *  - All calls on a device share the one array, which keeps whatever the previous call left.
+ *    Nothing in it has to start at zero - every word a call reads it has written first - but
+ *    two calls that overlap on the GPU (different streams, or concurrent host threads) race on
+ *    it: serialise them on one stream. */
+#define PT_STATIC_SCRATCH_BYTES (8u << 20)
+pt_status pt_kernel_decode_attn_static(const void* q, const void* pool_l, int64_t pool_track_stride,
+                                       const int32_t* block_table, int32_t maxp, const int32_t* kv_len,
+                                       int32_t T, int32_t B, int32_t nq, int32_t nkv, int32_t dh, int32_t ps,
+                                       int32_t num_pages, void* out, void* status, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

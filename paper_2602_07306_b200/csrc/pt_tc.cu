@@ -277,3 +277,40 @@ extern "C" pt_status pt_kernel_decode_attn(const void* q, const void* pool_l, in
     return decode_attn_with_scratch(q, pool_l, pool_track_stride, block_table, maxp, kv_len, T, B, nq, nkv, dh, ps,
                                     num_pages, out, (char*)scratch, status, (cudaStream_t)stream);
 }
+
+// ---- decode attention with built-in scratch -------------------------------------------------
+// The array lives in the library image, once per device that loads it.  In host code its name
+// is only a handle: the device address comes from cudaGetSymbolAddress, looked up once per
+// device with that device current.
+static __device__ __align__(256) unsigned char g_static_scratch[PT_STATIC_SCRATCH_BYTES];
+
+namespace pt {
+constexpr int kMaxDevices = 64;
+static void* g_static_scratch_addr[kMaxDevices] = {};
+}
+
+extern "C" pt_status pt_kernel_decode_attn_static(const void* q, const void* pool_l, int64_t pool_track_stride,
+                                                  const int32_t* block_table, int32_t maxp, const int32_t* kv_len,
+                                                  int32_t T, int32_t B, int32_t nq, int32_t nkv, int32_t dh, int32_t ps,
+                                                  int32_t num_pages, void* out, void* status, void* stream) {
+    using namespace pt;
+    pt_status s = decode_attn_check_args(q, pool_l, block_table, maxp, kv_len, T, B, nq, nkv, dh, ps, num_pages, out, status);
+    if (s != PT_OK) return s;
+    size_t need = decode_scratch_layout(T, B, nq, dh).total;
+    if (need > PT_STATIC_SCRATCH_BYTES) {
+        set_error("problem needs %zu bytes of scratch, the built-in array holds %u: use pt_kernel_decode_attn with a caller buffer",
+                  need, (unsigned)PT_STATIC_SCRATCH_BYTES);
+        return PT_ERR_BUFFER_TOO_SMALL;
+    }
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) { set_error("cudaGetDevice: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
+    if (!g_static_scratch_addr[dev]) {
+        void* ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess || !ptr) { set_error("cudaGetSymbolAddress: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
+        g_static_scratch_addr[dev] = ptr;
+    }
+    return decode_attn_with_scratch(q, pool_l, pool_track_stride, block_table, maxp, kv_len, T, B, nq, nkv, dh, ps,
+                                    num_pages, out, (char*)g_static_scratch_addr[dev], status, (cudaStream_t)stream);
+}

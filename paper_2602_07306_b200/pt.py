@@ -66,6 +66,8 @@ _PROTOS = {
     "pt_kernel_decode_attn_scratch_bytes": (_I32, [_I32, _I32, _I32, _I32, C.POINTER(_SZ)]),
     "pt_kernel_decode_attn": (_I32, [_P, _P, _I64, _P, _I32, C.POINTER(_I32), _I32, _I32, _I32, _I32, _I32, _I32, _I32,
                                      _P, _P, _SZ, _P, _P]),
+    "pt_kernel_decode_attn_static": (_I32, [_P, _P, _I64, _P, _I32, C.POINTER(_I32), _I32, _I32, _I32, _I32, _I32, _I32, _I32,
+                                            _P, _P, _P]),
     "pt_last_error": (C.c_char_p, []),
 }
 EXPORTS = tuple(_PROTOS)
@@ -342,4 +344,22 @@ def kernel_decode_attn(q, pool_l, block_table, kv_len, *, nq, nkv, dh, ps, scrat
                                           block_table.shape[1], plens, T, B, nq, nkv, dh, ps, pages, out.data_ptr(),
                                           scratch.data_ptr(), scratch.numel(), status.data_ptr(),
                                           torch.cuda.current_stream().cuda_stream))
+    return out, status
+
+
+def kernel_decode_attn_static(q, pool_l, block_table, kv_len, *, nq, nkv, dh, ps, out=None, status=None):
+    """pt_kernel_decode_attn for callers that may not allocate device memory: the scratch is an
+    8 MiB array built into the library.  Pass preallocated ``out`` / ``status`` tensors to keep the
+    call itself free of allocations; calls on one device must not overlap on the GPU."""
+    import torch
+    T, B, _ = q.shape
+    if out is None:
+        out = torch.empty_like(q)
+    if status is None:
+        status = torch.zeros(16, dtype=torch.int32, device=q.device)
+    lens, plens = _i32arr(kv_len)
+    with torch.cuda.device(q.device):
+        check(lib().pt_kernel_decode_attn_static(q.data_ptr(), pool_l.data_ptr(), pool_l.stride(0), block_table.data_ptr(),
+                                                 block_table.shape[1], plens, T, B, nq, nkv, dh, ps, pool_l.shape[1],
+                                                 out.data_ptr(), status.data_ptr(), torch.cuda.current_stream().cuda_stream))
     return out, status
