@@ -242,6 +242,221 @@ k_flash_prefill(const AttnP p) {
 
 // ------------------------------------------------------------------------------------ decode
 
+// Merge the four warps' partial (max, sum, output) of the G query heads through shared memory
+// and store either the final output (one key range) or this range's partial.  All threads of
+// the CTA call it after a __syncthreads() that retired every use of `mg`.
+template <int DH>
+__device__ __forceinline__ void decode_merge_store(const AttnP& p, float* mg, float (*o)[4], float m_run, float l_run,
+                                                   int t, int b, int kvh, int split) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int G = p.nq / p.nkv;
+    const int g_lo = lane >> 2;
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+    if (g_lo < G) {                                           // per-warp partials: [warp][g][DH + 2] floats
+        float* dst = mg + ((size_t)warp * 8 + g_lo) * (DH + 2);
+        const int c = (lane & 3) * 2;
+#pragma unroll
+        for (int i = 0; i < DH / 8; ++i) { dst[i * 8 + c] = o[i][0]; dst[i * 8 + c + 1] = o[i][1]; }
+        if ((lane & 3) == 0) { dst[DH] = m_run; dst[DH + 1] = l_run; }
+    }
+    __syncthreads();
+    const int ns = p.nsplit[b];
+    for (int idx = threadIdx.x; idx < G * DH; idx += kThreads) {
+        const int g = idx / DH, d = idx % DH;
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) M = fmaxf(M, mg[((size_t)w * 8 + g) * (DH + 2) + DH]);
+        float L = 0.f, acc = 0.f;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            const float* src = mg + ((size_t)w * 8 + g) * (DH + 2);
+            float f = src[DH] == -INFINITY ? 0.f : exp2f(src[DH] - M);
+            L += src[DH + 1] * f;
+            acc += src[d] * f;
+        }
+        const int head = kvh * G + g;
+        if (ns == 1) {
+            p.o[((size_t)t * p.M + b) * (size_t)(p.nq * DH) + (size_t)head * DH + d] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
+        } else {
+            float* dst = p.part + ((((size_t)t * p.B + b) * p.nq + head) * p.max_splits + split) * (DH + 2);
+            dst[d] = acc;
+            if (d == 0) { dst[DH] = M; dst[DH + 1] = L; }
+        }
+    }
+}
+
+// ---- TMA-fed decode attention (page size a multiple of 16, head_dim 64 or 128) ----------------
+// Each warp streams its own pages: lane 0 issues one tensor-map load per 128-byte-wide half of
+// the K and V blocks of a 16-token page (hardware 128-byte swizzle, so ldmatrix reads are
+// conflict-free) into the warp's private ring of kDecStages slots and waits on the slot's
+// mbarrier; no CTA-wide barrier is taken until the final merge.  Waits are bounded.
+constexpr int kDecStages = 3;
+constexpr uint32_t kDecSpin = 1u << 24;
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                 ::"r"(dst), "l"((uint64_t)map), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar)) : "memory");
+}
+
+// Byte offset of 16-byte chunk `chunk` of row `row` (0..15) inside one page block as the tensor
+// map lays it out: 128-byte-wide halves of 16 rows each, chunks XOR-swizzled with row % 8.
+template <int DH> __device__ __forceinline__ uint32_t page_off(int row, int chunk) {
+    return (uint32_t)((chunk >> 3) * 2048 + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
+}
+
+template <int DH>
+__global__ void __launch_bounds__(kThreads)
+k_decode_attn_tma(const __grid_constant__ CUtensorMap kvmap, const AttnP p) {
+    constexpr int PAGE_BYTES = 16 * DH * 2;                   // one K or V block of 16 tokens
+    constexpr int SLOT_BYTES = 2 * PAGE_BYTES;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint64_t* bars = (uint64_t*)(smem + 4 * kDecStages * SLOT_BYTES);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int32_t* item = p.items + (size_t)blockIdx.x * 4;
+    const int b = item[0], kstart = item[1], kcount = item[2], split = item[3];
+    const int kvh = blockIdx.y, t = blockIdx.z;
+    const int G = p.nq / p.nkv;
+    const int key_end = min(kstart + kcount, p.kvlen[b]);
+    const int npages = (key_end - kstart + 15) >> 4;          // 16-token groups of this key range
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 4 * kDecStages; ++i) mbar_init(&bars[i], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    uint8_t* ring = smem + warp * kDecStages * SLOT_BYTES;
+    uint64_t* wbar = bars + warp * kDecStages;
+    bool bad_page = false;
+    // lane 0: fetch the K and V blocks of local 16-token group `g` into slot g % kDecStages
+    auto issue = [&](int gidx) {
+        const int key0 = kstart + gidx * 16;
+        int page = p.bt[(size_t)b * p.maxp + key0 / p.ps];
+        if (page < 0 || page >= p.num_pages) { bad_page = true; page = 0; }
+        const int slot = (gidx >> 2) % kDecStages;
+        const uint32_t dst = smem_u32(ring + slot * SLOT_BYTES);
+        const int row_k = ((page * 2 + 0) * p.nkv + kvh) * p.ps + key0 % p.ps;
+        const int row_v = row_k + p.nkv * p.ps;
+        mbar_expect_tx(&wbar[slot], SLOT_BYTES);
+#pragma unroll
+        for (int h = 0; h < DH / 64; ++h) {
+            tma_load_3d(dst + h * 2048, &kvmap, &wbar[slot], h * 64, row_k, t);
+            tma_load_3d(dst + PAGE_BYTES + h * 2048, &kvmap, &wbar[slot], h * 64, row_v, t);
+        }
+    };
+
+    const int g_lo = lane >> 2;
+    const __nv_bfloat16* qrow = p.q + ((size_t)t * p.M + b) * (size_t)(p.nq * DH) + (size_t)(kvh * G) * DH;
+    uint32_t qf[DH / 16][4];
+    load_q_frags<DH>(qf, g_lo < G ? qrow + (size_t)g_lo * DH : nullptr, nullptr, lane);
+    float o[DH / 8][4];
+#pragma unroll
+    for (int i = 0; i < DH / 8; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+    float m_run = -INFINITY, l_run = 0.f;
+
+    // warp w owns local groups w, w + 4, w + 8, ...
+    if (lane == 0)
+        for (int s = 0; s < kDecStages; ++s) { int gi = warp + 4 * s; if (gi < npages) issue(gi); }
+    bool timed_out = false;
+    int it = 0;
+    for (int gi = warp; gi < npages; gi += 4, ++it) {
+        const int slot = it % kDecStages;
+        const uint32_t parity = (it / kDecStages) & 1;
+        bool ok = false;
+        for (uint32_t spin = 0; spin < kDecSpin; ++spin) if (mbar_try(&wbar[slot], parity)) { ok = true; break; }
+        if (!__all_sync(0xffffffffu, ok)) { timed_out = true; break; }
+        const uint32_t k_base = smem_u32(ring + slot * SLOT_BYTES), v_base = k_base + PAGE_BYTES;
+        const int key0 = kstart + gi * 16;
+        const int nvalid = key_end - key0;                    // >= 1
+        if (nvalid < 16) {                                    // tail of the sequence: unused slots may hold anything
+            for (int i = lane; i < (16 - nvalid) * (DH / 8); i += 32) {
+                int row = nvalid + i / (DH / 8), chunk = i % (DH / 8);
+                *reinterpret_cast<uint4*>(ring + slot * SLOT_BYTES + PAGE_BYTES + page_off<DH>(row, chunk)) = make_uint4(0, 0, 0, 0);
+            }
+            __syncwarp();
+        }
+        float s[2][4] = {};
+        {
+            const int row = (lane >> 4) * 8 + (lane & 7);
+            const int cofs = (lane >> 3) & 1;
+#pragma unroll
+            for (int ks = 0; ks < DH / 16; ++ks) {
+                uint32_t b0, b1, b2, b3;
+                ldsm_x4(k_base + page_off<DH>(row, ks * 2 + cofs), b0, b1, b2, b3);
+                mma_bf16(s[0], qf[ks], b0, b1);
+                mma_bf16(s[1], qf[ks], b2, b3);
+            }
+        }
+        float mx = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                int key = i * 8 + (lane & 3) * 2 + e;
+                float v = key < nvalid ? s[i][e] * p.scale_log2 : -INFINITY;
+                s[i][e] = v;
+                mx = fmaxf(mx, v);
+            }
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        const float mn = fmaxf(m_run, mx);
+        const float corr = exp2f(m_run - mn);
+        m_run = mn;
+        float sum = 0.f;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) { s[i][0] = exp2f(s[i][0] - mn); s[i][1] = exp2f(s[i][1] - mn); sum += s[i][0] + s[i][1]; }
+        l_run = l_run * corr + sum;
+        if (__any_sync(0xffffffffu, corr != 1.f)) {
+#pragma unroll
+            for (int i = 0; i < DH / 8; ++i) { o[i][0] *= corr; o[i][1] *= corr; }
+        }
+        uint32_t pf[4];
+        pf[0] = pack_bf16(s[0][0], s[0][1]); pf[1] = 0u;
+        pf[2] = pack_bf16(s[1][0], s[1][1]); pf[3] = 0u;
+        {
+            const int row = ((lane >> 3) & 1) * 8 + (lane & 7);
+            const int cofs = lane >> 4;
+#pragma unroll
+            for (int dc = 0; dc < DH / 16; ++dc) {
+                uint32_t b0, b1, b2, b3;
+                ldsm_x4_t(v_base + page_off<DH>(row, dc * 2 + cofs), b0, b1, b2, b3);
+                mma_bf16(o[dc * 2], pf, b0, b1);
+                mma_bf16(o[dc * 2 + 1], pf, b2, b3);
+            }
+        }
+        __syncwarp();                                         // every lane is done reading the slot
+        if (lane == 0) {
+            int gn = gi + 4 * kDecStages;
+            if (gn < npages) { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); issue(gn); }
+        }
+    }
+    if (timed_out) {
+        // give the copies this warp still has in flight a bounded chance to land, then give up
+        for (int s2 = 0; s2 < kDecStages; ++s2)
+            for (uint32_t spin = 0; spin < (1u << 16); ++spin) if (mbar_try(&wbar[s2], 0) || mbar_try(&wbar[s2], 1)) break;
+        if (lane == 0) report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_DECODE_PAGE);
+    }
+    if (bad_page) report(p.status, PT_ERR_DEVICE_BOUNDS, LOC_DECODE_PAGE);
+    __syncthreads();                                          // every warp has drained its ring
+    decode_merge_store<DH>(p, reinterpret_cast<float*>(smem), o, m_run, l_run, t, b, kvh, split);
+}
+
+
 template <int DH>
 __global__ void __launch_bounds__(kThreads)
 k_decode_attn(const AttnP p) {
@@ -321,41 +536,7 @@ k_decode_attn(const AttnP p) {
     cp_async_wait<0>();
     __syncthreads();                                          // tiles are dead: reuse shared memory for the merge
     if (bad_page && lane == 0) report(p.status, PT_ERR_DEVICE_BOUNDS, LOC_DECODE_PAGE);
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-    // per-warp partials: [warp][g][DH + 2] floats
-    float* mg = reinterpret_cast<float*>(smem);
-    if (g_lo < G) {
-        float* dst = mg + ((size_t)warp * 8 + g_lo) * (DH + 2);
-        const int c = (lane & 3) * 2;
-#pragma unroll
-        for (int i = 0; i < DH / 8; ++i) { dst[i * 8 + c] = o[i][0]; dst[i * 8 + c + 1] = o[i][1]; }
-        if ((lane & 3) == 0) { dst[DH] = m_run; dst[DH + 1] = l_run; }
-    }
-    __syncthreads();
-    const int ns = p.nsplit[b];
-    for (int idx = threadIdx.x; idx < G * DH; idx += kThreads) {
-        const int g = idx / DH, d = idx % DH;
-        float M = -INFINITY;
-#pragma unroll
-        for (int w = 0; w < 4; ++w) M = fmaxf(M, mg[((size_t)w * 8 + g) * (DH + 2) + DH]);
-        float L = 0.f, acc = 0.f;
-#pragma unroll
-        for (int w = 0; w < 4; ++w) {
-            const float* src = mg + ((size_t)w * 8 + g) * (DH + 2);
-            float f = src[DH] == -INFINITY ? 0.f : exp2f(src[DH] - M);
-            L += src[DH + 1] * f;
-            acc += src[d] * f;
-        }
-        const int head = kvh * G + g;
-        if (ns == 1) {
-            p.o[((size_t)t * p.M + b) * (size_t)(p.nq * DH) + (size_t)head * DH + d] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
-        } else {
-            float* dst = p.part + ((((size_t)t * p.B + b) * p.nq + head) * p.max_splits + split) * (DH + 2);
-            dst[d] = acc;
-            if (d == 0) { dst[DH] = M; dst[DH + 1] = L; }
-        }
-    }
+    decode_merge_store<DH>(p, reinterpret_cast<float*>(smem), o, m_run, l_run, t, b, kvh, split);
 }
 
 // Merge the key ranges of one (track, sequence, head): one warp each.
@@ -422,6 +603,21 @@ pt_status launch_flash_prefill(Call& k, const __nv_bfloat16* q, const __nv_bfloa
 
 pt_status launch_decode_attn_p(const AttnP& p, int T, int dh, int n_items, int max_splits, cudaStream_t st) {
     dim3 grid(n_items, p.nkv, T);
+    if (p.ps % 16 == 0 && (dh == 64 || dh == 128)) {
+        // tensor map over one layer's slabs: (head_dim, rows of a slab, track); a box is 16 tokens x 128 bytes
+        CUtensorMap kvmap;
+        pt_status s = make_map_bf16_strided(&kvmap, p.pool_l, dh, (int64_t)p.num_pages * 2 * p.nkv * p.ps, T,
+                                            p.pool_tstride * 2, 16);
+        if (s != PT_OK) return s;
+        const int smem = 1024 + 4 * kDecStages * 2 * 16 * dh * 2 + 4 * kDecStages * 8;
+#define GOT(DH_) { static bool done = false; if (!done) { if ((s = set_smem(k_decode_attn_tma<DH_>, smem)) != PT_OK) return s; done = true; } \
+                   k_decode_attn_tma<DH_><<<grid, kThreads, smem, st>>>(kvmap, p); \
+                   if (max_splits > 1) { k_decode_combine<DH_><<<dim3((p.B * p.nq * 32 + 127) / 128, T), 128, 0, st>>>(p); g_launches.fetch_add(1, std::memory_order_relaxed); } }
+        if (dh == 64) GOT(64) else GOT(128)
+#undef GOT
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        return PT_OK;
+    }
     const int smem = std::max(3 * 2 * kTileKeys * dh * 2, 4 * 8 * (dh + 2) * 4);
     pt_status s = PT_OK;
 #define GO(DH_) { static bool done = false; if (!done) { if ((s = set_smem(k_decode_attn<DH_>, smem)) != PT_OK) return s; done = true; } \

@@ -393,10 +393,15 @@ pt_status launch_t(const CUtensorMap& ta, const CUtensorMap& tb, GemmP p, cudaSt
 }  // namespace
 
 pt_status make_map_bf16(CUtensorMap* out, const void* base, int64_t k, int64_t rows, int64_t tracks, int box_rows) {
+    return make_map_bf16_strided(out, base, k, rows, tracks, k * 2 * rows, box_rows);
+}
+
+pt_status make_map_bf16_strided(CUtensorMap* out, const void* base, int64_t k, int64_t rows, int64_t tracks,
+                                int64_t track_stride_bytes, int box_rows) {
     EncodeFn enc = get_encode();
     if (!enc) { set_error("cuTensorMapEncodeTiled is not available from this driver"); return PT_ERR_CUDA; }
     cuuint64_t dims[3] = {(cuuint64_t)k, (cuuint64_t)rows, (cuuint64_t)tracks};
-    cuuint64_t strides[2] = {(cuuint64_t)k * 2, (cuuint64_t)k * 2 * (cuuint64_t)rows};
+    cuuint64_t strides[2] = {(cuuint64_t)k * 2, (cuuint64_t)track_stride_bytes};
     cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)std::min<int64_t>(box_rows, rows), 1};
     cuuint32_t es[3] = {1, 1, 1};
     CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,

@@ -1,0 +1,91 @@
+"""Time one kernel of the PT forward pass through its kernel-level C-ABI entry point.
+
+    python -m paper_2602_07306_b200.kbench decode --T 8 --B 64 --nq 8 --nkv 8 --dh 128 --len 2048
+    python -m paper_2602_07306_b200.kbench gemm --T 8 --M 32768 --N 3072 --K 1024 [--bn 256] [--fold]
+
+Prints one JSON line: average device time per launch (CUDA events on the launching stream,
+after warm-up) and the achieved GB/s (decode: K/V bytes read) or TFLOP/s (gemm).  Small cases of
+the same commands are what the ncu summaries under profiles/ were captured on.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import numpy as np
+import torch
+
+from paper_2602_07306_b200 import pt
+
+
+def decode(a):
+    dev = torch.device("cuda:0")
+    ps = a.ps
+    lens = [a.len] * a.B if a.ragged == 0 else np.random.default_rng(0).integers(a.ragged, a.len + 1, a.B).tolist()
+    maxp = max(-(-n // ps) for n in lens)
+    pages = sum(-(-n // ps) for n in lens)
+    g = torch.Generator(device=dev).manual_seed(0)
+    pool = torch.randn((a.T, pages, 2, a.nkv, ps, a.dh), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    q = torch.randn((a.T, a.B, a.nq * a.dh), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    perm = torch.randperm(pages, generator=torch.Generator().manual_seed(0)).to(torch.int32)
+    bt = torch.zeros((a.B, maxp), dtype=torch.int32)
+    nxt = 0
+    for b, n in enumerate(lens):
+        k = -(-n // ps)
+        bt[b, :k] = perm[nxt:nxt + k]
+        nxt += k
+    bt = bt.to(dev)
+    n = pt._SZ()
+    pt.check(pt.lib().pt_kernel_decode_attn_scratch_bytes(a.T, a.B, a.nq, a.dh, pt.C.byref(n)))
+    scratch = torch.empty(n.value, dtype=torch.uint8, device=dev)
+    for _ in range(a.warmup):
+        out, status = pt.kernel_decode_attn(q, pool, bt, lens, nq=a.nq, nkv=a.nkv, dh=a.dh, ps=ps, scratch=scratch)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(a.iters):
+        out, status = pt.kernel_decode_attn(q, pool, bt, lens, nq=a.nq, nkv=a.nkv, dh=a.dh, ps=ps, scratch=scratch)
+    e1.record()
+    torch.cuda.synchronize()
+    assert status[:2].tolist() == [0, 0]
+    ms = e0.elapsed_time(e1) / a.iters
+    byts = a.T * 2 * a.nkv * a.dh * 2 * sum(lens)
+    print(json.dumps({"kernel": "decode_attn", "ms": ms, "GBps": byts / ms / 1e6, "bytes": byts, "args": vars(a)}))
+
+
+def gemm(a):
+    dev = torch.device("cuda:0")
+    g = torch.Generator(device=dev).manual_seed(0)
+    A = torch.randn((a.T, a.M, a.K), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    W = (torch.randn((a.T, a.N, a.K), generator=g, device=dev, dtype=torch.float32) * 0.05).to(torch.bfloat16)
+    for _ in range(a.warmup):
+        c, status = pt.kernel_gemm_bf16(A, W, bn=a.bn, fold_tracks=a.fold)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(a.iters):
+        c, status = pt.kernel_gemm_bf16(A, W, bn=a.bn, fold_tracks=a.fold)
+    e1.record()
+    torch.cuda.synchronize()
+    assert status[:2].tolist() == [0, 0]
+    ms = e0.elapsed_time(e1) / a.iters
+    flops = 2.0 * a.T * a.M * a.N * a.K
+    print(json.dumps({"kernel": "gemm_bf16", "ms": ms, "TFLOPs": flops / ms / 1e9, "args": vars(a)}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    sub = ap.add_subparsers(dest="cmd", required=True)
+    d = sub.add_parser("decode")
+    for k, v in dict(T=8, B=64, nq=8, nkv=8, dh=128, len=2048, ps=16, ragged=0, iters=20, warmup=3).items():
+        d.add_argument("--" + k, type=int, default=v)
+    gm = sub.add_parser("gemm")
+    for k, v in dict(T=8, M=4096, N=3072, K=1024, bn=0, iters=20, warmup=3).items():
+        gm.add_argument("--" + k, type=int, default=v)
+    gm.add_argument("--fold", action="store_true")
+    a = ap.parse_args()
+    (decode if a.cmd == "decode" else gemm)(a)
+
+
+if __name__ == "__main__":
+    main()
