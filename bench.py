@@ -156,7 +156,7 @@ def run_decode(wl, dev, steps, warmup, barrier, rank):
     cache = model.new_cache(num_pages, ps)
     seq_ids = list(range(B))
     # fill the cache by real prefills of N(0,1) inputs, grouped by length, in bounded sub-batches
-    g = torch.Generator(device=dev).manual_seed(wl.seed + 1)
+    g = torch.Generator(device=dev).manual_seed(rank_batch_seed(wl.seed, rank))
     t_fill = time.time()
     order = np.argsort(-lens, kind="stable")
     i = 0
@@ -252,7 +252,7 @@ def run_prefill(wl, dev, steps, warmup, barrier, rank):
     pages = B * ((S + ps - 1) // ps)
     cache = model.new_cache(pages, ps)
     seq_ids = list(range(B))
-    g = torch.Generator(device=dev).manual_seed(wl.seed + 1)
+    g = torch.Generator(device=dev).manual_seed(rank_batch_seed(wl.seed, rank))
     x = torch.randn((wl.T, B, S, wl.hidden), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
     out = torch.empty((B, S, wl.hidden), dtype=torch.float32, device=dev)
 
@@ -371,6 +371,31 @@ def oracle_sample(wl, budget_s=20.0):
                             f"tokens/s scaled by {wl.D}/{wl.L}"), dt, cores
 
 
+# ------------------------------------------------------------------------------ ranks
+
+def rank_batch_seed(seed, rank):
+    """Seed of the inputs of one rank's batch: rank r owns sequences [r*B, (r+1)*B) of the job's
+    global batch, drawn from its own stream; the model weights are the same on every rank."""
+    return int(seed) + 1 + 7919 * int(rank)
+
+
+def aggregate_over_ranks(ms, tokens, e2e_tokens_per_s, world, device):
+    """Whole-job numbers of a weak-scaling run: every rank processed `tokens` tokens per step on
+    its own batch in `ms` device milliseconds (no data-path collective).  The job's step time is
+    the slowest rank's, the job's tokens are the sum; the same for the end-to-end leg.  Only
+    these three scalars cross ranks.  Returns (ms, total_tokens, e2e_tokens_per_s)."""
+    if world <= 1:
+        return float(ms), float(tokens), float(e2e_tokens_per_s)
+    import torch
+    import torch.distributed as dist
+    tmax = torch.tensor([float(ms), float(tokens) / float(e2e_tokens_per_s)], dtype=torch.float64, device=device)
+    dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+    toks = torch.tensor([float(tokens)], dtype=torch.float64, device=device)
+    dist.all_reduce(toks, op=dist.ReduceOp.SUM)
+    total = float(toks.item())
+    return float(tmax[0].item()), total, total / float(tmax[1].item())
+
+
 # ------------------------------------------------------------------------------ main
 
 def main():
@@ -424,19 +449,8 @@ def main():
 
     run = run_decode if wl.mode == "decode" else run_prefill
     r = run(wl, dev, a.steps, a.warmup, barrier, rank)
-    ms = r["ms"]
-    if world > 1:
-        tmax = torch.tensor([ms], device=dev)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms = float(tmax.item())
-        toks = torch.tensor([float(r["tokens"])], device=dev)
-        dist.all_reduce(toks, op=dist.ReduceOp.SUM)
-        total_tokens = float(toks.item())
-        e2e_t = torch.tensor([r["tokens"] / r["e2e"]["value"]], device=dev)
-        dist.all_reduce(e2e_t, op=dist.ReduceOp.MAX)
-        r["e2e"]["value"] = total_tokens / float(e2e_t.item())
-    else:
-        total_tokens = float(r["tokens"])
+    ms, total_tokens, e2e_value = aggregate_over_ranks(r["ms"], r["tokens"], r["e2e"]["value"], world, dev)
+    r["e2e"]["value"] = e2e_value
     extra = {}
     if world == 1 and a.extra:
         for name in [n for n in a.extra.split(",") if n and n != a.workload]:
