@@ -75,7 +75,10 @@ typedef struct {
     int32_t sync_op;    /* 0 = SUM (the all-reduce of Algorithm 1), 1 = MEAN          */
     int32_t max_pos;    /* positions 0..max_pos-1 are valid (size of the rotary table)*/
     int32_t flags;      /* bit 0: run the plain SIMT kernels even for bf16 (diagnostic
-                           cross-check; the fp32 dtype always uses them)              */
+                           cross-check; the fp32 dtype always uses them)
+                           bit 1: prefill attention on the warp-level mma.sync kernel
+                           instead of the tensor-memory (tcgen05) one (diagnostic; that
+                           kernel also serves head_dim 32 and 8-token pages)           */
 } pt_config;
 
 typedef struct pt_model pt_model;

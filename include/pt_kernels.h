@@ -46,6 +46,22 @@ pt_status pt_kernel_decode_attn(const void* q, const void* pool_l, int64_t pool_
                                 int32_t num_pages, void* out, void* scratch, size_t scratch_bytes,
                                 void* status, void* stream);
 
+/* Causal prefill attention over the paged per-track KV cache (the attention of a track layer
+ * when S new tokens per sequence are processed at once; every track attends only to its own
+ * cache - Section 2.2).  The K and V of the new tokens must already be in the cache:
+ *   out[t][b*S+s][h] = softmax_{j <= pos}( q[t][b*S+s][h] . K[t][b][h / G][j] / sqrt(dh) ) V[t][b][h / G][j],
+ *   pos = kv_len[b] - S + s.
+ *   q, out        device bf16 [T][B*S][nq*dh]
+ *   pool_l, block_table, status   as for pt_kernel_decode_attn
+ *   kv_len        DEVICE int32 [B]: keys cached per sequence, the S new ones included (>= S)
+ *   impl          0 = tensor-memory kernel (tcgen05; head_dim 64 or 128, pages of a multiple of
+ *                 16 tokens), 1 = warp-level mma.sync kernel (head_dim 32, 64, 128; any page size)
+ * Asynchronous on `stream`; nothing is allocated. */
+pt_status pt_kernel_prefill_attn(const void* q, const void* pool_l, int64_t pool_track_stride,
+                                 const int32_t* block_table, int32_t maxp, const int32_t* kv_len,
+                                 int32_t T, int32_t B, int32_t S, int32_t nq, int32_t nkv, int32_t dh, int32_t ps,
+                                 int32_t num_pages, void* out, int32_t impl, void* status, void* stream);
+
 /* The same decode attention for callers that cannot allocate device memory.  (The paper has no
  * counterpart: this is a packaging variant of pt_kernel_decode_attn.)
  *

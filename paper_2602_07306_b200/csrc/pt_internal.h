@@ -24,6 +24,8 @@ enum : int {
     LOC_ROPE_PAGE = 1, LOC_ATTN_PAGE = 2, LOC_GEMM_TMA_WAIT = 3, LOC_GEMM_MMA_WAIT = 4,
     LOC_GEMM_EPI_WAIT = 5, LOC_GEMM_EMPTY_WAIT = 6, LOC_DECODE_PAGE = 7, LOC_FLASH_PAGE = 8,
     LOC_GEMM_ACC_WAIT = 9,
+    LOC_FLASH_KEMPTY = 10, LOC_FLASH_VEMPTY = 11, LOC_FLASH_VRAW = 12, LOC_FLASH_KFULL = 13, LOC_FLASH_QFULL = 14,
+    LOC_FLASH_PFULL = 15, LOC_FLASH_VFULL = 16, LOC_FLASH_SFULL = 17, LOC_FLASH_OREADY = 18,
 };
 
 extern std::atomic<long long> g_launches;

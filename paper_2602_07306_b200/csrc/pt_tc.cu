@@ -255,6 +255,30 @@ pt_status decode_attn_check_args(const void* q, const void* pool_l, const int32_
 
 }  // namespace pt
 
+extern "C" pt_status pt_kernel_prefill_attn(const void* q, const void* pool_l, int64_t pool_track_stride,
+                                            const int32_t* block_table, int32_t maxp, const int32_t* kv_len,
+                                            int32_t T, int32_t B, int32_t S, int32_t nq, int32_t nkv, int32_t dh, int32_t ps,
+                                            int32_t num_pages, void* out, int32_t impl, void* status, void* stream) {
+    using namespace pt;
+    if (!q || !pool_l || !block_table || !kv_len || !out || !status) { set_error("null argument"); return PT_ERR_INVALID_ARG; }
+    if (T < 1 || B < 1 || S < 1 || nq < 1 || nkv < 1 || nq % nkv || maxp < 1 || num_pages < 1 || (int64_t)B * S > (1 << 30)) { set_error("bad sizes"); return PT_ERR_INVALID_ARG; }
+    if (dh != 32 && dh != 64 && dh != 128) { set_error("head_dim %d not in {32, 64, 128}", dh); return PT_ERR_UNSUPPORTED; }
+    if (ps < 8 || ps > 64 || ps % 8) { set_error("page size must be a multiple of 8 in [8, 64]"); return PT_ERR_INVALID_ARG; }
+    if (impl != 0 && impl != 1) { set_error("impl must be 0 or 1"); return PT_ERR_INVALID_ARG; }
+    if (impl == 0 && !flash_tc_supported(dh, ps)) { set_error("impl 0 needs head_dim 64 or 128 and pages of a multiple of 16 tokens"); return PT_ERR_UNSUPPORTED; }
+    AttnP p{};
+    p.q = (const __nv_bfloat16*)q; p.pool_l = (const __nv_bfloat16*)pool_l; p.pool_tstride = pool_track_stride;
+    p.o = (__nv_bfloat16*)out; p.bt = block_table; p.maxp = maxp; p.kvlen = kv_len;
+    p.B = B; p.S = S; p.M = B * S; p.nq = nq; p.nkv = nkv; p.ps = ps; p.num_pages = num_pages;
+    p.scale_log2 = 1.4426950408889634f / sqrtf((float)dh);
+    p.status = (int*)status;
+    pt_status s = launch_flash_prefill_p(p, T, dh, impl == 1, (cudaStream_t)stream);
+    if (s != PT_OK) return s;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_error("kernel launch failed: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
+    return PT_OK;
+}
+
 extern "C" pt_status pt_kernel_decode_attn_scratch_bytes(int32_t T, int32_t B, int32_t nq, int32_t dh, size_t* bytes) {
     using namespace pt;
     if (!bytes || T < 1 || B < 1 || nq < 1 || dh < 1) { set_error("bad argument"); return PT_ERR_INVALID_ARG; }

@@ -53,6 +53,7 @@ struct AttnP {
     const int32_t* items; const int32_t* nsplit; float* part; int max_splits;
 };
 
+pt_status launch_flash_prefill_p(const AttnP& p, int T, int dh, bool legacy, cudaStream_t st);
 pt_status launch_decode_attn_p(const AttnP& p, int T, int dh, int n_items, int max_splits, cudaStream_t st);
 
 pt_status make_map_bf16(CUtensorMap* out, const void* base, int64_t k, int64_t rows, int64_t tracks, int box_rows);
@@ -64,6 +65,10 @@ pt_status launch_gemm(int epi, int bn, const CUtensorMap& ta, const CUtensorMap&
 // pt_simt.cu
 void tap_copy(Call& k, int layer, int point, const float* src, size_t src_tstride);
 void launch_simt_attn_bf16(Call& k, const __nv_bfloat16* q, int q_row_stride, const __nv_bfloat16* pool_l, __nv_bfloat16* o);
+
+// pt_tc_flash.cu
+bool flash_tc_supported(int dh, int ps);
+pt_status launch_flash_prefill_tc(const AttnP& p, int T, int dh, cudaStream_t st);
 
 // pt_tc_attn.cu
 pt_status launch_flash_prefill(Call& k, const __nv_bfloat16* q, const __nv_bfloat16* pool_l, __nv_bfloat16* o);

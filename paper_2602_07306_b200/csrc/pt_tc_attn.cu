@@ -587,18 +587,22 @@ pt_status set_smem(F* fn, int bytes) {
 
 }  // namespace
 
-pt_status launch_flash_prefill(Call& k, const __nv_bfloat16* q, const __nv_bfloat16* pool_l, __nv_bfloat16* o) {
-    AttnP p = make_params(k, q, pool_l, o);
-    const int dh = k.m->dh;
-    dim3 grid((k.S + 63) / 64, p.nq, k.m->cfg.T * k.B);
+pt_status launch_flash_prefill_p(const AttnP& p, int T, int dh, bool legacy, cudaStream_t st) {
+    if (flash_tc_supported(dh, p.ps) && !legacy) return launch_flash_prefill_tc(p, T, dh, st);
+    dim3 grid((p.S + 63) / 64, p.nq, T * p.B);
     const int smem = 2 * 2 * kTileKeys * dh * 2;
     pt_status s = PT_OK;
 #define GO(DH_) { static bool done = false; if (!done) { if ((s = set_smem(k_flash_prefill<DH_>, smem)) != PT_OK) return s; done = true; } \
-                  k_flash_prefill<DH_><<<grid, kThreads, smem, k.st>>>(p); }
+                  k_flash_prefill<DH_><<<grid, kThreads, smem, st>>>(p); }
     if (dh == 32) GO(32) else if (dh == 64) GO(64) else GO(128)
 #undef GO
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return PT_OK;
+}
+
+pt_status launch_flash_prefill(Call& k, const __nv_bfloat16* q, const __nv_bfloat16* pool_l, __nv_bfloat16* o) {
+    AttnP p = make_params(k, q, pool_l, o);
+    return launch_flash_prefill_p(p, k.m->cfg.T, k.m->dh, (k.m->cfg.flags & 2) != 0, k.st);
 }
 
 pt_status launch_decode_attn_p(const AttnP& p, int T, int dh, int n_items, int max_splits, cudaStream_t st) {

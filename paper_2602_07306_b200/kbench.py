@@ -1,6 +1,7 @@
 """Time one kernel of the PT forward pass through its kernel-level C-ABI entry point.
 
     python -m paper_2602_07306_b200.kbench decode --T 8 --B 64 --nq 8 --nkv 8 --dh 128 --len 2048
+    python -m paper_2602_07306_b200.kbench prefill --T 8 --B 8 --S 4096 --nq 8 --nkv 8 --dh 128 [--impl 1]
     python -m paper_2602_07306_b200.kbench gemm --T 8 --M 32768 --N 3072 --K 1024 [--bn 256] [--fold]
 
 Prints one JSON line: average device time per launch (CUDA events on the launching stream,
@@ -53,6 +54,36 @@ def decode(a):
     print(json.dumps({"kernel": "decode_attn", "ms": ms, "GBps": byts / ms / 1e6, "bytes": byts, "args": vars(a)}))
 
 
+def prefill(a):
+    dev = torch.device("cuda:0")
+    ps = a.ps
+    n = a.S + a.start
+    maxp = -(-n // ps)
+    pages = a.B * maxp
+    g = torch.Generator(device=dev).manual_seed(0)
+    pool = torch.randn((a.T, pages, 2, a.nkv, ps, a.dh), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    q = torch.randn((a.T, a.B * a.S, a.nq * a.dh), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    perm = torch.randperm(pages, generator=torch.Generator().manual_seed(0)).to(torch.int32)
+    bt = perm.reshape(a.B, maxp).contiguous().to(dev)
+    lens = torch.full((a.B,), n, dtype=torch.int32, device=dev)
+    run = lambda: pt.kernel_prefill_attn(q, pool, bt, lens, S=a.S, nq=a.nq, nkv=a.nkv, dh=a.dh, ps=ps, impl=a.impl)
+    for _ in range(a.warmup):
+        out, status = run()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(a.iters):
+        out, status = run()
+    e1.record()
+    torch.cuda.synchronize()
+    assert status[:2].tolist() == [0, 0], status[:2].tolist()
+    ms = e0.elapsed_time(e1) / a.iters
+    # causal triangle only: row s sees start + s + 1 keys
+    keys = a.S * a.start + a.S * (a.S + 1) // 2
+    flops = 4.0 * a.T * a.B * a.nq * a.dh * keys
+    print(json.dumps({"kernel": "prefill_attn", "ms": ms, "TFLOPs": flops / ms / 1e9, "args": vars(a)}))
+
+
 def gemm(a):
     dev = torch.device("cuda:0")
     g = torch.Generator(device=dev).manual_seed(0)
@@ -79,12 +110,15 @@ def main():
     d = sub.add_parser("decode")
     for k, v in dict(T=8, B=64, nq=8, nkv=8, dh=128, len=2048, ps=16, ragged=0, iters=20, warmup=3).items():
         d.add_argument("--" + k, type=int, default=v)
+    pf = sub.add_parser("prefill")
+    for k, v in dict(T=8, B=8, S=4096, start=0, nq=8, nkv=8, dh=128, ps=16, impl=0, iters=10, warmup=3).items():
+        pf.add_argument("--" + k, type=int, default=v)
     gm = sub.add_parser("gemm")
     for k, v in dict(T=8, M=4096, N=3072, K=1024, bn=0, iters=20, warmup=3).items():
         gm.add_argument("--" + k, type=int, default=v)
     gm.add_argument("--fold", action="store_true")
     a = ap.parse_args()
-    (decode if a.cmd == "decode" else gemm)(a)
+    {"decode": decode, "gemm": gemm, "prefill": prefill}[a.cmd](a)
 
 
 if __name__ == "__main__":

@@ -63,6 +63,7 @@ _PROTOS = {
     "pt_profile_read": (_I32, [_P, C.POINTER(C.c_float), C.POINTER(_I64)]),
     "pt_launch_count": (_I64, []),
     "pt_kernel_gemm_bf16": (_I32, [_P, _P, _P, _I32, _I32, _I32, _I32, _I32, _I32, _P, _P]),
+    "pt_kernel_prefill_attn": (_I32, [_P, _P, _I64, _P, _I32, _P, _I32, _I32, _I32, _I32, _I32, _I32, _I32, _I32, _P, _I32, _P, _P]),
     "pt_kernel_decode_attn_scratch_bytes": (_I32, [_I32, _I32, _I32, _I32, C.POINTER(_SZ)]),
     "pt_kernel_decode_attn": (_I32, [_P, _P, _I64, _P, _I32, C.POINTER(_I32), _I32, _I32, _I32, _I32, _I32, _I32, _I32,
                                      _P, _P, _SZ, _P, _P]),
@@ -344,6 +345,24 @@ def kernel_decode_attn(q, pool_l, block_table, kv_len, *, nq, nkv, dh, ps, scrat
                                           block_table.shape[1], plens, T, B, nq, nkv, dh, ps, pages, out.data_ptr(),
                                           scratch.data_ptr(), scratch.numel(), status.data_ptr(),
                                           torch.cuda.current_stream().cuda_stream))
+    return out, status
+
+
+def kernel_prefill_attn(q, pool_l, block_table, kv_len, *, S, nq, nkv, dh, ps, impl=0):
+    """q bf16 [T, B*S, nq*dh]; pool_l bf16 [T, pages, 2, nkv, ps, dh]; block_table int32 [B, maxp] and kv_len
+    int32 [B] on the device (keys cached per sequence, the S new ones included).
+    Returns (out bf16 [T, B*S, nq*dh], status int32[16])."""
+    import torch
+    T, M, _ = q.shape
+    B = M // S
+    assert q.is_contiguous() and pool_l.is_contiguous() and block_table.is_contiguous() and kv_len.is_cuda
+    assert q.dtype == pool_l.dtype == torch.bfloat16 and block_table.dtype == kv_len.dtype == torch.int32
+    out = torch.empty_like(q)
+    status = torch.zeros(16, dtype=torch.int32, device=q.device)
+    with torch.cuda.device(q.device):
+        check(lib().pt_kernel_prefill_attn(q.data_ptr(), pool_l.data_ptr(), pool_l.stride(0), block_table.data_ptr(),
+                                           block_table.shape[1], kv_len.data_ptr(), T, B, S, nq, nkv, dh, ps, pool_l.shape[1],
+                                           out.data_ptr(), impl, status.data_ptr(), torch.cuda.current_stream().cuda_stream))
     return out, status
 
 

@@ -99,3 +99,64 @@ def test_decode_attention_kernel_reports_bad_page():
     torch.cuda.synchronize()
     assert status[0].item() == 8 and status[1].item() == 7
     assert torch.isfinite(out.float()).all()
+
+
+def prefill_case(T, B, S, nq, nkv, dh, ps, starts, seed):
+    """Random paged cache holding starts[b] + S keys per sequence (slots past a sequence's last
+    key hold NaN: they must never reach a result) + queries for the last S positions; the
+    float64 result comes from oracle.attention, one sequence and track at a time."""
+    import torch
+    from oracle import pt_oracle as O
+    rng = np.random.default_rng(seed)
+    lens = [int(s0) + S for s0 in starts]
+    maxp = max(-(-n // ps) for n in lens)
+    pages = sum(-(-n // ps) for n in lens) + 2
+    perm = I.free_list_permutation(pages, seed=seed)
+    bt = np.zeros((B, maxp), np.int32)
+    nxt = 0
+    for b, n in enumerate(lens):
+        k = -(-n // ps)
+        bt[b, :k] = perm[nxt:nxt + k]
+        nxt += k
+    pool = I.round_to_bf16(rng.standard_normal((T, pages, 2, nkv, ps, dh), dtype=np.float32))
+    q = I.round_to_bf16(rng.standard_normal((T, B * S, nq * dh), dtype=np.float32))
+    ref = np.zeros((T, B * S, nq * dh))
+    valid = np.zeros((pages, ps), bool)
+    for t in range(T):
+        for b, n in enumerate(lens):
+            pos = np.arange(n)
+            valid[bt[b, pos // ps], pos % ps] = True
+            k = pool[t, bt[b, pos // ps], 0, :, pos % ps, :].astype(np.float64)
+            v = pool[t, bt[b, pos // ps], 1, :, pos % ps, :].astype(np.float64)
+            qb = q[t, b * S:(b + 1) * S].reshape(S, nq, dh).astype(np.float64)
+            ref[t, b * S:(b + 1) * S] = O.attention(qb, k, v, starts[b] + np.arange(S)).reshape(S, -1)
+    pool = np.where(valid[None, :, None, None, :, None], pool, np.float32(np.nan))
+    dev = lambda a, dt: torch.from_numpy(a).cuda().to(dt).contiguous()
+    return (dev(q, torch.bfloat16), dev(pool, torch.bfloat16), dev(bt, torch.int32),
+            dev(np.asarray(lens, np.int32), torch.int32), ref)
+
+
+PREFILL_CASES = [
+    (1, 1, 128, 1, 1, 128, 16, [0]),                 # one query tile, one key tile
+    (1, 1, 256, 2, 2, 128, 16, [0]),                 # both query tiles of a CTA, 1 and 2 key tiles
+    (2, 2, 300, 4, 2, 128, 16, [0, 213]),            # ragged tails, earlier keys in the cache (chunked prefill), GQA 2:1
+    (1, 3, 37, 2, 1, 64, 16, [0, 5, 100]),           # short chunks, head_dim 64
+    (1, 2, 700, 2, 2, 64, 32, [513, 0]),             # 32-token pages, several CTAs per sequence
+    (2, 1, 1024, 2, 1, 128, 16, [0]),                # keys end exactly on a tile boundary
+    (1, 2, 1, 2, 2, 128, 16, [130, 0]),              # single new token per sequence
+]
+
+
+@pytest.mark.parametrize("impl", [0, 1])
+@pytest.mark.parametrize("T,B,S,nq,nkv,dh,ps,starts", PREFILL_CASES)
+def test_prefill_attention_kernel_matches_oracle(T, B, S, nq, nkv, dh, ps, starts, impl):
+    import torch
+    from paper_2602_07306_b200 import pt
+    q, pool, bt, lens, ref = prefill_case(T, B, S, nq, nkv, dh, ps, starts, seed=S + sum(starts))
+    out, status = pt.kernel_prefill_attn(q, pool, bt, lens, S=S, nq=nq, nkv=nkv, dh=dh, ps=ps, impl=impl)
+    torch.cuda.synchronize()
+    assert status[:2].tolist() == [0, 0]
+    got = out.float().cpu().numpy().astype(np.float64)
+    assert np.all(np.isfinite(got))
+    d = np.abs(got - ref)
+    assert d.max() <= 2e-2 * np.abs(ref).max() and d.mean() <= 4e-3 * np.abs(ref).mean(), (d.max() / np.abs(ref).max(), d.mean() / np.abs(ref).mean())
