@@ -113,6 +113,21 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// Packed fp32 pairs (one instruction for two lanes of arithmetic) and the three-input maximum.
+__device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, float s, float b) {   // a * s + b
+    asm("{\n .reg .b64 ra, rs, rb, rd;\n mov.b64 ra, {%2, %3};\n mov.b64 rs, {%4, %4};\n mov.b64 rb, {%5, %5};\n"
+        " fma.rn.f32x2 rd, ra, rs, rb;\n mov.b64 {%0, %1}, rd;\n}"
+        : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(s), "f"(b));
+}
+__device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1) {                    // d += a
+    asm("{\n .reg .b64 ra, rd;\n mov.b64 ra, {%2, %3};\n mov.b64 rd, {%0, %1};\n add.rn.f32x2 rd, rd, ra;\n mov.b64 {%0, %1}, rd;\n}"
+        : "+f"(d0), "+f"(d1) : "f"(a0), "f"(a1));
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -194,6 +209,10 @@ k_flash_prefill_tc(const __grid_constant__ CUtensorMap qmap, const __grid_consta
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    // the copy and MMA warps need few registers; hand theirs to the softmax groups, whose threads
+    // keep a whole 128-column score row each
+    if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -307,8 +326,10 @@ k_flash_prefill_tc(const __grid_constant__ CUtensorMap qmap, const __grid_consta
             }
         }
         __syncwarp();
-    } else if (warp >= 4) {
+    }
+    } else {
         // ------------------------------------------------------------------ softmax groups
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
         const int i = (warp - 4) >> 2;                             // query tile of this warp group
         const int w4 = warp & 3;                                   // tensor-memory lane quarter of this warp
         const int n_i = n_t[i];
@@ -328,21 +349,20 @@ k_flash_prefill_tc(const __grid_constant__ CUtensorMap qmap, const __grid_consta
             tc_fence_after();
             const int key0 = j * 128;
             const bool need_mask = key0 + 127 > tile_limit;
-            // pass 1: row maximum of the raw scores
+            // the whole score row of this thread lives in registers: one round trip to tensor memory
+            float v[128];
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) tm_ld32(t_s + cc * 32, v + cc * 32);
+            tm_wait_ld();
+            if (need_mask) {
+#pragma unroll
+                for (int e = 0; e < 128; ++e) if (key0 + e > limit) v[e] = -INFINITY;
+            }
             float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll 1
-            for (int cc = 0; cc < 4; ++cc) {
-                float v[32];
-                tm_ld32(t_s + cc * 32, v);
-                tm_wait_ld();
-                if (need_mask) {
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) if (key0 + cc * 32 + e > limit) v[e] = -INFINITY;
-                }
-#pragma unroll
-                for (int e = 0; e < 32; e += 4) {
-                    mx0 = fmaxf(mx0, v[e]); mx1 = fmaxf(mx1, v[e + 1]); mx2 = fmaxf(mx2, v[e + 2]); mx3 = fmaxf(mx3, v[e + 3]);
-                }
+            for (int e = 0; e < 128; e += 8) {
+                mx0 = max3(mx0, v[e], v[e + 1]); mx1 = max3(mx1, v[e + 2], v[e + 3]);
+                mx2 = max3(mx2, v[e + 4], v[e + 5]); mx3 = max3(mx3, v[e + 6], v[e + 7]);
             }
             const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
             if (j == 0) {
@@ -369,24 +389,24 @@ k_flash_prefill_tc(const __grid_constant__ CUtensorMap qmap, const __grid_consta
                 }
             }
             const float mc = m_ref * c;
-            // pass 2: P = exp2(c s - c m) as bf16 over the first half of the score columns
+            // P = exp2(c s - c m) as bf16 over the first half of the score columns (masked scores are
+            // -inf and give exactly 0)
             float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
-#pragma unroll 1
+            const float nmc = -mc;
+#pragma unroll
             for (int cc = 0; cc < 4; ++cc) {
-                float v[32];
-                tm_ld32(t_s + cc * 32, v);
-                tm_wait_ld();
-#pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    float pe = ex2(fmaf(v[e], c, -mc));
-                    if (need_mask && key0 + cc * 32 + e > limit) pe = 0.f;
-                    v[e] = pe;
-                }
-#pragma unroll
-                for (int e = 0; e < 32; e += 4) { l0 += v[e]; l1 += v[e + 1]; l2 += v[e + 2]; l3 += v[e + 3]; }
                 uint32_t pk[16];
 #pragma unroll
-                for (int e = 0; e < 16; ++e) pk[e] = pack_bf16(v[2 * e], v[2 * e + 1]);
+                for (int e = 0; e < 32; e += 4) {
+                    float x0, x1, x2, x3;
+                    fma2(x0, x1, v[cc * 32 + e], v[cc * 32 + e + 1], c, nmc);
+                    fma2(x2, x3, v[cc * 32 + e + 2], v[cc * 32 + e + 3], c, nmc);
+                    x0 = ex2(x0); x1 = ex2(x1); x2 = ex2(x2); x3 = ex2(x3);
+                    add2(l0, l1, x0, x1);
+                    add2(l2, l3, x2, x3);
+                    pk[e >> 1] = pack_bf16(x0, x1);
+                    pk[(e >> 1) + 1] = pack_bf16(x2, x3);
+                }
                 tm_st16(t_s + cc * 16, pk);
             }
             l_run += (l0 + l1) + (l2 + l3);
