@@ -23,6 +23,7 @@ namespace {
 constexpr int kFlashThreads = 384;
 constexpr int kStages = 2;                 // K ring and V ring depth
 constexpr uint32_t kSpin = 1u << 26;
+constexpr int kPolyOf8 = 0;                // of every 8 scores, 2 (value 4) or 4 (value 8) take the polynomial exp2
 constexpr int kHalfBytes = 128 * 128;      // 128 rows x 64 bf16: one swizzled column block of a tile
 
 enum { B_QFULL = 0, B_KFULL = 2, B_KEMPTY = 4, B_VFULL = 6, B_VEMPTY = 8, B_SFULL = 10, B_PFULL = 12,
@@ -123,6 +124,29 @@ __device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1) {
     asm("{\n .reg .b64 ra, rd;\n mov.b64 ra, {%2, %3};\n mov.b64 rd, {%0, %1};\n add.rn.f32x2 rd, rd, ra;\n mov.b64 {%0, %1}, rd;\n}"
         : "+f"(d0), "+f"(d1) : "f"(a0), "f"(a1));
 }
+// (a0, a1) * (b0, b1) + (c0, c1)
+__device__ __forceinline__ void fma2v(float& d0, float& d1, float a0, float a1, float b0, float b1, float c0, float c1) {
+    asm("{\n .reg .b64 ra, rb, rc, rd;\n mov.b64 ra, {%2, %3};\n mov.b64 rb, {%4, %5};\n mov.b64 rc, {%6, %7};\n"
+        " fma.rn.f32x2 rd, ra, rb, rc;\n mov.b64 {%0, %1}, rd;\n}"
+        : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1), "f"(c0), "f"(c1));
+}
+// 2^x for a pair of x <= 0 without the special-function unit: x = r + f with r = round(x) taken
+// from the low mantissa bits of x + 1.5*2^23, 2^f from a cubic fitted on [-0.5, 0.5] (relative
+// error below 8e-5, far inside the bf16 rounding P receives), 2^r added into the exponent field.
+__device__ __forceinline__ void ex2_poly2(float& x0, float& x1) {
+    constexpr float kMagic = 12582912.0f;
+    constexpr float k0 = 0.99992895f, k1 = 0.69327623f, k2 = 0.24260405f, k3 = 0.05508868f;
+    x0 = fmaxf(x0, -126.0f); x1 = fmaxf(x1, -126.0f);
+    float t0, t1, r0, r1, f0, f1, p0, p1;
+    fma2v(t0, t1, x0, x1, 1.0f, 1.0f, kMagic, kMagic);
+    fma2v(r0, r1, t0, t1, 1.0f, 1.0f, -kMagic, -kMagic);
+    fma2v(f0, f1, r0, r1, -1.0f, -1.0f, x0, x1);
+    fma2v(p0, p1, f0, f1, k3, k3, k2, k2);
+    fma2v(p0, p1, p0, p1, f0, f1, k1, k1);
+    fma2v(p0, p1, p0, p1, f0, f1, k0, k0);
+    x0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(t0) << 23));
+    x1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
+}
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float d;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -181,9 +205,11 @@ k_flash_prefill_tc(const __grid_constant__ CUtensorMap qmap, const __grid_consta
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int head = blockIdx.x, kvh = head / (p.nq / p.nkv);
-    const int t = blockIdx.y / p.B, b = blockIdx.y % p.B;
-    const int qb = gridDim.z - 1 - blockIdx.z;                     // longest query blocks first
+    // consecutive CTAs are the query blocks of one (track, sequence, head), longest first: they read
+    // the same K/V pages at about the same time, so all but the first find them in L2
+    const int qb = gridDim.x - 1 - blockIdx.x;
+    const int head = blockIdx.y, kvh = head / (p.nq / p.nkv);
+    const int t = blockIdx.z / p.B, b = blockIdx.z % p.B;
     const int key_end = p.kvlen[b];
     const int start = key_end - p.S;                               // position of the sequence's first new token
     int n_t[2];
@@ -212,7 +238,7 @@ k_flash_prefill_tc(const __grid_constant__ CUtensorMap qmap, const __grid_consta
     // the copy and MMA warps need few registers; hand theirs to the softmax groups, whose threads
     // keep a whole 128-column score row each
     if (warp < 4) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -329,7 +355,7 @@ k_flash_prefill_tc(const __grid_constant__ CUtensorMap qmap, const __grid_consta
     }
     } else {
         // ------------------------------------------------------------------ softmax groups
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
         const int i = (warp - 4) >> 2;                             // query tile of this warp group
         const int w4 = warp & 3;                                   // tensor-memory lane quarter of this warp
         const int n_i = n_t[i];
@@ -401,7 +427,8 @@ k_flash_prefill_tc(const __grid_constant__ CUtensorMap qmap, const __grid_consta
                     float x0, x1, x2, x3;
                     fma2(x0, x1, v[cc * 32 + e], v[cc * 32 + e + 1], c, nmc);
                     fma2(x2, x3, v[cc * 32 + e + 2], v[cc * 32 + e + 3], c, nmc);
-                    x0 = ex2(x0); x1 = ex2(x1); x2 = ex2(x2); x3 = ex2(x3);
+                    x0 = ex2(x0); x1 = ex2(x1);
+                    if ((e & 7) < kPolyOf8) ex2_poly2(x2, x3); else { x2 = ex2(x2); x3 = ex2(x3); }
                     add2(l0, l1, x0, x1);
                     add2(l2, l3, x2, x3);
                     pk[e >> 1] = pack_bf16(x0, x1);
@@ -455,13 +482,13 @@ bool flash_tc_supported(int dh, int ps) { return (dh == 64 || dh == 128) && ps %
 
 pt_status launch_flash_prefill_tc(const AttnP& p, int T, int dh, cudaStream_t st) {
     if (!flash_tc_supported(dh, p.ps)) { set_error("tensor-memory prefill attention needs head_dim 64 or 128 and pages of a multiple of 16 tokens"); return PT_ERR_UNSUPPORTED; }
-    if ((int64_t)T * p.B > 65535 || (p.S + 255) / 256 > 65535) { set_error("prefill attention grid too large"); return PT_ERR_INVALID_ARG; }
+    if ((int64_t)T * p.B > 65535 || p.nq > 65535) { set_error("prefill attention grid too large"); return PT_ERR_INVALID_ARG; }
     CUtensorMap qmap, kvmap;
     pt_status s;
     if ((s = make_map_bf16(&qmap, p.q, (int64_t)p.nq * dh, p.M, T, 128)) != PT_OK) return s;
     if ((s = make_map_bf16_strided(&kvmap, p.pool_l, dh, (int64_t)p.num_pages * 2 * p.nkv * p.ps, T, p.pool_tstride * 2, 16)) != PT_OK) return s;
     const int q_box_rows = std::min(128, p.M);
-    dim3 grid(p.nq, T * p.B, (p.S + 255) / 256);
+    dim3 grid((p.S + 255) / 256, p.nq, T * p.B);
 #define GO(DH_) { static bool done = false; \
         if (!done) { cudaError_t e = cudaFuncSetAttribute(k_flash_prefill_tc<DH_>, cudaFuncAttributeMaxDynamicSharedMemorySize, FlashCfg<DH_>::SMEM); \
                      if (e != cudaSuccess) { set_error("cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; } done = true; } \
