@@ -7,8 +7,8 @@
 //     P_i = exp2(c S_i - c m)  written back over S_i as bf16 by the softmax warps
 //     O_i += P_i V           (tcgen05.mma with P_i read from tensor memory, V as an MN-major tile)
 // Roles: warp 0 streams Q once and K/V page by page with TMA (16-token boxes of the cache's
-// [page][K|V][head][slot][dh] blocks, 128-byte swizzle) through two-stage rings; lane 0 of warp 1
-// issues every MMA; warps 4-7 and 8-11 are the softmax groups of tile 0 and tile 1, one thread per
+// [page][K|V][head][slot][dh] blocks, 128-byte swizzle) through two-stage rings; warp 1
+// issues every MMA (one elected lane); warps 4-7 and 8-11 are the softmax groups of tile 0 and tile 1, one thread per
 // query row (row max and row sum need no shuffles).  While one group works on its scores the
 // tensor pipe runs the other tile's products.  The running maximum is only raised when it grows
 // by more than 2^8 (the accumulator is then rescaled in tensor memory), so rescales are rare.
@@ -58,17 +58,19 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// The MMA warp runs its issue loop with all 32 lanes (so addresses and descriptors stay
+// warp-uniform values) and one elected lane executes each tcgen05 instruction.
 __device__ __forceinline__ void tc_commit(uint64_t* bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+    asm volatile("{\n .reg .pred e;\n elect.sync _|e, 0xffffffff;\n @e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}" ::"r"(smem_u32(bar)) : "memory");
 }
 // D[tmem] (+)= A[smem] * B[smem]
 __device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
-    asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+    asm volatile("{\n .reg .pred p, e;\n elect.sync _|e, 0xffffffff;\n setp.ne.b32 p, %4, 0;\n @e tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
                  ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem]
 __device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t acc) {
-    asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+    asm volatile("{\n .reg .pred p, e;\n elect.sync _|e, 0xffffffff;\n setp.ne.b32 p, %4, 0;\n @e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
                  ::"r"(d), "r"(a_tmem), "l"(b), "r"(idesc), "r"(acc) : "memory");
 }
 __device__ __forceinline__ void tm_ld32(uint32_t taddr, float* v) {
@@ -300,14 +302,14 @@ k_flash_prefill_tc(const __grid_constant__ CUtensorMap qmap, const __grid_consta
         }
         if (bad_page) report(p.status, PT_ERR_DEVICE_BOUNDS, LOC_FLASH_PAGE);
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // ------------------------------------------------------------------ MMA issuer (whole warp, see tc_commit)
+        {
             constexpr uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
             constexpr uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(DH >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
             bool ok = true;
             auto wait = [&](int bar, uint32_t parity, int loc) {
                 if (!ok) return;
-                if (!mbar_wait(&bars[bar], parity, abort_flag)) { ok = false; report(p.status, PT_ERR_DEVICE_TIMEOUT, loc); *abort_flag = 1; }
+                if (!__all_sync(0xffffffffu, mbar_wait(&bars[bar], parity, abort_flag))) { ok = false; if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, loc); *abort_flag = 1; } }
                 tc_fence_after();
             };
             auto qk = [&](int i, int s) {                          // S_i = Q_i K_s^T
