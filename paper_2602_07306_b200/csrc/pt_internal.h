@@ -16,7 +16,7 @@
 namespace pt {
 
 constexpr int kStatusWords = 16;          // device status word block (int32 each)
-constexpr int kSsqTile = 128;             // columns covered by one partial sum of squares
+constexpr int kSsqTile = 64;              // columns covered by one partial sum of squares
 constexpr int kMaxSplits = 16;            // upper bound of KV key ranges per sequence in decode
 
 // Location codes written next to PT_ERR_DEVICE_* in the status block.

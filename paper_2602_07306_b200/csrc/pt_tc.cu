@@ -17,23 +17,25 @@ __global__ void k_tc_prep(const __nv_bfloat16* __restrict__ x, int64_t x_stride,
     if (warp >= M) return;
     const __nv_bfloat16* xr = x + (size_t)t * x_stride + (size_t)warp * H;
     size_t ro = ((size_t)t * M + warp) * H;
-    for (int tile = 0; tile < tiles; ++tile) {
-        int c = tile * kSsqTile + lane * 4;
+    // 128 columns per pass: lanes 0-15 cover one kSsqTile-column group, lanes 16-31 the next
+    for (int g = 0; g * 128 < H; ++g) {
+        int c = g * 128 + lane * 4;
         float s = 0.f;
         if (c < H) {
             uint2 raw = *reinterpret_cast<const uint2*>(xr + c);
             __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162*>(&raw.x), b = *reinterpret_cast<__nv_bfloat162*>(&raw.y);
             float v0 = __low2float(a), v1 = __high2float(a), v2 = __low2float(b), v3 = __high2float(b);
             *reinterpret_cast<float4*>(h + ro + c) = make_float4(v0, v1, v2, v3);
-            float4 g = *reinterpret_cast<const float4*>(gain + (size_t)t * H + c);
-            __nv_bfloat162 o0 = __floats2bfloat162_rn(v0 * g.x, v1 * g.y), o1 = __floats2bfloat162_rn(v2 * g.z, v3 * g.w);
+            float4 gn = *reinterpret_cast<const float4*>(gain + (size_t)t * H + c);
+            __nv_bfloat162 o0 = __floats2bfloat162_rn(v0 * gn.x, v1 * gn.y), o1 = __floats2bfloat162_rn(v2 * gn.z, v3 * gn.w);
             uint2 ov;
             ov.x = *reinterpret_cast<uint32_t*>(&o0); ov.y = *reinterpret_cast<uint32_t*>(&o1);
             *reinterpret_cast<uint2*>(hb + ro + c) = ov;
             s = v0 * v0 + v1 * v1 + v2 * v2 + v3 * v3;
         }
-        for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-        if (lane == 0) ssq[((size_t)t * M + warp) * tiles + tile] = s;
+        for (int o = 8; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        int tile = g * 2 + (lane >> 4);
+        if ((lane & 15) == 0 && tile < tiles) ssq[((size_t)t * M + warp) * tiles + tile] = s;
     }
 }
 

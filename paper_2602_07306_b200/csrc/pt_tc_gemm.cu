@@ -1,8 +1,8 @@
 // Track-grouped bf16 GEMM for sm_100a: C[t] = A[t] * W[t]^T with fp32 accumulation in tensor
 // memory.  Persistent, warp-specialised: warp 0 feeds a ring of shared-memory stages with TMA
 // (3-D tensor maps, coordinates (k, row, track), 128-byte swizzle), warp 1 issues tcgen05.mma
-// (128 x BN x 16 per instruction) into one of two TMEM accumulators, warps 2-5 drain the other
-// accumulator with tcgen05.ld and run the fused epilogue:
+// (128 x BN x 16 per instruction, one elected lane) into one of two TMEM accumulators, warps 2-9
+// drain the other accumulator with tcgen05.ld and run the fused epilogue:
 //   EPI_QKV     per-row 1/rms scale (RMSNorm), rotary embedding on q and k heads, q to a dense
 //               buffer, k and v straight into the paged KV cache
 //   EPI_SWIGLU  per-row 1/rms scale, silu(gate) * up on interleaved gate/up columns
@@ -11,6 +11,14 @@
 //               fp32 stream out, gain-scaled bf16 copy for the next GEMM, partial sums of squares
 //               for the next RMSNorm
 //   EPI_PLAIN   fp32 C (kernel-level tests)
+// Epilogue data path: a warp owns 32 accumulator rows (its tensor-memory lane quarter) and works in
+// units of 32 columns.  tcgen05.ld hands every thread one row; whatever needs the whole row
+// (1/rms, SiLU pairing, the sum of squares) happens there.  The unit then goes through a padded
+// 32 x 33 shared-memory tile so that the global loads and stores run with lane = column: every
+// instruction touches one contiguous 64- or 128-byte piece of one row instead of 32 rows.  Global
+// loads that do not depend on the accumulator (row statistics, rotary table, residual rows) are
+// issued before the wait for the accumulator and one unit ahead, so their latency hides behind
+// the tensor pipe.
 // Every mbarrier wait is bounded; on a timeout the CTA records PT_ERR_DEVICE_TIMEOUT, stops
 // issuing work, frees its tensor memory and exits.
 #include "pt_tc.h"
@@ -20,6 +28,10 @@ namespace pt {
 namespace {
 
 constexpr int BM = 128, BK = 64;
+constexpr int kEpiWarps = 8;
+constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
+constexpr int kPitch = 33;                         // floats per row of a staging tile (odd: no bank conflicts)
+constexpr int kStageTileBytes = 32 * kPitch * 4;
 constexpr uint32_t kSpinLimit = 1u << 26;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -56,12 +68,16 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, u
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// The MMA warp runs its loop with all 32 lanes, so addresses and descriptors stay warp-uniform
+// values, and one elected lane executes each tcgen05 instruction.
 __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+    asm volatile("{\n .reg .pred p, e;\n elect.sync _|e, 0xffffffff;\n setp.ne.b32 p, %4, 0;\n"
+                 " @e tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
                  ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void tc_commit(uint64_t* bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+    asm volatile("{\n .reg .pred e;\n elect.sync _|e, 0xffffffff;\n"
+                 " @e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ void tc_ld16(uint32_t taddr, float* v) {
     uint32_t r[16];
@@ -91,34 +107,276 @@ __device__ __forceinline__ void report(int* status, int code, int loc) {
     if (atomicCAS(status, 0, code) == 0) status[1] = loc;
 }
 
-__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
-    __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
-    return *reinterpret_cast<uint32_t*>(&v);
-}
-// 16 floats -> 16 bf16 (32 bytes, two 16-byte stores)
-__device__ __forceinline__ void store16_bf16(__nv_bfloat16* dst, const float* v) {
-    uint4 a, b;
-    a.x = pack_bf16(v[0], v[1]); a.y = pack_bf16(v[2], v[3]); a.z = pack_bf16(v[4], v[5]); a.w = pack_bf16(v[6], v[7]);
-    b.x = pack_bf16(v[8], v[9]); b.y = pack_bf16(v[10], v[11]); b.z = pack_bf16(v[12], v[13]); b.w = pack_bf16(v[14], v[15]);
-    reinterpret_cast<uint4*>(dst)[0] = a;
-    reinterpret_cast<uint4*>(dst)[1] = b;
-}
-
 template <int BN> struct Cfg {
     static constexpr int STAGES = BN == 256 ? 4 : 6;
     static constexpr int A_BYTES = BM * BK * 2;
     static constexpr int B_BYTES = BN * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int SMEM = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static constexpr int RING_BYTES = STAGES * STAGE_BYTES;
+    static constexpr int SMEM = RING_BYTES + kEpiWarps * kStageTileBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
+// ---- epilogue ------------------------------------------------------------------------------
+// Row domain: after tcgen05.ld thread `lane` holds columns of row row0 + lane.  Column domain:
+// after the trip through the staging tile lane `l` holds column l of each of the warp's rows in
+// turn.
+__device__ __forceinline__ void put_row(float* tile_s, int lane, const float* v) {
+#pragma unroll
+    for (int k = 0; k < 32; ++k) tile_s[lane * kPitch + k] = v[k];
+}
+
+// 1 / rms of this thread's row from the producer's partial sums of squares.
+__device__ __forceinline__ float row_rinv(const GemmP& p, int t, int row, bool row_ok) {
+    if (!row_ok) return 1.f;
+    const float* sp = p.ssq_in + (size_t)t * p.ssq_in_tstride + (size_t)row * p.ssq_tiles;
+    float s = 0.f;
+    for (int i = 0; i < p.ssq_tiles; ++i) s += sp[i];
+    return 1.0f / sqrtf(s / (float)p.K + p.eps);
+}
+
+// Every epilogue first issues whatever global loads do not depend on the accumulator, then calls
+// wait() for the accumulator: the loads are in flight while the tensor pipe still works on the tile.
+template <int BN, class Wait>
+__device__ __forceinline__ bool epi_plain(const GemmP& p, uint32_t taddr, float* tile_s, int t, int row0, int nrows,
+                                          int n0, int half, int lane, Wait wait) {
+    constexpr int UNITS = BN / 64;                        // 32-column units per warp
+    if (!wait()) return false;
+    for (int u = 0; u < UNITS; ++u) {
+        const int c = (half * UNITS + u) * 32;
+        if (n0 + c >= p.N) break;                          // uniform across the warp
+        float v[32];
+        tc_ld16(taddr + c, v);
+        tc_ld16(taddr + c + 16, v + 16);
+        tc_wait_ld();
+        put_row(tile_s, lane, v);
+        __syncwarp();
+        const int col = n0 + c + lane;
+        if (col < p.N) {
+            float* dst = p.c_out + ((size_t)t * p.M + row0) * p.N + col;
+#pragma unroll 8
+            for (int rr = 0; rr < 32; ++rr) if (rr < nrows) dst[(size_t)rr * p.N] = tile_s[rr * kPitch + lane];
+        }
+        __syncwarp();
+    }
+    return true;
+}
+
+// Accumulator columns come in groups of 32: 16 gate columns followed by their 16 up columns.  A
+// unit here is 64 accumulator columns = 32 outputs z = silu(gate / rms) * (up / rms).
+template <int BN, class Wait>
+__device__ __forceinline__ bool epi_swiglu(const GemmP& p, uint32_t taddr, float* tile_s, int t, int row0, int row,
+                                           bool row_ok, int nrows, int n0, int half, int lane, Wait wait) {
+    constexpr int UNITS = BN / 128;                       // 64-column units per warp
+    const float rinv = row_rinv(p, t, row, row_ok);
+    const int F = p.N >> 1;
+    if (!wait()) return false;
+    for (int u = 0; u < UNITS; ++u) {
+        const int c = (half * UNITS + u) * 64;
+        if (n0 + c >= p.N) break;
+        float z[32], gu[64];
+#pragma unroll
+        for (int g4 = 0; g4 < 4; ++g4) tc_ld16(taddr + c + g4 * 16, gu + g4 * 16);
+        tc_wait_ld();
+#pragma unroll
+        for (int g2 = 0; g2 < 2; ++g2) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float gv = gu[g2 * 32 + i] * rinv, uv = gu[g2 * 32 + 16 + i] * rinv;
+                z[g2 * 16 + i] = __fdividef(gv, 1.0f + __expf(-gv)) * uv;
+            }
+        }
+        put_row(tile_s, lane, z);
+        __syncwarp();
+        const int zc = ((n0 + c) >> 1) + lane;             // output column of this lane
+        if (zc < F) {
+            __nv_bfloat16* dst = p.z_out + ((size_t)t * p.M + row0) * F + zc;
+#pragma unroll 8
+            for (int rr = 0; rr < 32; ++rr) if (rr < nrows) dst[(size_t)rr * F] = __float2bfloat16_rn(tile_s[rr * kPitch + lane]);
+        }
+        __syncwarp();
+    }
+    return true;
+}
+
+// A unit is 32 accumulator columns of one head: for q and k heads the 16 columns j0..j0+15 and
+// their rotary partners j0+dh/2.., for v heads 32 consecutive columns.  In the column domain
+// lanes 0-15 hold a unit's low columns and fetch cos, lanes 16-31 hold the partners and fetch
+// sin; one shuffle pairs them up.  The table entries of a unit are fetched one unit ahead.
+template <int BN, class Wait>
+__device__ __forceinline__ bool epi_qkv(const GemmP& p, uint32_t taddr, float* tile_s, int t, int row0, int row,
+                                        bool row_ok, int nrows, int n0, int half, int lane, Wait wait) {
+    constexpr int UNITS = BN / 64;                        // units per warp
+    const int dh = p.dh, halfdh = dh >> 1, upd = dh >> 5;  // units per head
+    const int heads_total = p.nq + 2 * p.nkv;
+    int pos = 0; int64_t kvoff = 0;
+    if (row_ok) { pos = p.row_pos[row]; kvoff = p.row_kvoff[row]; }
+    const float rinv = row_rinv(p, t, row, row_ok);
+    const bool slot_ok = row_ok && kvoff >= 0 && kvoff + (int64_t)(2 * p.nkv - 1) * p.ps * dh + dh <= p.slab_elems;
+    if (row_ok && !slot_ok) report(p.status, PT_ERR_DEVICE_BOUNDS, LOC_ROPE_PAGE);
+    const uint32_t slot_mask = __ballot_sync(0xffffffffu, slot_ok);
+    const int kv_lo = (int)(uint32_t)(kvoff & 0xffffffffll), kv_hi = (int)(kvoff >> 32);
+    const float* table = lane < 16 ? p.cs : p.sn;
+    // cos (lanes 0-15) or sin (lanes 16-31) of this lane's column for each of the warp's rows
+    auto fetch = [&](int uu, float* tab) {
+        const int u = half * UNITS + uu;
+        const int hs = n0 / dh + u / upd;
+        if (hs >= p.nq + p.nkv) return;                    // v heads and columns past N: no rotation
+        const int j = (u % upd) * 16 + (lane & 15);
+#pragma unroll
+        for (int rr = 0; rr < 32; ++rr) {
+            const int pr = __shfl_sync(0xffffffffu, pos, rr);
+            tab[rr] = rr < nrows ? table[(size_t)pr * halfdh + j] : 0.f;
+        }
+    };
+    float tab[2][32];
+    fetch(0, tab[0]);
+    if (!wait()) return false;
+#pragma unroll
+    for (int uu = 0; uu < UNITS; ++uu) {
+        const int u = half * UNITS + uu;
+        const int hc = u / upd, sub = u % upd;
+        const int hs = n0 / dh + hc;                       // head slot: q heads, then k heads, then v heads
+        if (hs >= heads_total) break;                      // uniform across the warp
+        const bool is_v = hs >= p.nq + p.nkv;
+        if (uu + 1 < UNITS) fetch(uu + 1, tab[(uu + 1) & 1]);
+        float v[32];
+        if (!is_v) {
+            tc_ld16(taddr + hc * dh + sub * 16, v);
+            tc_ld16(taddr + hc * dh + halfdh + sub * 16, v + 16);
+        } else {
+            tc_ld16(taddr + hc * dh + sub * 32, v);
+            tc_ld16(taddr + hc * dh + sub * 32 + 16, v + 16);
+        }
+        tc_wait_ld();
+#pragma unroll
+        for (int k = 0; k < 32; ++k) v[k] *= rinv;
+        put_row(tile_s, lane, v);
+        __syncwarp();
+        // column domain
+        const int j = sub * 16 + (lane & 15);
+        const int col = is_v ? sub * 32 + lane : (lane < 16 ? j : j + halfdh);      // column inside the head
+        __nv_bfloat16* qdst = nullptr;
+        int64_t head_off = 0;
+        if (hs < p.nq) {
+            qdst = p.q_out + ((size_t)t * p.M + row0) * (size_t)(p.nq * dh) + (size_t)hs * dh + col;
+        } else {
+            const int kv = is_v ? 1 : 0, head = hs - p.nq - kv * p.nkv;
+            head_off = (int64_t)t * p.pool_tstride + ((int64_t)kv * p.nkv + head) * p.ps * dh + col;
+        }
+        const float* tb = tab[uu & 1];
+#pragma unroll
+        for (int rr = 0; rr < 32; ++rr) {
+            float y = tile_s[rr * kPitch + lane];
+            if (!is_v) {
+                const float partner = __shfl_xor_sync(0xffffffffu, y, 16);
+                const float other = __shfl_xor_sync(0xffffffffu, tb[rr], 16);   // sin for the low lanes, cos for the high
+                // low column: x cos - x' sin;  partner column: x' cos + x sin
+                y = lane < 16 ? y * tb[rr] - partner * other : y * other + partner * tb[rr];
+            }
+            if (qdst) {
+                if (rr < nrows) qdst[(size_t)rr * (p.nq * dh)] = __float2bfloat16_rn(y);
+            } else {
+                const int lo = __shfl_sync(0xffffffffu, kv_lo, rr), hi = __shfl_sync(0xffffffffu, kv_hi, rr);
+                if (rr < nrows && ((slot_mask >> rr) & 1u)) {
+                    const int64_t off = ((int64_t)hi << 32) | (uint32_t)lo;
+                    p.pool_l[off + head_off] = __float2bfloat16_rn(y);
+                }
+            }
+        }
+        __syncwarp();
+    }
+    return true;
+}
+
+// Residual add (+ track-sync sum), fp32 stream out, gain-scaled bf16 copy, partial sums of squares.
+// The residual rows of a unit are fetched (lane = column) one unit ahead of their use.
+template <int BN, class Wait>
+__device__ __forceinline__ bool epi_resid(const GemmP& p, uint32_t taddr, float* tile_s, int t, int row0, int row,
+                                          bool row_ok, int nrows, int n0, int half, int lane, Wait wait) {
+    constexpr int UNITS = BN / 64;                        // 32-column units per warp
+    auto fetch = [&](int u, float* h) {
+        const int col = n0 + (half * UNITS + u) * 32 + lane;
+        const bool col_ok = col < p.N;
+        const float* hp = p.h_in + (size_t)(p.n_sum > 1 ? 0 : t) * p.h_in_tstride + (size_t)row0 * p.N + col;
+#pragma unroll
+        for (int rr = 0; rr < 32; ++rr) h[rr] = (col_ok && rr < nrows) ? hp[(size_t)rr * p.N] : 0.f;
+        for (int tt = 1; tt < p.n_sum; ++tt) {
+            hp += p.h_in_tstride;
+#pragma unroll
+            for (int rr = 0; rr < 32; ++rr) if (col_ok && rr < nrows) h[rr] += hp[(size_t)rr * p.N];
+        }
+    };
+    float hres[2][32];
+    fetch(0, hres[0]);
+    if (!wait()) return false;
+    float ssq = 0.f;
+#pragma unroll
+    for (int u = 0; u < UNITS; ++u) {
+        const int c = (half * UNITS + u) * 32;
+        if (n0 + c >= p.N) break;                          // uniform across the warp
+        float v[32];
+        tc_ld16(taddr + c, v);
+        tc_ld16(taddr + c + 16, v + 16);
+        if (u + 1 < UNITS) fetch(u + 1, hres[(u + 1) & 1]);
+        const int col = n0 + c + lane;
+        const bool col_ok = col < p.N;
+        // column domain: residual values into the staging tile
+#pragma unroll
+        for (int rr = 0; rr < 32; ++rr) tile_s[rr * kPitch + lane] = hres[u & 1][rr];
+        __syncwarp();
+        tc_wait_ld();
+        // row domain: add, scale, statistics
+        if (lane < nrows) {
+#pragma unroll
+            for (int k = 0; k < 32; ++k) {
+                const float x = (v[k] + tile_s[lane * kPitch + k]) * p.scale;
+                ssq += x * x;
+                tile_s[lane * kPitch + k] = x;
+            }
+        }
+        __syncwarp();
+        // column domain: stream out, and the next GEMM's operand for every track that continues from it
+        if (col_ok) {
+            float* ho = p.h_out + (size_t)t * p.h_out_tstride + (size_t)row0 * p.N + col;
+#pragma unroll 8
+            for (int rr = 0; rr < 32; ++rr) if (rr < nrows) ho[(size_t)rr * p.N] = tile_s[rr * kPitch + lane];
+            if (p.hb_out) {
+                for (int to = 0; to < p.n_out; ++to) {
+                    const int tg = p.n_out > 1 ? to : t;
+                    const float g = p.gain[(size_t)tg * p.N + col];
+                    __nv_bfloat16* hb = p.hb_out + ((size_t)tg * p.M + row0) * p.N + col;
+#pragma unroll 8
+                    for (int rr = 0; rr < 32; ++rr) if (rr < nrows) hb[(size_t)rr * p.N] = __float2bfloat16_rn(tile_s[rr * kPitch + lane] * g);
+                }
+            }
+        }
+        __syncwarp();
+        if ((u & 1) == 1 || n0 + c + 32 >= p.N) {          // a kSsqTile-column group is complete
+            if (row_ok && p.ssq_out)
+                p.ssq_out[(size_t)t * p.ssq_out_tstride + (size_t)row * p.ssq_out_tiles + (n0 + c) / kSsqTile] = ssq;
+            ssq = 0.f;
+        }
+    }
+    return true;
+}
+
+template <int BN, int EPI, class Wait>
+__device__ __forceinline__ bool epilogue(const GemmP& p, uint32_t taddr, float* tile_s, int t, int row0, int row,
+                                         bool row_ok, int nrows, int n0, int half, int lane, Wait wait) {
+    if (EPI == EPI_PLAIN) return epi_plain<BN>(p, taddr, tile_s, t, row0, nrows, n0, half, lane, wait);
+    else if (EPI == EPI_QKV) return epi_qkv<BN>(p, taddr, tile_s, t, row0, row, row_ok, nrows, n0, half, lane, wait);
+    else if (EPI == EPI_SWIGLU) return epi_swiglu<BN>(p, taddr, tile_s, t, row0, row, row_ok, nrows, n0, half, lane, wait);
+    else return epi_resid<BN>(p, taddr, tile_s, t, row0, row, row_ok, nrows, n0, half, lane, wait);
+}
+
 template <int BN, int EPI>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_tc(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensorMap tb, const GemmP p) {
     using C = Cfg<BN>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint64_t* full = (uint64_t*)(smem + C::STAGES * C::STAGE_BYTES);
+    float* stage_tiles = (float*)(smem + C::RING_BYTES);
+    uint64_t* full = (uint64_t*)(smem + C::RING_BYTES + kEpiWarps * kStageTileBytes);
     uint64_t* empty = full + C::STAGES;
     uint64_t* acc_full = empty + C::STAGES;
     uint64_t* acc_empty = acc_full + 2;
@@ -128,7 +386,7 @@ gemm_tc(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensor
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 4); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], kEpiWarps); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -166,183 +424,59 @@ gemm_tc(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensor
         }
         __syncwarp();
     } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-            int s = 0; uint32_t ph = 0;
-            int a = 0; uint32_t aph = 0;
-            bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                if (!mbar_wait(&acc_empty[a], aph ^ 1, abort_flag)) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_ACC_WAIT); *abort_flag = 1; break; }
-                tc_fence_after();
-                uint32_t d_tmem = tmem_base + a * BN;
-                for (int kb = 0; kb < kblocks; ++kb) {
-                    if (!mbar_wait(&full[s], ph, abort_flag)) { ok = false; report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_TMA_WAIT); *abort_flag = 1; break; }
-                    tc_fence_after();
-                    uint32_t sa = smem_u32(smem + s * C::STAGE_BYTES);
-                    uint64_t da = smem_desc(sa), db = smem_desc(sa + C::A_BYTES);
-#pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)
-                        tc_mma(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
-                    tc_commit(&empty[s]);                 // frees the stage when these MMAs retire
-                    if (++s == C::STAGES) { s = 0; ph ^= 1; }
-                }
-                if (!ok) break;
-                tc_commit(&acc_full[a]);                  // accumulator complete
-                if (++a == 2) { a = 0; aph ^= 1; }
+        // whole warp walks the loop; the tcgen05 instructions run on one elected lane
+        constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+        const uint64_t desc0 = smem_desc(smem_u32(smem));
+        int s = 0; uint32_t ph = 0;
+        int a = 0; uint32_t aph = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            if (!__all_sync(0xffffffffu, mbar_wait(&acc_empty[a], aph ^ 1, abort_flag))) {
+                if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_ACC_WAIT); *abort_flag = 1; }
+                break;
             }
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + a * BN;
+            for (int kb = 0; kb < kblocks; ++kb) {
+                if (!__all_sync(0xffffffffu, mbar_wait(&full[s], ph, abort_flag))) {
+                    ok = false;
+                    if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_TMA_WAIT); *abort_flag = 1; }
+                    break;
+                }
+                tc_fence_after();
+                const uint64_t da = desc0 + (uint64_t)((s * C::STAGE_BYTES) >> 4), db = da + (uint64_t)(C::A_BYTES >> 4);
+#pragma unroll
+                for (int k = 0; k < BK / 16; ++k)
+                    tc_mma(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+                tc_commit(&empty[s]);                     // frees the stage when these MMAs retire
+                if (++s == C::STAGES) { s = 0; ph ^= 1; }
+            }
+            if (!ok) break;
+            tc_commit(&acc_full[a]);                      // accumulator complete
+            if (++a == 2) { a = 0; aph ^= 1; }
         }
         __syncwarp();
     } else {
-        const int ew = warp & 3;                           // TMEM lane quarter this warp may read
+        const int q = warp & 3;                            // TMEM lane quarter this warp may read
+        const int half = (warp - 2) >> 2;                  // which half of the tile's 32-column units it takes
+        float* tile_s = stage_tiles + (warp - 2) * (32 * kPitch);
         int a = 0; uint32_t aph = 0;
         for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
             int nt = tile % p.tiles_n, mt = (tile / p.tiles_n) % p.tiles_m, t = tile / (p.tiles_n * p.tiles_m);
-            bool ok = mbar_wait(&acc_full[a], aph, abort_flag);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) { if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_EPI_WAIT); *abort_flag = 1; } break; }
-            tc_fence_after();
-            const int row = mt * BM + ew * 32 + lane;
+            const int row0 = mt * BM + q * 32;             // first row of this warp
+            const int row = row0 + lane;                   // the row this thread holds after tcgen05.ld
             const bool row_ok = row < p.M;
+            const int nrows = min(32, p.M - row0);         // rows of this warp inside the matrix (may be <= 0)
             const int n0 = nt * BN;
-            const uint32_t taddr = tmem_base + ((uint32_t)(ew * 32) << 16) + a * BN;
-            const size_t trow = (size_t)t * p.M + row;
-
-            float rinv = 1.f;
-            if ((EPI == EPI_QKV || EPI == EPI_SWIGLU) && row_ok) {
-                const float* sp = p.ssq_in + (size_t)t * p.ssq_in_tstride + (size_t)row * p.ssq_tiles;
-                float s = 0.f;
-                for (int i = 0; i < p.ssq_tiles; ++i) s += sp[i];
-                rinv = 1.0f / sqrtf(s / (float)p.K + p.eps);
-            }
-
-            if (EPI == EPI_PLAIN) {
-                for (int c = 0; c < BN; c += 16) {
-                    float v[16];
-                    tc_ld16(taddr + c, v);
-                    tc_wait_ld();
-                    if (row_ok && n0 + c < p.N) {
-                        float4* dst = (float4*)(p.c_out + trow * p.N + n0 + c);
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-                    }
-                }
-            } else if (EPI == EPI_QKV) {
-                const int dh = p.dh, half = dh >> 1;
-                int pos = 0; int64_t kvoff = 0;
-                if (row_ok) { pos = p.row_pos[row]; kvoff = p.row_kvoff[row]; }
-                bool slot_ok = row_ok && kvoff >= 0 && kvoff + (int64_t)(2 * p.nkv - 1) * p.ps * dh + dh <= p.slab_elems;
-                if (row_ok && !slot_ok) report(p.status, PT_ERR_DEVICE_BOUNDS, LOC_ROPE_PAGE);
-                const float* cs = p.cs + (size_t)pos * half;
-                const float* sn = p.sn + (size_t)pos * half;
-                for (int hc = 0; hc < BN; hc += dh) {
-                    const int col = n0 + hc;
-                    if (col >= p.N) break;                              // uniform across the CTA
-                    const int hs = col / dh;                            // head slot: q heads, k heads, v heads
-                    __nv_bfloat16* dst;
-                    bool st_ok;
-                    if (hs < p.nq) { dst = p.q_out + trow * (size_t)(p.nq * dh) + (size_t)hs * dh; st_ok = row_ok; }
-                    else {
-                        int kv = hs >= p.nq + p.nkv, head = hs - p.nq - kv * p.nkv;
-                        dst = p.pool_l + (size_t)t * p.pool_tstride + kvoff + ((int64_t)kv * p.nkv + head) * p.ps * dh;
-                        st_ok = slot_ok;
-                    }
-                    if (hs < p.nq + p.nkv) {
-                        for (int j0 = 0; j0 < half; j0 += 16) {
-                            float lo[16], hi[16];
-                            tc_ld16(taddr + hc + j0, lo);
-                            tc_ld16(taddr + hc + half + j0, hi);
-                            tc_wait_ld();
-                            if (st_ok) {
-                                float c[16], s[16];
-#pragma unroll
-                                for (int i = 0; i < 4; ++i) {
-                                    float4 cv = ((const float4*)(cs + j0))[i], sv = ((const float4*)(sn + j0))[i];
-                                    c[4 * i] = cv.x; c[4 * i + 1] = cv.y; c[4 * i + 2] = cv.z; c[4 * i + 3] = cv.w;
-                                    s[4 * i] = sv.x; s[4 * i + 1] = sv.y; s[4 * i + 2] = sv.z; s[4 * i + 3] = sv.w;
-                                }
-#pragma unroll
-                                for (int i = 0; i < 16; ++i) {
-                                    float l = lo[i] * rinv, h = hi[i] * rinv;
-                                    lo[i] = l * c[i] - h * s[i];
-                                    hi[i] = h * c[i] + l * s[i];
-                                }
-                                store16_bf16(dst + j0, lo);
-                                store16_bf16(dst + half + j0, hi);
-                            }
-                        }
-                    } else {
-                        for (int j0 = 0; j0 < dh; j0 += 16) {
-                            float v[16];
-                            tc_ld16(taddr + hc + j0, v);
-                            tc_wait_ld();
-                            if (st_ok) {
-#pragma unroll
-                                for (int i = 0; i < 16; ++i) v[i] *= rinv;
-                                store16_bf16(dst + j0, v);
-                            }
-                        }
-                    }
-                }
-            } else if (EPI == EPI_SWIGLU) {
-                for (int c = 0; c < BN; c += 32) {
-                    if (n0 + c >= p.N) break;
-                    float g[16], u[16];
-                    tc_ld16(taddr + c, g);
-                    tc_ld16(taddr + c + 16, u);
-                    tc_wait_ld();
-                    if (row_ok) {
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            float gv = g[i] * rinv, uv = u[i] * rinv;
-                            g[i] = gv / (1.0f + __expf(-gv)) * uv;
-                        }
-                        store16_bf16(p.z_out + trow * (size_t)(p.N >> 1) + ((n0 + c) >> 1), g);
-                    }
-                }
-            } else {  // EPI_RESID
-                float ssq = 0.f;
-                for (int c = 0; c < BN; c += 16) {
-                    if (n0 + c >= p.N) break;
-                    float v[16];
-                    tc_ld16(taddr + c, v);
-                    tc_wait_ld();
-                    if (row_ok) {
-                        const size_t eo = (size_t)row * p.N + n0 + c;
-                        for (int tt = 0; tt < p.n_sum; ++tt) {
-                            const float4* hp = (const float4*)(p.h_in + (size_t)(p.n_sum > 1 ? tt : t) * p.h_in_tstride + eo);
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) { float4 h = hp[i]; v[4 * i] += h.x; v[4 * i + 1] += h.y; v[4 * i + 2] += h.z; v[4 * i + 3] += h.w; }
-                        }
-                        if (p.scale != 1.0f) {
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) v[i] *= p.scale;
-                        }
-                        float4* ho = (float4*)(p.h_out + (size_t)t * p.h_out_tstride + eo);
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) ho[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) ssq += v[i] * v[i];
-                        if (p.hb_out) {
-                            for (int to = 0; to < p.n_out; ++to) {
-                                const int tg = p.n_out > 1 ? to : t;
-                                const float* gp = p.gain + (size_t)tg * p.N + n0 + c;
-                                float w[16];
-#pragma unroll
-                                for (int i = 0; i < 4; ++i) {
-                                    float4 g = ((const float4*)gp)[i];
-                                    w[4 * i] = v[4 * i] * g.x; w[4 * i + 1] = v[4 * i + 1] * g.y; w[4 * i + 2] = v[4 * i + 2] * g.z; w[4 * i + 3] = v[4 * i + 3] * g.w;
-                                }
-                                store16_bf16(p.hb_out + ((size_t)tg * p.M + row) * p.N + n0 + c, w);
-                            }
-                        }
-                    }
-                    if (((c + 16) % kSsqTile) == 0 || n0 + c + 16 >= p.N) {
-                        if (row_ok && p.ssq_out)
-                            p.ssq_out[(size_t)t * p.ssq_out_tstride + (size_t)row * p.ssq_out_tiles + (n0 + c) / kSsqTile] = ssq;
-                        ssq = 0.f;
-                    }
-                }
-            }
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN;
+            auto wait_acc = [&]() -> bool {
+                bool ok = mbar_wait(&acc_full[a], aph, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) { if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_EPI_WAIT); *abort_flag = 1; } return false; }
+                tc_fence_after();
+                return true;
+            };
+            if (!epilogue<BN, EPI>(p, taddr, tile_s, t, row0, row, row_ok, nrows, n0, half, lane, wait_acc)) break;
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[a]);
@@ -385,7 +519,7 @@ pt_status launch_t(const CUtensorMap& ta, const CUtensorMap& tb, GemmP p, cudaSt
     p.tiles_n = (p.N + BN - 1) / BN;
     int tiles = p.tiles_m * p.tiles_n * p.T;
     int grid = std::min(tiles, sms);
-    gemm_tc<BN, EPI><<<grid, 192, C::SMEM, st>>>(ta, tb, p);
+    gemm_tc<BN, EPI><<<grid, kGemmThreads, C::SMEM, st>>>(ta, tb, p);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return PT_OK;
 }
