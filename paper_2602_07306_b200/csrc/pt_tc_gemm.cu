@@ -11,14 +11,11 @@
 //               fp32 stream out, gain-scaled bf16 copy for the next GEMM, partial sums of squares
 //               for the next RMSNorm
 //   EPI_PLAIN   fp32 C (kernel-level tests)
-// Epilogue data path: a warp owns 32 accumulator rows (its tensor-memory lane quarter) and works in
-// units of 32 columns.  tcgen05.ld hands every thread one row; whatever needs the whole row
-// (1/rms, SiLU pairing, the sum of squares) happens there.  The unit then goes through a padded
-// 32 x 33 shared-memory tile so that the global loads and stores run with lane = column: every
-// instruction touches one contiguous 64- or 128-byte piece of one row instead of 32 rows.  Global
-// loads that do not depend on the accumulator (row statistics, rotary table, residual rows) are
-// issued before the wait for the accumulator and one unit ahead, so their latency hides behind
-// the tensor pipe.
+// Epilogue data path: a warp owns 32 accumulator rows (its tensor-memory lane quarter); the two
+// warps of a quarter split the tile's columns.  tcgen05.ld hands every thread one row, and the
+// thread reads and writes whole 32-byte sectors of that row.  Global loads that do not depend on
+// the accumulator (row statistics, rotary table, residual rows) are issued before the wait for
+// the accumulator and one 32-column unit ahead, so their latency hides behind the tensor pipe.
 // Every mbarrier wait is bounded; on a timeout the CTA records PT_ERR_DEVICE_TIMEOUT, stops
 // issuing work, frees its tensor memory and exits.
 #include "pt_tc.h"
@@ -30,8 +27,6 @@ namespace {
 constexpr int BM = 128, BK = 64;
 constexpr int kEpiWarps = 8;
 constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
-constexpr int kPitch = 33;                         // floats per row of a staging tile (odd: no bank conflicts)
-constexpr int kStageTileBytes = 32 * kPitch * 4;
 constexpr uint32_t kSpinLimit = 1u << 26;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -113,16 +108,27 @@ template <int BN> struct Cfg {
     static constexpr int B_BYTES = BN * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int RING_BYTES = STAGES * STAGE_BYTES;
-    static constexpr int SMEM = RING_BYTES + kEpiWarps * kStageTileBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static constexpr int SMEM = RING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
 // ---- epilogue ------------------------------------------------------------------------------
-// Row domain: after tcgen05.ld thread `lane` holds columns of row row0 + lane.  Column domain:
-// after the trip through the staging tile lane `l` holds column l of each of the warp's rows in
-// turn.
-__device__ __forceinline__ void put_row(float* tile_s, int lane, const float* v) {
-#pragma unroll
-    for (int k = 0; k < 32; ++k) tile_s[lane * kPitch + k] = v[k];
+// tcgen05.ld hands every thread one accumulator row (row0 + lane); a warp works through its share
+// of the tile's columns in units of 32.  Each thread reads and writes 64- or 128-byte pieces of
+// its own row (whole 32-byte sectors).  Global loads that do not depend on the accumulator (row
+// statistics, rotary table, residual rows) are issued before the wait for the accumulator and one
+// unit ahead of their use, so their latency hides behind the tensor pipe and the previous unit.
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+// 16 floats -> 16 bf16 (32 bytes, two 16-byte stores)
+__device__ __forceinline__ void store16_bf16(__nv_bfloat16* dst, const float* v) {
+    uint4 a, b;
+    a.x = pack_bf16(v[0], v[1]); a.y = pack_bf16(v[2], v[3]); a.z = pack_bf16(v[4], v[5]); a.w = pack_bf16(v[6], v[7]);
+    b.x = pack_bf16(v[8], v[9]); b.y = pack_bf16(v[10], v[11]); b.z = pack_bf16(v[12], v[13]); b.w = pack_bf16(v[14], v[15]);
+    reinterpret_cast<uint4*>(dst)[0] = a;
+    reinterpret_cast<uint4*>(dst)[1] = b;
 }
 
 // 1 / rms of this thread's row from the producer's partial sums of squares.
@@ -134,13 +140,11 @@ __device__ __forceinline__ float row_rinv(const GemmP& p, int t, int row, bool r
     return 1.0f / sqrtf(s / (float)p.K + p.eps);
 }
 
-// Every epilogue first issues whatever global loads do not depend on the accumulator, then calls
-// wait() for the accumulator: the loads are in flight while the tensor pipe still works on the tile.
 template <int BN, class Wait>
-__device__ __forceinline__ bool epi_plain(const GemmP& p, uint32_t taddr, float* tile_s, int t, int row0, int nrows,
-                                          int n0, int half, int lane, Wait wait) {
+__device__ __forceinline__ bool epi_plain(const GemmP& p, uint32_t taddr, int t, int row, bool row_ok, int n0, int half, Wait wait) {
     constexpr int UNITS = BN / 64;                        // 32-column units per warp
     if (!wait()) return false;
+#pragma unroll 1
     for (int u = 0; u < UNITS; ++u) {
         const int c = (half * UNITS + u) * 32;
         if (n0 + c >= p.N) break;                          // uniform across the warp
@@ -148,15 +152,12 @@ __device__ __forceinline__ bool epi_plain(const GemmP& p, uint32_t taddr, float*
         tc_ld16(taddr + c, v);
         tc_ld16(taddr + c + 16, v + 16);
         tc_wait_ld();
-        put_row(tile_s, lane, v);
-        __syncwarp();
-        const int col = n0 + c + lane;
-        if (col < p.N) {
-            float* dst = p.c_out + ((size_t)t * p.M + row0) * p.N + col;
-#pragma unroll 8
-            for (int rr = 0; rr < 32; ++rr) if (rr < nrows) dst[(size_t)rr * p.N] = tile_s[rr * kPitch + lane];
+        if (row_ok) {
+            float4* dst = (float4*)(p.c_out + ((size_t)t * p.M + row) * p.N + n0 + c);
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if (n0 + c + 4 * i < p.N) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
         }
-        __syncwarp();
     }
     return true;
 }
@@ -164,47 +165,39 @@ __device__ __forceinline__ bool epi_plain(const GemmP& p, uint32_t taddr, float*
 // Accumulator columns come in groups of 32: 16 gate columns followed by their 16 up columns.  A
 // unit here is 64 accumulator columns = 32 outputs z = silu(gate / rms) * (up / rms).
 template <int BN, class Wait>
-__device__ __forceinline__ bool epi_swiglu(const GemmP& p, uint32_t taddr, float* tile_s, int t, int row0, int row,
-                                           bool row_ok, int nrows, int n0, int half, int lane, Wait wait) {
+__device__ __forceinline__ bool epi_swiglu(const GemmP& p, uint32_t taddr, int t, int row, bool row_ok, int n0, int half, Wait wait) {
     constexpr int UNITS = BN / 128;                       // 64-column units per warp
     const float rinv = row_rinv(p, t, row, row_ok);
     const int F = p.N >> 1;
     if (!wait()) return false;
+#pragma unroll 1
     for (int u = 0; u < UNITS; ++u) {
         const int c = (half * UNITS + u) * 64;
         if (n0 + c >= p.N) break;
-        float z[32], gu[64];
+        float gu[64];
 #pragma unroll
         for (int g4 = 0; g4 < 4; ++g4) tc_ld16(taddr + c + g4 * 16, gu + g4 * 16);
         tc_wait_ld();
 #pragma unroll
         for (int g2 = 0; g2 < 2; ++g2) {
+            float z[16];
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
                 const float gv = gu[g2 * 32 + i] * rinv, uv = gu[g2 * 32 + 16 + i] * rinv;
-                z[g2 * 16 + i] = __fdividef(gv, 1.0f + __expf(-gv)) * uv;
+                z[i] = __fdividef(gv, 1.0f + __expf(-gv)) * uv;
             }
+            const int zc = ((n0 + c) >> 1) + g2 * 16;      // first output column of this group
+            if (row_ok && zc < F) store16_bf16(p.z_out + ((size_t)t * p.M + row) * F + zc, z);
         }
-        put_row(tile_s, lane, z);
-        __syncwarp();
-        const int zc = ((n0 + c) >> 1) + lane;             // output column of this lane
-        if (zc < F) {
-            __nv_bfloat16* dst = p.z_out + ((size_t)t * p.M + row0) * F + zc;
-#pragma unroll 8
-            for (int rr = 0; rr < 32; ++rr) if (rr < nrows) dst[(size_t)rr * F] = __float2bfloat16_rn(tile_s[rr * kPitch + lane]);
-        }
-        __syncwarp();
     }
     return true;
 }
 
 // A unit is 32 accumulator columns of one head: for q and k heads the 16 columns j0..j0+15 and
-// their rotary partners j0+dh/2.., for v heads 32 consecutive columns.  In the column domain
-// lanes 0-15 hold a unit's low columns and fetch cos, lanes 16-31 hold the partners and fetch
-// sin; one shuffle pairs them up.  The table entries of a unit are fetched one unit ahead.
+// their rotary partners j0+dh/2.., for v heads 32 consecutive columns.  The 16 cos and 16 sin
+// values of the row's position are fetched one unit ahead.
 template <int BN, class Wait>
-__device__ __forceinline__ bool epi_qkv(const GemmP& p, uint32_t taddr, float* tile_s, int t, int row0, int row,
-                                        bool row_ok, int nrows, int n0, int half, int lane, Wait wait) {
+__device__ __forceinline__ bool epi_qkv(const GemmP& p, uint32_t taddr, int t, int row, bool row_ok, int n0, int half, Wait wait) {
     constexpr int UNITS = BN / 64;                        // units per warp
     const int dh = p.dh, halfdh = dh >> 1, upd = dh >> 5;  // units per head
     const int heads_total = p.nq + 2 * p.nkv;
@@ -213,160 +206,156 @@ __device__ __forceinline__ bool epi_qkv(const GemmP& p, uint32_t taddr, float* t
     const float rinv = row_rinv(p, t, row, row_ok);
     const bool slot_ok = row_ok && kvoff >= 0 && kvoff + (int64_t)(2 * p.nkv - 1) * p.ps * dh + dh <= p.slab_elems;
     if (row_ok && !slot_ok) report(p.status, PT_ERR_DEVICE_BOUNDS, LOC_ROPE_PAGE);
-    const uint32_t slot_mask = __ballot_sync(0xffffffffu, slot_ok);
-    const int kv_lo = (int)(uint32_t)(kvoff & 0xffffffffll), kv_hi = (int)(kvoff >> 32);
-    const float* table = lane < 16 ? p.cs : p.sn;
-    // cos (lanes 0-15) or sin (lanes 16-31) of this lane's column for each of the warp's rows
-    auto fetch = [&](int uu, float* tab) {
+    const float4* cs4 = (const float4*)(p.cs + (size_t)pos * halfdh);
+    const float4* sn4 = (const float4*)(p.sn + (size_t)pos * halfdh);
+    auto fetch = [&](int uu, float4* tab) {               // tab[0..3] = cos, tab[4..7] = sin of columns j0..j0+15
         const int u = half * UNITS + uu;
         const int hs = n0 / dh + u / upd;
-        if (hs >= p.nq + p.nkv) return;                    // v heads and columns past N: no rotation
-        const int j = (u % upd) * 16 + (lane & 15);
+        if (hs >= p.nq + p.nkv || !row_ok) return;         // v heads, columns past N, rows past M: no rotation
+        const int j4 = (u % upd) * 4;
 #pragma unroll
-        for (int rr = 0; rr < 32; ++rr) {
-            const int pr = __shfl_sync(0xffffffffu, pos, rr);
-            tab[rr] = rr < nrows ? table[(size_t)pr * halfdh + j] : 0.f;
-        }
+        for (int i = 0; i < 4; ++i) { tab[i] = cs4[j4 + i]; tab[4 + i] = sn4[j4 + i]; }
     };
-    float tab[2][32];
-    fetch(0, tab[0]);
+    float4 tab[8], nxt[8];
+    fetch(0, tab);
     if (!wait()) return false;
-#pragma unroll
+#pragma unroll 1
     for (int uu = 0; uu < UNITS; ++uu) {
         const int u = half * UNITS + uu;
         const int hc = u / upd, sub = u % upd;
         const int hs = n0 / dh + hc;                       // head slot: q heads, then k heads, then v heads
         if (hs >= heads_total) break;                      // uniform across the warp
         const bool is_v = hs >= p.nq + p.nkv;
-        if (uu + 1 < UNITS) fetch(uu + 1, tab[(uu + 1) & 1]);
-        float v[32];
-        if (!is_v) {
-            tc_ld16(taddr + hc * dh + sub * 16, v);
-            tc_ld16(taddr + hc * dh + halfdh + sub * 16, v + 16);
-        } else {
-            tc_ld16(taddr + hc * dh + sub * 32, v);
-            tc_ld16(taddr + hc * dh + sub * 32 + 16, v + 16);
-        }
-        tc_wait_ld();
-#pragma unroll
-        for (int k = 0; k < 32; ++k) v[k] *= rinv;
-        put_row(tile_s, lane, v);
-        __syncwarp();
-        // column domain
-        const int j = sub * 16 + (lane & 15);
-        const int col = is_v ? sub * 32 + lane : (lane < 16 ? j : j + halfdh);      // column inside the head
-        __nv_bfloat16* qdst = nullptr;
-        int64_t head_off = 0;
+        float lo[16], hi[16];
+        const int c_lo = hc * dh + (is_v ? sub * 32 : sub * 16);
+        const int c_hi = is_v ? c_lo + 16 : c_lo + halfdh;
+        tc_ld16(taddr + c_lo, lo);
+        tc_ld16(taddr + c_hi, hi);
+        if (uu + 1 < UNITS) fetch(uu + 1, nxt);
+        __nv_bfloat16* dst;
+        bool st_ok;
         if (hs < p.nq) {
-            qdst = p.q_out + ((size_t)t * p.M + row0) * (size_t)(p.nq * dh) + (size_t)hs * dh + col;
+            dst = p.q_out + ((size_t)t * p.M + row) * (size_t)(p.nq * dh) + (size_t)hs * dh;
+            st_ok = row_ok;
         } else {
             const int kv = is_v ? 1 : 0, head = hs - p.nq - kv * p.nkv;
-            head_off = (int64_t)t * p.pool_tstride + ((int64_t)kv * p.nkv + head) * p.ps * dh + col;
+            dst = p.pool_l + (size_t)t * p.pool_tstride + kvoff + ((int64_t)kv * p.nkv + head) * p.ps * dh;
+            st_ok = slot_ok;
         }
-        const float* tb = tab[uu & 1];
-#pragma unroll
-        for (int rr = 0; rr < 32; ++rr) {
-            float y = tile_s[rr * kPitch + lane];
+        tc_wait_ld();
+        if (st_ok) {
             if (!is_v) {
-                const float partner = __shfl_xor_sync(0xffffffffu, y, 16);
-                const float other = __shfl_xor_sync(0xffffffffu, tb[rr], 16);   // sin for the low lanes, cos for the high
-                // low column: x cos - x' sin;  partner column: x' cos + x sin
-                y = lane < 16 ? y * tb[rr] - partner * other : y * other + partner * tb[rr];
-            }
-            if (qdst) {
-                if (rr < nrows) qdst[(size_t)rr * (p.nq * dh)] = __float2bfloat16_rn(y);
-            } else {
-                const int lo = __shfl_sync(0xffffffffu, kv_lo, rr), hi = __shfl_sync(0xffffffffu, kv_hi, rr);
-                if (rr < nrows && ((slot_mask >> rr) & 1u)) {
-                    const int64_t off = ((int64_t)hi << 32) | (uint32_t)lo;
-                    p.pool_l[off + head_off] = __float2bfloat16_rn(y);
+                float c[16], s[16];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    c[4 * i] = tab[i].x; c[4 * i + 1] = tab[i].y; c[4 * i + 2] = tab[i].z; c[4 * i + 3] = tab[i].w;
+                    s[4 * i] = tab[4 + i].x; s[4 * i + 1] = tab[4 + i].y; s[4 * i + 2] = tab[4 + i].z; s[4 * i + 3] = tab[4 + i].w;
                 }
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const float l = lo[i] * rinv, h = hi[i] * rinv;
+                    lo[i] = l * c[i] - h * s[i];
+                    hi[i] = h * c[i] + l * s[i];
+                }
+                store16_bf16(dst + sub * 16, lo);
+                store16_bf16(dst + halfdh + sub * 16, hi);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) { lo[i] *= rinv; hi[i] *= rinv; }
+                store16_bf16(dst + sub * 32, lo);
+                store16_bf16(dst + sub * 32 + 16, hi);
             }
         }
-        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < 8; ++i) tab[i] = nxt[i];       // last: the fetch stays in flight until here
     }
     return true;
 }
 
 // Residual add (+ track-sync sum), fp32 stream out, gain-scaled bf16 copy, partial sums of squares.
-// The residual rows of a unit are fetched (lane = column) one unit ahead of their use.
+// The 32 residual values of a unit (128 bytes of the thread's row) are fetched one unit ahead.
 template <int BN, class Wait>
-__device__ __forceinline__ bool epi_resid(const GemmP& p, uint32_t taddr, float* tile_s, int t, int row0, int row,
-                                          bool row_ok, int nrows, int n0, int half, int lane, Wait wait) {
+__device__ __forceinline__ bool epi_resid(const GemmP& p, uint32_t taddr, int t, int row, bool row_ok, int n0, int half, Wait wait) {
     constexpr int UNITS = BN / 64;                        // 32-column units per warp
-    auto fetch = [&](int u, float* h) {
-        const int col = n0 + (half * UNITS + u) * 32 + lane;
-        const bool col_ok = col < p.N;
-        const float* hp = p.h_in + (size_t)(p.n_sum > 1 ? 0 : t) * p.h_in_tstride + (size_t)row0 * p.N + col;
+    const float* hrow = p.h_in + (size_t)(p.n_sum > 1 ? 0 : t) * p.h_in_tstride + (size_t)row * p.N;
+    auto fetch = [&](int u, float4* h) {
+        const int col = n0 + (half * UNITS + u) * 32;
 #pragma unroll
-        for (int rr = 0; rr < 32; ++rr) h[rr] = (col_ok && rr < nrows) ? hp[(size_t)rr * p.N] : 0.f;
-        for (int tt = 1; tt < p.n_sum; ++tt) {
-            hp += p.h_in_tstride;
+        for (int i = 0; i < 8; ++i) h[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (!row_ok) return;
+        for (int tt = 0; tt < p.n_sum; ++tt) {
+            const float4* hp = (const float4*)(hrow + (size_t)tt * p.h_in_tstride + col);
 #pragma unroll
-            for (int rr = 0; rr < 32; ++rr) if (col_ok && rr < nrows) h[rr] += hp[(size_t)rr * p.N];
+            for (int i = 0; i < 8; ++i)
+                if (col + 4 * i < p.N) { const float4 x = hp[i]; h[i].x += x.x; h[i].y += x.y; h[i].z += x.z; h[i].w += x.w; }
         }
     };
-    float hres[2][32];
-    fetch(0, hres[0]);
+    float4 hres[8], hnxt[8];
+    fetch(0, hres);
     if (!wait()) return false;
     float ssq = 0.f;
-#pragma unroll
+#pragma unroll 1
     for (int u = 0; u < UNITS; ++u) {
         const int c = (half * UNITS + u) * 32;
-        if (n0 + c >= p.N) break;                          // uniform across the warp
+        const int col = n0 + c;
+        if (col >= p.N) break;                             // uniform across the warp
         float v[32];
         tc_ld16(taddr + c, v);
         tc_ld16(taddr + c + 16, v + 16);
-        if (u + 1 < UNITS) fetch(u + 1, hres[(u + 1) & 1]);
-        const int col = n0 + c + lane;
-        const bool col_ok = col < p.N;
-        // column domain: residual values into the staging tile
-#pragma unroll
-        for (int rr = 0; rr < 32; ++rr) tile_s[rr * kPitch + lane] = hres[u & 1][rr];
-        __syncwarp();
+        if (u + 1 < UNITS) fetch(u + 1, hnxt);
         tc_wait_ld();
-        // row domain: add, scale, statistics
-        if (lane < nrows) {
+        if (row_ok) {
 #pragma unroll
-            for (int k = 0; k < 32; ++k) {
-                const float x = (v[k] + tile_s[lane * kPitch + k]) * p.scale;
-                ssq += x * x;
-                tile_s[lane * kPitch + k] = x;
+            for (int i = 0; i < 8; ++i) {
+                v[4 * i] = (v[4 * i] + hres[i].x) * p.scale; v[4 * i + 1] = (v[4 * i + 1] + hres[i].y) * p.scale;
+                v[4 * i + 2] = (v[4 * i + 2] + hres[i].z) * p.scale; v[4 * i + 3] = (v[4 * i + 3] + hres[i].w) * p.scale;
             }
-        }
-        __syncwarp();
-        // column domain: stream out, and the next GEMM's operand for every track that continues from it
-        if (col_ok) {
-            float* ho = p.h_out + (size_t)t * p.h_out_tstride + (size_t)row0 * p.N + col;
-#pragma unroll 8
-            for (int rr = 0; rr < 32; ++rr) if (rr < nrows) ho[(size_t)rr * p.N] = tile_s[rr * kPitch + lane];
+            float4* ho = (float4*)(p.h_out + (size_t)t * p.h_out_tstride + (size_t)row * p.N + col);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (col + 4 * i < p.N) {
+                    ho[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                    ssq += v[4 * i] * v[4 * i] + v[4 * i + 1] * v[4 * i + 1] + v[4 * i + 2] * v[4 * i + 2] + v[4 * i + 3] * v[4 * i + 3];
+                }
+            }
             if (p.hb_out) {
                 for (int to = 0; to < p.n_out; ++to) {
                     const int tg = p.n_out > 1 ? to : t;
-                    const float g = p.gain[(size_t)tg * p.N + col];
-                    __nv_bfloat16* hb = p.hb_out + ((size_t)tg * p.M + row0) * p.N + col;
-#pragma unroll 8
-                    for (int rr = 0; rr < 32; ++rr) if (rr < nrows) hb[(size_t)rr * p.N] = __float2bfloat16_rn(tile_s[rr * kPitch + lane] * g);
+                    const float4* gp = (const float4*)(p.gain + (size_t)tg * p.N + col);
+                    __nv_bfloat16* hb = p.hb_out + ((size_t)tg * p.M + row) * p.N + col;
+#pragma unroll
+                    for (int g2 = 0; g2 < 2; ++g2) {
+                        if (col + 16 * g2 < p.N) {
+                            float w[16];
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const float4 g = gp[4 * g2 + i];
+                                w[4 * i] = v[16 * g2 + 4 * i] * g.x; w[4 * i + 1] = v[16 * g2 + 4 * i + 1] * g.y;
+                                w[4 * i + 2] = v[16 * g2 + 4 * i + 2] * g.z; w[4 * i + 3] = v[16 * g2 + 4 * i + 3] * g.w;
+                            }
+                            store16_bf16(hb + 16 * g2, w);
+                        }
+                    }
                 }
             }
         }
-        __syncwarp();
-        if ((u & 1) == 1 || n0 + c + 32 >= p.N) {          // a kSsqTile-column group is complete
+        if ((u & 1) == 1 || col + 32 >= p.N) {             // a kSsqTile-column group is complete
             if (row_ok && p.ssq_out)
-                p.ssq_out[(size_t)t * p.ssq_out_tstride + (size_t)row * p.ssq_out_tiles + (n0 + c) / kSsqTile] = ssq;
+                p.ssq_out[(size_t)t * p.ssq_out_tstride + (size_t)row * p.ssq_out_tiles + col / kSsqTile] = ssq;
             ssq = 0.f;
         }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) hres[i] = hnxt[i];      // last: the fetch stays in flight until here
     }
     return true;
 }
 
 template <int BN, int EPI, class Wait>
-__device__ __forceinline__ bool epilogue(const GemmP& p, uint32_t taddr, float* tile_s, int t, int row0, int row,
-                                         bool row_ok, int nrows, int n0, int half, int lane, Wait wait) {
-    if (EPI == EPI_PLAIN) return epi_plain<BN>(p, taddr, tile_s, t, row0, nrows, n0, half, lane, wait);
-    else if (EPI == EPI_QKV) return epi_qkv<BN>(p, taddr, tile_s, t, row0, row, row_ok, nrows, n0, half, lane, wait);
-    else if (EPI == EPI_SWIGLU) return epi_swiglu<BN>(p, taddr, tile_s, t, row0, row, row_ok, nrows, n0, half, lane, wait);
-    else return epi_resid<BN>(p, taddr, tile_s, t, row0, row, row_ok, nrows, n0, half, lane, wait);
+__device__ __forceinline__ bool epilogue(const GemmP& p, uint32_t taddr, int t, int row, bool row_ok, int n0, int half, Wait wait) {
+    if (EPI == EPI_PLAIN) return epi_plain<BN>(p, taddr, t, row, row_ok, n0, half, wait);
+    else if (EPI == EPI_QKV) return epi_qkv<BN>(p, taddr, t, row, row_ok, n0, half, wait);
+    else if (EPI == EPI_SWIGLU) return epi_swiglu<BN>(p, taddr, t, row, row_ok, n0, half, wait);
+    else return epi_resid<BN>(p, taddr, t, row, row_ok, n0, half, wait);
 }
 
 template <int BN, int EPI>
@@ -375,8 +364,7 @@ gemm_tc(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensor
     using C = Cfg<BN>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    float* stage_tiles = (float*)(smem + C::RING_BYTES);
-    uint64_t* full = (uint64_t*)(smem + C::RING_BYTES + kEpiWarps * kStageTileBytes);
+    uint64_t* full = (uint64_t*)(smem + C::RING_BYTES);
     uint64_t* empty = full + C::STAGES;
     uint64_t* acc_full = empty + C::STAGES;
     uint64_t* acc_empty = acc_full + 2;
@@ -459,14 +447,11 @@ gemm_tc(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensor
     } else {
         const int q = warp & 3;                            // TMEM lane quarter this warp may read
         const int half = (warp - 2) >> 2;                  // which half of the tile's 32-column units it takes
-        float* tile_s = stage_tiles + (warp - 2) * (32 * kPitch);
         int a = 0; uint32_t aph = 0;
         for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
             int nt = tile % p.tiles_n, mt = (tile / p.tiles_n) % p.tiles_m, t = tile / (p.tiles_n * p.tiles_m);
-            const int row0 = mt * BM + q * 32;             // first row of this warp
-            const int row = row0 + lane;                   // the row this thread holds after tcgen05.ld
+            const int row = mt * BM + q * 32 + lane;       // the row this thread holds after tcgen05.ld
             const bool row_ok = row < p.M;
-            const int nrows = min(32, p.M - row0);         // rows of this warp inside the matrix (may be <= 0)
             const int n0 = nt * BN;
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN;
             auto wait_acc = [&]() -> bool {
@@ -476,7 +461,7 @@ gemm_tc(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensor
                 tc_fence_after();
                 return true;
             };
-            if (!epilogue<BN, EPI>(p, taddr, tile_s, t, row0, row, row_ok, nrows, n0, half, lane, wait_acc)) break;
+            if (!epilogue<BN, EPI>(p, taddr, t, row, row_ok, n0, half, wait_acc)) break;
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[a]);

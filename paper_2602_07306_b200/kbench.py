@@ -2,6 +2,7 @@
 
     python -m paper_2602_07306_b200.kbench decode --T 8 --B 64 --nq 8 --nkv 8 --dh 128 --len 2048
     python -m paper_2602_07306_b200.kbench prefill --T 8 --B 8 --S 4096 --nq 8 --nkv 8 --dh 128 [--impl 1]
+    python -m paper_2602_07306_b200.kbench layer --T 8 --B 2 --S 4096 --H 1024 --nq 8 --nkv 8 --F 2816
     python -m paper_2602_07306_b200.kbench gemm --T 8 --M 32768 --N 3072 --K 1024 [--bn 256] [--fold]
 
 Prints one JSON line: average device time per launch (CUDA events on the launching stream,
@@ -84,6 +85,40 @@ def prefill(a):
     print(json.dumps({"kernel": "prefill_attn", "ms": ms, "TFLOPs": flops / ms / 1e9, "args": vars(a)}))
 
 
+def layer(a):
+    """One PT layer of the given width (all tracks, L = D = 1) as a prefill: the four fused GEMMs and the
+    attention kernel in their real launch configuration, small enough to capture under a profiler."""
+    from paper_2602_07306_b200 import inputs as I
+    dev = torch.device("cuda:0")
+    m = pt.Model(T=a.T, D=1, L=1, hidden=a.H, heads=a.nq, kv_heads=a.nkv, ffn=a.F, dtype="bf16", max_pos=a.S, device=dev)
+    m.init_random(0)
+    cache = m.new_cache(a.B * (-(-a.S // a.ps)), a.ps)
+    g = torch.Generator(device=dev).manual_seed(0)
+    x = torch.randn((a.T, a.B, a.S, a.H), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    out = torch.empty((a.B, a.S, a.H), dtype=torch.float32, device=dev)
+    ids = list(range(a.B))
+
+    def step():
+        m.prefill(cache, x, ids, out)
+        for s_ in ids:
+            cache.truncate(s_, 0)
+    for _ in range(a.warmup):
+        step()
+    torch.cuda.synchronize()
+    m.profile(True)
+    for _ in range(a.iters):
+        step()
+    torch.cuda.synchronize()
+    prof = m.profile_read()
+    assert m.device_status() == (0, 0)
+    tok = a.B * a.S
+    fl = {"gemm_qkv": 2.0 * a.T * tok * a.H * (a.nq + 2 * a.nkv) * (a.H // a.nq), "gemm_out": 2.0 * a.T * tok * a.H * a.H,
+          "gemm_gate_up": 4.0 * a.T * tok * a.H * a.F, "gemm_down_sync": 2.0 * a.T * tok * a.H * a.F}
+    res = {k: {"ms": v[0] / max(v[1], 1), "TFLOPs": fl[k] / (v[0] / max(v[1], 1)) / 1e9 if k in fl and v[1] else None}
+           for k, v in prof.items() if v[1]}
+    print(json.dumps({"kernel": "layer", "per_launch": res, "args": vars(a)}))
+
+
 def gemm(a):
     dev = torch.device("cuda:0")
     g = torch.Generator(device=dev).manual_seed(0)
@@ -113,12 +148,15 @@ def main():
     pf = sub.add_parser("prefill")
     for k, v in dict(T=8, B=8, S=4096, start=0, nq=8, nkv=8, dh=128, ps=16, impl=0, iters=10, warmup=3).items():
         pf.add_argument("--" + k, type=int, default=v)
+    ly = sub.add_parser("layer")
+    for k, v in dict(T=8, B=2, S=4096, H=1024, nq=8, nkv=8, F=2816, ps=16, iters=3, warmup=1).items():
+        ly.add_argument("--" + k, type=int, default=v)
     gm = sub.add_parser("gemm")
     for k, v in dict(T=8, M=4096, N=3072, K=1024, bn=0, iters=20, warmup=3).items():
         gm.add_argument("--" + k, type=int, default=v)
     gm.add_argument("--fold", action="store_true")
     a = ap.parse_args()
-    {"decode": decode, "gemm": gemm, "prefill": prefill}[a.cmd](a)
+    {"decode": decode, "gemm": gemm, "prefill": prefill, "layer": layer}[a.cmd](a)
 
 
 if __name__ == "__main__":
