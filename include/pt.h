@@ -155,12 +155,13 @@ pt_status pt_workspace_bytes(const pt_model* m, int64_t max_tokens, int32_t max_
                              int32_t page_size, size_t* bytes);
 
 /* Algorithm 1 over B sequences of S new tokens each.
- *   x         device, model dtype, [T][B][S][hidden]; track t starts at x + t*x_track_stride
- *             elements (0 = every track starts from the same x, Algorithm 1's literal case)
+ *   x         device, 16-byte aligned, model dtype, [T][B][S][hidden]; track t starts at
+ *             x + t*x_track_stride elements (0 = every track starts from the same x,
+ *             Algorithm 1's literal case)
  *   seq_ids   host, int32[B], distinct; the S tokens of row b are appended to sequence
  *             seq_ids[b] at positions len..len+S-1 (pages are reserved by the call) and attend
  *             to everything cached for it, themselves included causally
- *   out_h     device, fp32 [B][S][hidden]: the activation h after the last sync
+ *   out_h     device, 32-byte aligned, fp32 [B][S][hidden]: the activation h after the last sync
  *   workspace device, 256-byte aligned, >= pt_workspace_bytes(B*S, B, page_size)
  * On success the sequences' lengths grow by S.  Errors: PT_ERR_CACHE_FULL,
  * PT_ERR_BUFFER_TOO_SMALL, PT_ERR_INVALID_ARG (position >= max_pos, duplicate ids),

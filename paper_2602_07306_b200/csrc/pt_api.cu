@@ -364,8 +364,8 @@ static pt_status forward(pt_model* m, pt_kv_cache* c, const void* x, int64_t x_s
     if (!m->wbuf) PT_FAIL(PT_ERR_STATE, "pt_model_bind_weights has not been called");
     if (B < 1 || S < 1) PT_FAIL(PT_ERR_INVALID_ARG, "B and S must be >= 1");
     if (x_stride < 0) PT_FAIL(PT_ERR_INVALID_ARG, "negative track stride");
-    if ((uintptr_t)workspace % 256 || (uintptr_t)x % 16 || (uintptr_t)out_h % 16)
-        PT_FAIL(PT_ERR_MISALIGNED, "workspace must be 256-byte aligned, x and out_h 16-byte aligned");
+    if ((uintptr_t)workspace % 256 || (uintptr_t)x % 16 || (uintptr_t)out_h % 32)
+        PT_FAIL(PT_ERR_MISALIGNED, "workspace must be 256-byte aligned, x 16-byte and out_h 32-byte aligned");
     const pt_config& g = m->cfg;
     if (x_stride % 8) PT_FAIL(PT_ERR_MISALIGNED, "x_track_stride must be a multiple of 8 elements");
     int64_t M = (int64_t)B * S;

@@ -122,13 +122,22 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&v);
 }
-// 16 floats -> 16 bf16 (32 bytes, two 16-byte stores)
+// 256-bit global accesses (32-byte aligned): every lane moves one whole sector per instruction,
+// which halves the load/store-unit work of these row-per-thread access patterns.
+__device__ __forceinline__ void ld256(const float* p, float* v) {
+    asm volatile("ld.global.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]) : "l"(p));
+}
+__device__ __forceinline__ void st256(float* p, const float* v) {
+    asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(p), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]) : "memory");
+}
+// 16 floats -> 16 bf16: one 32-byte store
 __device__ __forceinline__ void store16_bf16(__nv_bfloat16* dst, const float* v) {
-    uint4 a, b;
-    a.x = pack_bf16(v[0], v[1]); a.y = pack_bf16(v[2], v[3]); a.z = pack_bf16(v[4], v[5]); a.w = pack_bf16(v[6], v[7]);
-    b.x = pack_bf16(v[8], v[9]); b.y = pack_bf16(v[10], v[11]); b.z = pack_bf16(v[12], v[13]); b.w = pack_bf16(v[14], v[15]);
-    reinterpret_cast<uint4*>(dst)[0] = a;
-    reinterpret_cast<uint4*>(dst)[1] = b;
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(dst), "r"(pack_bf16(v[0], v[1])), "r"(pack_bf16(v[2], v[3])), "r"(pack_bf16(v[4], v[5])), "r"(pack_bf16(v[6], v[7])),
+                   "r"(pack_bf16(v[8], v[9])), "r"(pack_bf16(v[10], v[11])), "r"(pack_bf16(v[12], v[13])), "r"(pack_bf16(v[14], v[15]))
+                 : "memory");
 }
 
 // 1 / rms of this thread's row from the producer's partial sums of squares.
@@ -136,7 +145,15 @@ __device__ __forceinline__ float row_rinv(const GemmP& p, int t, int row, bool r
     if (!row_ok) return 1.f;
     const float* sp = p.ssq_in + (size_t)t * p.ssq_in_tstride + (size_t)row * p.ssq_tiles;
     float s = 0.f;
-    for (int i = 0; i < p.ssq_tiles; ++i) s += sp[i];
+    if ((p.ssq_tiles & 7) == 0) {
+        for (int i = 0; i < p.ssq_tiles; i += 8) {
+            float v[8];
+            ld256(sp + i, v);
+            s += ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
+        }
+    } else {
+        for (int i = 0; i < p.ssq_tiles; ++i) s += sp[i];
+    }
     return 1.0f / sqrtf(s / (float)p.K + p.eps);
 }
 
@@ -206,17 +223,17 @@ __device__ __forceinline__ bool epi_qkv(const GemmP& p, uint32_t taddr, int t, i
     const float rinv = row_rinv(p, t, row, row_ok);
     const bool slot_ok = row_ok && kvoff >= 0 && kvoff + (int64_t)(2 * p.nkv - 1) * p.ps * dh + dh <= p.slab_elems;
     if (row_ok && !slot_ok) report(p.status, PT_ERR_DEVICE_BOUNDS, LOC_ROPE_PAGE);
-    const float4* cs4 = (const float4*)(p.cs + (size_t)pos * halfdh);
-    const float4* sn4 = (const float4*)(p.sn + (size_t)pos * halfdh);
-    auto fetch = [&](int uu, float4* tab) {               // tab[0..3] = cos, tab[4..7] = sin of columns j0..j0+15
+    const float* csr = p.cs + (size_t)pos * halfdh;
+    const float* snr = p.sn + (size_t)pos * halfdh;
+    auto fetch = [&](int uu, float* tab) {                // tab[0..15] = cos, tab[16..31] = sin of columns j0..j0+15
         const int u = half * UNITS + uu;
         const int hs = n0 / dh + u / upd;
         if (hs >= p.nq + p.nkv || !row_ok) return;         // v heads, columns past N, rows past M: no rotation
-        const int j4 = (u % upd) * 4;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) { tab[i] = cs4[j4 + i]; tab[4 + i] = sn4[j4 + i]; }
+        const int j0 = (u % upd) * 16;
+        ld256(csr + j0, tab); ld256(csr + j0 + 8, tab + 8);
+        ld256(snr + j0, tab + 16); ld256(snr + j0 + 8, tab + 24);
     };
-    float4 tab[8], nxt[8];
+    float tab[32], nxt[32];
     fetch(0, tab);
     if (!wait()) return false;
 #pragma unroll 1
@@ -245,17 +262,11 @@ __device__ __forceinline__ bool epi_qkv(const GemmP& p, uint32_t taddr, int t, i
         tc_wait_ld();
         if (st_ok) {
             if (!is_v) {
-                float c[16], s[16];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    c[4 * i] = tab[i].x; c[4 * i + 1] = tab[i].y; c[4 * i + 2] = tab[i].z; c[4 * i + 3] = tab[i].w;
-                    s[4 * i] = tab[4 + i].x; s[4 * i + 1] = tab[4 + i].y; s[4 * i + 2] = tab[4 + i].z; s[4 * i + 3] = tab[4 + i].w;
-                }
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
                     const float l = lo[i] * rinv, h = hi[i] * rinv;
-                    lo[i] = l * c[i] - h * s[i];
-                    hi[i] = h * c[i] + l * s[i];
+                    lo[i] = l * tab[i] - h * tab[16 + i];
+                    hi[i] = h * tab[i] + l * tab[16 + i];
                 }
                 store16_bf16(dst + sub * 16, lo);
                 store16_bf16(dst + halfdh + sub * 16, hi);
@@ -267,7 +278,7 @@ __device__ __forceinline__ bool epi_qkv(const GemmP& p, uint32_t taddr, int t, i
             }
         }
 #pragma unroll
-        for (int i = 0; i < 8; ++i) tab[i] = nxt[i];       // last: the fetch stays in flight until here
+        for (int i = 0; i < 32; ++i) tab[i] = nxt[i];      // last: the fetch stays in flight until here
     }
     return true;
 }
@@ -278,19 +289,26 @@ template <int BN, class Wait>
 __device__ __forceinline__ bool epi_resid(const GemmP& p, uint32_t taddr, int t, int row, bool row_ok, int n0, int half, Wait wait) {
     constexpr int UNITS = BN / 64;                        // 32-column units per warp
     const float* hrow = p.h_in + (size_t)(p.n_sum > 1 ? 0 : t) * p.h_in_tstride + (size_t)row * p.N;
-    auto fetch = [&](int u, float4* h) {
+    auto fetch = [&](int u, float* h) {                   // h[0..31]: residual (summed over tracks at a sync)
         const int col = n0 + (half * UNITS + u) * 32;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) h[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int i = 0; i < 32; ++i) h[i] = 0.f;
         if (!row_ok) return;
-        for (int tt = 0; tt < p.n_sum; ++tt) {
-            const float4* hp = (const float4*)(hrow + (size_t)tt * p.h_in_tstride + col);
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
-                if (col + 4 * i < p.N) { const float4 x = hp[i]; h[i].x += x.x; h[i].y += x.y; h[i].z += x.z; h[i].w += x.w; }
+        for (int i = 0; i < 4; ++i) if (col + 8 * i < p.N) ld256(hrow + col + 8 * i, h + 8 * i);
+        for (int tt = 1; tt < p.n_sum; ++tt) {
+            float x[32];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                if (col + 8 * i < p.N) {
+                    ld256(hrow + (size_t)tt * p.h_in_tstride + col + 8 * i, x + 8 * i);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) h[8 * i + k] += x[8 * i + k];
+                }
+            }
         }
     };
-    float4 hres[8], hnxt[8];
+    float hres[32], hnxt[32];
     fetch(0, hres);
     if (!wait()) return false;
     float ssq = 0.f;
@@ -306,16 +324,14 @@ __device__ __forceinline__ bool epi_resid(const GemmP& p, uint32_t taddr, int t,
         tc_wait_ld();
         if (row_ok) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                v[4 * i] = (v[4 * i] + hres[i].x) * p.scale; v[4 * i + 1] = (v[4 * i + 1] + hres[i].y) * p.scale;
-                v[4 * i + 2] = (v[4 * i + 2] + hres[i].z) * p.scale; v[4 * i + 3] = (v[4 * i + 3] + hres[i].w) * p.scale;
-            }
-            float4* ho = (float4*)(p.h_out + (size_t)t * p.h_out_tstride + (size_t)row * p.N + col);
+            for (int i = 0; i < 32; ++i) v[i] = (v[i] + hres[i]) * p.scale;
+            float* ho = p.h_out + (size_t)t * p.h_out_tstride + (size_t)row * p.N + col;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                if (col + 4 * i < p.N) {
-                    ho[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-                    ssq += v[4 * i] * v[4 * i] + v[4 * i + 1] * v[4 * i + 1] + v[4 * i + 2] * v[4 * i + 2] + v[4 * i + 3] * v[4 * i + 3];
+            for (int i = 0; i < 4; ++i) {
+                if (col + 8 * i < p.N) {
+                    st256(ho + 8 * i, v + 8 * i);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) ssq += v[8 * i + k] * v[8 * i + k];
                 }
             }
             if (p.hb_out) {
@@ -345,7 +361,7 @@ __device__ __forceinline__ bool epi_resid(const GemmP& p, uint32_t taddr, int t,
             ssq = 0.f;
         }
 #pragma unroll
-        for (int i = 0; i < 8; ++i) hres[i] = hnxt[i];      // last: the fetch stays in flight until here
+        for (int i = 0; i < 32; ++i) hres[i] = hnxt[i];     // last: the fetch stays in flight until here
     }
     return true;
 }
