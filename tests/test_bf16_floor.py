@@ -17,29 +17,34 @@ from paper_2602_07306_b200 import inputs as I
 from tests import helpers as Hp
 
 
-def _layer(h, w, pos, nq, dh, rnd):
+def _layer(h, w, pos, nq, nkv, dh, rnd):
     R = (lambda a: I.round_to_bf16(np.asarray(a, np.float32)).astype(np.float64)) if rnd else (lambda a: a)
     S = h.shape[0]
     rinv = 1.0 / np.sqrt(np.mean(h * h, -1, keepdims=True) + 1e-6)
     a = R(h * w["g1"]) * rinv
     q = R(O.rope((a @ w["wq"].T).reshape(S, nq, dh), pos, 1e4))
-    k = R(O.rope((a @ w["wk"].T).reshape(S, nq, dh), pos, 1e4))
-    v = R((a @ w["wv"].T).reshape(S, nq, dh))
+    k = R(O.rope((a @ w["wk"].T).reshape(S, nkv, dh), pos, 1e4))
+    v = R((a @ w["wv"].T).reshape(S, nkv, dh))
     o = np.empty_like(q)
     for i in range(nq):
-        s = q[:, i] @ k[:, i].T / np.sqrt(dh)
+        j = i // (nq // nkv)
+        s = q[:, i] @ k[:, j].T / np.sqrt(dh)
         s = np.where(pos[None, :] <= pos[:, None], s, -np.inf)
         p = np.exp(s - s.max(-1, keepdims=True))
-        o[:, i] = (R(p) @ v[:, i]) / p.sum(-1, keepdims=True)
+        o[:, i] = (R(p) @ v[:, j]) / p.sum(-1, keepdims=True)
     h = h + R(o.reshape(S, -1)) @ w["wo"].T
     rinv = 1.0 / np.sqrt(np.mean(h * h, -1, keepdims=True) + 1e-6)
     c = R(h * w["g2"]) * rinv
     return h + R(O.silu(c @ w["wg"].T) * (c @ w["wu"].T)) @ w["wd"].T
 
 
-def test_rounding_only_the_tensor_core_operands_already_exceeds_2e_3_at_hidden_1024():
-    S, T, D = 12, 8, 8
-    wl = I.Workload("block", T=T, L=D, D=D, hidden=1024, heads=8, kv_heads=8, ffn=2816, dtype="bf16",
+import pytest
+
+
+@pytest.mark.parametrize("T,D,H,nq,nkv,F,tol", [(8, 8, 1024, 8, 8, 2816, Hp.DEEP_MEAN_TOL), (4, 2, 2048, 16, 4, 5632, Hp.WIDE_MEAN_TOL)])
+def test_rounding_only_the_tensor_core_operands_already_exceeds_2e_3_on_the_wide_models(T, D, H, nq, nkv, F, tol):
+    S = 12
+    wl = I.Workload("block", T=T, L=D, D=D, hidden=H, heads=nq, kv_heads=nkv, ffn=F, dtype="bf16",
                     mode="prefill", batch=1, seq=S)
     ws = I.WeightSource(wl)
     x = I.prefill_inputs(wl).astype(np.float64)
@@ -49,9 +54,10 @@ def test_rounding_only_the_tensor_core_operands_already_exceeds_2e_3_at_hidden_1
     for l in range(D):
         for t in range(T):
             w = {k: np.asarray(v, np.float64) for k, v in ws.get(t, l).items()}
-            exact[t] = _layer(exact[t], w, pos, wl.heads, wl.head_dim, False)
-            rounded[t] = _layer(rounded[t], w, pos, wl.heads, wl.head_dim, True)
+            exact[t] = _layer(exact[t], w, pos, nq, nkv, wl.head_dim, False)
+            rounded[t] = _layer(rounded[t], w, pos, nq, nkv, wl.head_dim, True)
     e, r = sum(exact), sum(rounded)                           # the track-sync that closes the block
     mx, mean = Hp.rel_errs(r, e)
-    assert 2.0e-3 < mean < Hp.DEEP_MEAN_TOL, mean
+    print(f"hidden {H}: floor mean-rel {mean:.3e}, max-rel {mx:.3e}")
+    assert 2.0e-3 < mean < tol, mean
     assert mx < 2e-2

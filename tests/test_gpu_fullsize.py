@@ -136,8 +136,8 @@ def _decode_equals_prefill_row(model, wl, lens, seed, sub_tokens=16384):
 def test_decode_full_size_equals_prefill_row_cfg2(mid_model):
     wl3, ws, model = mid_model
     wl = I.WORKLOADS["cfg2"]
-    if _free_gib() < 150:
-        pytest.skip("needs about 150 GiB of free device memory")
+    if _free_gib() < 133:
+        pytest.skip(f"needs about 133 GiB of free device memory, {_free_gib():.0f} GiB are free")
     _decode_equals_prefill_row(model, wl, I.kv_lengths(wl), seed=7)
 
 
@@ -170,4 +170,4 @@ def test_wide_gqa_architecture_at_reduced_depth_matches_oracle():
     base = I.WORKLOADS["cfg4"]
     wl = I.Workload("cfg4-shallow", T=base.T, L=2, D=2, hidden=base.hidden, heads=base.heads, kv_heads=base.kv_heads,
                     ffn=base.ffn, dtype="bf16", mode="decode", batch=3, seq=0, ragged=base.ragged)
-    run_case(wl, B=3, S=150, chunks=[130, 20], decode_steps=2, shuffle=True)
+    run_case(wl, B=3, S=150, chunks=[130, 20], decode_steps=2, shuffle=True, mean_tol=Hp.WIDE_MEAN_TOL)
