@@ -30,6 +30,12 @@ sys.path.insert(0, ROOT)
 
 from paper_2602_07306_b200 import inputs as I  # noqa: E402
 
+# DRAM traffic of k_decode_attn_tma<128> from its ncu capture (profiles/decode_attn_tma_T8_B8_kv2049.md:
+# 8 sequences instead of 64, same kernel): dram read + write bytes per launch over the algorithmic K/V
+# bytes of that launch.  Traffic is proportional to the keys read, so a bench launch is scaled by its own
+# algorithmic bytes.  Set to None when the kernel changes until the counters are taken again.
+DECODE_ATTN_TRAFFIC_RATIO = (541.2e6 + 4.0e6) / 537.1e6
+
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -204,8 +210,10 @@ def run_decode(wl, dev, steps, warmup, barrier, rank):
     attn_avg_ms = attn_ms / max(attn_n, 1)
     achieved = alg["attn_bytes_per_layer"] / (attn_avg_ms * 1e-3) / 1e9
     roof = {"bound": "hbm", "kernel": "k_decode_attn", "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s",
-            "frac": achieved / pk["hbm_gbs"], "traffic": None, "peak_kind": f"of {pk_kind}",
-            "avg_launch_ms": attn_avg_ms, "launches": attn_n,
+            "frac": achieved / pk["hbm_gbs"],
+            "traffic": (alg["attn_bytes_per_layer"] * DECODE_ATTN_TRAFFIC_RATIO
+                        if DECODE_ATTN_TRAFFIC_RATIO and wl.head_dim == 128 and wl.page_size == 16 else None),
+            "peak_kind": f"of {pk_kind}", "avg_launch_ms": attn_avg_ms, "launches": attn_n,
             "step_hbm_gbs": alg["bytes"] / (ms * 1e-3) / 1e9, "step_frac": alg["bytes"] / (ms * 1e-3) / 1e9 / pk["hbm_gbs"],
             "step_frac_of_nominal_8tbs": alg["bytes"] / (ms * 1e-3) / 8e12}
     # end to end from pinned host buffers
