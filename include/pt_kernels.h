@@ -17,7 +17,7 @@ extern "C" {
  *   c[t][m][n] = sum_k a[t][m][k] * w[t][n][k]      t < T, m < M, n < N
  *   a  device bf16 [T][M][K] row-major        w  device bf16 [T][N][K] row-major
  *   c  device fp32 [T][M][N]                  status  device int32[16], zeroed by the caller
- * K must be a multiple of 8 and >= 64, N a multiple of 16; bn (N-tile width) is 128 or 256, 0 lets
+ * K must be a multiple of 8 and >= 64, N a multiple of 16; bn (N-tile width) is 64, 128 or 256, 0 lets
  * the library choose.  With fold_tracks != 0 the K loop runs over (track, k) and a single
  * c[0][m][n] = sum_t sum_k ... is produced: the contraction of the track-sync (Algorithm 1,
  * h = all-reduce(h_1..h_n)) fused into the last GEMM of a track block. */

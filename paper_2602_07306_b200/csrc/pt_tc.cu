@@ -39,7 +39,45 @@ __global__ void k_tc_prep(const __nv_bfloat16* __restrict__ x, int64_t x_stride,
     }
 }
 
-struct WMaps { CUtensorMap m[4][2]; };   // [qkv, o, gu, d][bn 128, bn 256]
+// Track-sync of a small batch (decode): h = scale * sum_t h_t in track order, the synced stream, every
+// track's gain-scaled bf16 operand for the next layer and the partial sums of squares.  One warp per row.
+// (With few rows the K-concatenated sync GEMM would run on N/128 CTAs only; the per-track down GEMM fills
+// the machine and this kernel finishes the reduction.)
+__global__ void k_track_sync(const float* __restrict__ hT, size_t tstride, int T, float scale,
+                             float* __restrict__ h_out, __nv_bfloat16* __restrict__ hb, const float* __restrict__ gain,
+                             float* __restrict__ ssq, int M, int H, int tiles) {
+    int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (warp >= M) return;
+    size_t ro = (size_t)warp * H;
+    for (int g = 0; g * 128 < H; ++g) {
+        int c = g * 128 + lane * 4;
+        float s = 0.f;
+        if (c < H) {
+            float4 a = *reinterpret_cast<const float4*>(hT + ro + c);
+            for (int t = 1; t < T; ++t) {
+                float4 b = *reinterpret_cast<const float4*>(hT + (size_t)t * tstride + ro + c);
+                a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+            }
+            a.x *= scale; a.y *= scale; a.z *= scale; a.w *= scale;
+            *reinterpret_cast<float4*>(h_out + ro + c) = a;
+            s = a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
+            if (hb) {
+                for (int t = 0; t < T; ++t) {
+                    float4 gn = *reinterpret_cast<const float4*>(gain + (size_t)t * H + c);
+                    __nv_bfloat162 o0 = __floats2bfloat162_rn(a.x * gn.x, a.y * gn.y), o1 = __floats2bfloat162_rn(a.z * gn.z, a.w * gn.w);
+                    uint2 ov;
+                    ov.x = *reinterpret_cast<uint32_t*>(&o0); ov.y = *reinterpret_cast<uint32_t*>(&o1);
+                    *reinterpret_cast<uint2*>(hb + (size_t)t * M * H + ro + c) = ov;
+                }
+            }
+        }
+        for (int o = 8; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        int tile = g * 2 + (lane >> 4);
+        if (ssq && (lane & 15) == 0 && tile < tiles) ssq[(size_t)warp * tiles + tile] = s;
+    }
+}
+
+struct WMaps { CUtensorMap m[4][3]; };   // [qkv, o, gu, d][bn 64, 128, 256]
 
 }  // namespace
 
@@ -54,8 +92,8 @@ pt_status tc_build_weight_maps(pt_model* m) {
     const __nv_bfloat16* wgu = (const __nv_bfloat16*)(m->wbuf + m->off_wgu);
     const __nv_bfloat16* wd = (const __nv_bfloat16*)(m->wbuf + m->off_wd);
     for (int l = 0; l < c.L; ++l)
-        for (int b = 0; b < 2; ++b) {
-            int bn = b ? 256 : 128;
+        for (int b = 0; b < 3; ++b) {
+            int bn = 64 << b;
             pt_status s;
             if ((s = make_map_bf16(&v[l].m[0][b], wqkv + (size_t)l * m->wqkv_layer(), c.hidden, m->Nqkv, c.T, bn)) != PT_OK) return s;
             if ((s = make_map_bf16(&v[l].m[1][b], wo + (size_t)l * m->wo_layer(), m->QD, c.hidden, c.T, bn)) != PT_OK) return s;
@@ -112,9 +150,9 @@ pt_status tc_forward(Call& k) {
             p.q_out = q; p.pool_l = pool_l; p.pool_tstride = pool_tstride; p.slab_elems = c->slab_elems;
             p.row_kvoff = w.meta.row_kvoff; p.row_pos = w.meta.row_pos; p.cs = m->rope_cos(); p.sn = m->rope_sin();
             p.nq = g.heads; p.nkv = g.kv_heads; p.dh = m->dh; p.ps = c->ps;
-            int bn = gemm_bn(p.N, M, T);
+            int bn = gemm_bn(p.N, M, T, EPI_QKV);
             ProfScope ps(m, st, 1);
-            if ((s = launch_gemm(EPI_QKV, bn, ta_h, wm[l].m[0][bn == 256], p, st)) != PT_OK) return s;
+            if ((s = launch_gemm(EPI_QKV, bn, ta_h, wm[l].m[0][bn_index(bn)], p, st)) != PT_OK) return s;
         }
         {
             ProfScope ps(m, st, 0);
@@ -128,9 +166,9 @@ pt_status tc_forward(Call& k) {
             p.h_in = hin; p.h_in_tstride = hin_stride; p.h_out = w.hT; p.h_out_tstride = MH;
             p.hb_out = hb; p.gain = m->gain(1, l);
             p.ssq_out = w.ssq; p.ssq_out_tstride = (size_t)M * tiles; p.ssq_out_tiles = tiles;
-            int bn = gemm_bn(p.N, M, T);
+            int bn = gemm_bn(p.N, M, T, EPI_RESID);
             ProfScope ps(m, st, 2);
-            if ((s = launch_gemm(EPI_RESID, bn, ta_o, wm[l].m[1][bn == 256], p, st)) != PT_OK) return s;
+            if ((s = launch_gemm(EPI_RESID, bn, ta_o, wm[l].m[1][bn_index(bn)], p, st)) != PT_OK) return s;
             ssq_tstride = (size_t)M * tiles;
         }
         tap_copy(k, l, 0, w.hT, MH);
@@ -139,9 +177,9 @@ pt_status tc_forward(Call& k) {
             p.N = 2 * F; p.K = H;
             p.ssq_in = w.ssq; p.ssq_in_tstride = ssq_tstride; p.ssq_tiles = tiles;
             p.z_out = z;
-            int bn = gemm_bn(p.N, M, T);
+            int bn = gemm_bn(p.N, M, T, EPI_SWIGLU);
             ProfScope ps(m, st, 3);
-            if ((s = launch_gemm(EPI_SWIGLU, bn, ta_h, wm[l].m[2][bn == 256], p, st)) != PT_OK) return s;
+            if ((s = launch_gemm(EPI_SWIGLU, bn, ta_h, wm[l].m[2][bn_index(bn)], p, st)) != PT_OK) return s;
         }
         {   // down projection + residual (+ track-sync when the layer closes a track block)
             const bool sync = (l + 1) % g.D == 0, last = l + 1 == g.L;
@@ -149,22 +187,31 @@ pt_status tc_forward(Call& k) {
             p.N = H; p.K = F;
             p.h_in = w.hT; p.h_in_tstride = MH;
             if (!last) { p.hb_out = hb; p.gain = m->gain(0, l + 1); p.ssq_out = w.ssq; p.ssq_out_tiles = tiles; }
-            if (sync) {
+            // a decode step (few rows): per-track down GEMM on the whole machine, then a small reduction kernel;
+            // many rows (prefill): one GEMM whose K loop runs over (track, k) and whose epilogue is the sync
+            const bool split_sync = sync && k.decode && M <= 256;
+            if (sync && !split_sync) {
                 p.T = 1; p.kt = T; p.n_sum = T; p.n_out = T;
                 p.scale = g.sync_op ? 1.0f / T : 1.0f;
                 p.h_out = last ? k.out : w.hS; p.h_out_tstride = 0;
                 p.ssq_out_tstride = 0;
-                ssq_tstride = 0;
-                hin = p.h_out; hin_stride = 0;
             } else {
                 p.h_out = w.hT; p.h_out_tstride = MH;
                 p.ssq_out_tstride = (size_t)M * tiles;
-                ssq_tstride = (size_t)M * tiles;
-                hin = w.hT; hin_stride = MH;
+                if (split_sync) { p.hb_out = nullptr; p.ssq_out = nullptr; }
             }
-            int bn = gemm_bn(p.N, M, p.T);
+            int bn = gemm_bn(p.N, M, p.T, EPI_RESID);
             ProfScope ps(m, st, sync ? 5 : 4);
-            if ((s = launch_gemm(EPI_RESID, bn, ta_z, wm[l].m[3][bn == 256], p, st)) != PT_OK) return s;
+            if ((s = launch_gemm(EPI_RESID, bn, ta_z, wm[l].m[3][bn_index(bn)], p, st)) != PT_OK) return s;
+            if (split_sync) {
+                float* ho = last ? k.out : w.hS;
+                k_track_sync<<<(M * 32 + 255) / 256, 256, 0, st>>>(w.hT, MH, T, g.sync_op ? 1.0f / T : 1.0f, ho,
+                                                                   last ? nullptr : hb, last ? nullptr : m->gain(0, l + 1),
+                                                                   last ? nullptr : w.ssq, M, H, tiles);
+                g_launches.fetch_add(1, std::memory_order_relaxed);
+            }
+            if (sync) { ssq_tstride = 0; hin = last ? k.out : w.hS; hin_stride = 0; }
+            else { ssq_tstride = (size_t)M * tiles; hin = w.hT; hin_stride = MH; }
         }
         tap_copy(k, l, 1, hin, hin_stride);
     }
@@ -182,8 +229,8 @@ extern "C" pt_status pt_kernel_gemm_bf16(const void* a, const void* w, void* c, 
     using namespace pt;
     if (!a || !w || !c || !status) { set_error("null argument"); return PT_ERR_INVALID_ARG; }
     if (T < 1 || M < 1 || N < 16 || N % 16 || K < 64 || K % 8) { set_error("unsupported GEMM shape"); return PT_ERR_INVALID_ARG; }
-    if (bn == 0) bn = gemm_bn(N, M, fold_tracks ? 1 : T);
-    if (bn != 128 && bn != 256) { set_error("bn must be 0, 128 or 256"); return PT_ERR_INVALID_ARG; }
+    if (bn == 0) bn = gemm_bn(N, M, fold_tracks ? 1 : T, EPI_PLAIN);
+    if (bn != 64 && bn != 128 && bn != 256) { set_error("bn must be 0, 64, 128 or 256"); return PT_ERR_INVALID_ARG; }
     CUtensorMap ta, tb;
     pt_status s;
     if ((s = make_map_bf16(&ta, a, K, M, T, 128)) != PT_OK) return s;

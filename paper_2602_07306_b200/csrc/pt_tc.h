@@ -59,7 +59,8 @@ pt_status launch_decode_attn_p(const AttnP& p, int T, int dh, int n_items, int m
 pt_status make_map_bf16(CUtensorMap* out, const void* base, int64_t k, int64_t rows, int64_t tracks, int box_rows);
 pt_status make_map_bf16_strided(CUtensorMap* out, const void* base, int64_t k, int64_t rows, int64_t tracks,
                                 int64_t track_stride_bytes, int box_rows);
-int gemm_bn(int N, int M, int T);
+int gemm_bn(int N, int M, int T, int epi);
+inline int bn_index(int bn) { return bn == 64 ? 0 : (bn == 128 ? 1 : 2); }
 pt_status launch_gemm(int epi, int bn, const CUtensorMap& ta, const CUtensorMap& tb, GemmP p, cudaStream_t st);
 
 // pt_simt.cu

@@ -103,7 +103,7 @@ __device__ __forceinline__ void report(int* status, int code, int loc) {
 }
 
 template <int BN> struct Cfg {
-    static constexpr int STAGES = BN == 256 ? 4 : 6;
+    static constexpr int STAGES = BN == 256 ? 4 : (BN == 128 ? 6 : 8);
     static constexpr int A_BYTES = BM * BK * 2;
     static constexpr int B_BYTES = BN * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
@@ -159,11 +159,11 @@ __device__ __forceinline__ float row_rinv(const GemmP& p, int t, int row, bool r
 
 template <int BN, class Wait>
 __device__ __forceinline__ bool epi_plain(const GemmP& p, uint32_t taddr, int t, int row, bool row_ok, int n0, int half, Wait wait) {
-    constexpr int UNITS = BN / 64;                        // 32-column units per warp
+    constexpr int UNITS = BN / 32;                        // 32-column units of the tile; 64-column groups alternate between the two warps
     if (!wait()) return false;
 #pragma unroll 1
-    for (int u = 0; u < UNITS; ++u) {
-        const int c = (half * UNITS + u) * 32;
+    for (int u = 2 * half; u < UNITS; u += (u & 1) ? 3 : 1) {
+        const int c = u * 32;
         if (n0 + c >= p.N) break;                          // uniform across the warp
         float v[32];
         tc_ld16(taddr + c, v);
@@ -183,13 +183,13 @@ __device__ __forceinline__ bool epi_plain(const GemmP& p, uint32_t taddr, int t,
 // unit here is 64 accumulator columns = 32 outputs z = silu(gate / rms) * (up / rms).
 template <int BN, class Wait>
 __device__ __forceinline__ bool epi_swiglu(const GemmP& p, uint32_t taddr, int t, int row, bool row_ok, int n0, int half, Wait wait) {
-    constexpr int UNITS = BN / 128;                       // 64-column units per warp
+    constexpr int UNITS = BN / 64;                        // 64-column units of the tile, alternating between the two warps
     const float rinv = row_rinv(p, t, row, row_ok);
     const int F = p.N >> 1;
     if (!wait()) return false;
 #pragma unroll 1
-    for (int u = 0; u < UNITS; ++u) {
-        const int c = (half * UNITS + u) * 64;
+    for (int u = half; u < UNITS; u += 2) {
+        const int c = u * 64;
         if (n0 + c >= p.N) break;
         float gu[64];
 #pragma unroll
@@ -215,7 +215,7 @@ __device__ __forceinline__ bool epi_swiglu(const GemmP& p, uint32_t taddr, int t
 // values of the row's position are fetched one unit ahead.
 template <int BN, class Wait>
 __device__ __forceinline__ bool epi_qkv(const GemmP& p, uint32_t taddr, int t, int row, bool row_ok, int n0, int half, Wait wait) {
-    constexpr int UNITS = BN / 64;                        // units per warp
+    constexpr int UNITS = BN / 32;                        // units of the tile, alternating between the two warps
     const int dh = p.dh, halfdh = dh >> 1, upd = dh >> 5;  // units per head
     const int heads_total = p.nq + 2 * p.nkv;
     int pos = 0; int64_t kvoff = 0;
@@ -225,8 +225,7 @@ __device__ __forceinline__ bool epi_qkv(const GemmP& p, uint32_t taddr, int t, i
     if (row_ok && !slot_ok) report(p.status, PT_ERR_DEVICE_BOUNDS, LOC_ROPE_PAGE);
     const float* csr = p.cs + (size_t)pos * halfdh;
     const float* snr = p.sn + (size_t)pos * halfdh;
-    auto fetch = [&](int uu, float* tab) {                // tab[0..15] = cos, tab[16..31] = sin of columns j0..j0+15
-        const int u = half * UNITS + uu;
+    auto fetch = [&](int u, float* tab) {                 // tab[0..15] = cos, tab[16..31] = sin of columns j0..j0+15
         const int hs = n0 / dh + u / upd;
         if (hs >= p.nq + p.nkv || !row_ok) return;         // v heads, columns past N, rows past M: no rotation
         const int j0 = (u % upd) * 16;
@@ -234,11 +233,10 @@ __device__ __forceinline__ bool epi_qkv(const GemmP& p, uint32_t taddr, int t, i
         ld256(snr + j0, tab + 16); ld256(snr + j0 + 8, tab + 24);
     };
     float tab[32], nxt[32];
-    fetch(0, tab);
+    fetch(half, tab);
     if (!wait()) return false;
 #pragma unroll 1
-    for (int uu = 0; uu < UNITS; ++uu) {
-        const int u = half * UNITS + uu;
+    for (int u = half; u < UNITS; u += 2) {
         const int hc = u / upd, sub = u % upd;
         const int hs = n0 / dh + hc;                       // head slot: q heads, then k heads, then v heads
         if (hs >= heads_total) break;                      // uniform across the warp
@@ -248,7 +246,7 @@ __device__ __forceinline__ bool epi_qkv(const GemmP& p, uint32_t taddr, int t, i
         const int c_hi = is_v ? c_lo + 16 : c_lo + halfdh;
         tc_ld16(taddr + c_lo, lo);
         tc_ld16(taddr + c_hi, hi);
-        if (uu + 1 < UNITS) fetch(uu + 1, nxt);
+        if (u + 2 < UNITS) fetch(u + 2, nxt);
         __nv_bfloat16* dst;
         bool st_ok;
         if (hs < p.nq) {
@@ -287,10 +285,10 @@ __device__ __forceinline__ bool epi_qkv(const GemmP& p, uint32_t taddr, int t, i
 // The 32 residual values of a unit (128 bytes of the thread's row) are fetched one unit ahead.
 template <int BN, class Wait>
 __device__ __forceinline__ bool epi_resid(const GemmP& p, uint32_t taddr, int t, int row, bool row_ok, int n0, int half, Wait wait) {
-    constexpr int UNITS = BN / 64;                        // 32-column units per warp
+    constexpr int UNITS = BN / 32;                        // 32-column units of the tile; 64-column groups alternate between the two warps
     const float* hrow = p.h_in + (size_t)(p.n_sum > 1 ? 0 : t) * p.h_in_tstride + (size_t)row * p.N;
     auto fetch = [&](int u, float* h) {                   // h[0..31]: residual (summed over tracks at a sync)
-        const int col = n0 + (half * UNITS + u) * 32;
+        const int col = n0 + u * 32;
 #pragma unroll
         for (int i = 0; i < 32; ++i) h[i] = 0.f;
         if (!row_ok) return;
@@ -309,18 +307,19 @@ __device__ __forceinline__ bool epi_resid(const GemmP& p, uint32_t taddr, int t,
         }
     };
     float hres[32], hnxt[32];
-    fetch(0, hres);
+    fetch(2 * half, hres);
     if (!wait()) return false;
     float ssq = 0.f;
 #pragma unroll 1
-    for (int u = 0; u < UNITS; ++u) {
-        const int c = (half * UNITS + u) * 32;
+    for (int u = 2 * half; u < UNITS; u += (u & 1) ? 3 : 1) {      // units 0,1, 4,5, ... or 2,3, 6,7, ...
+        const int c = u * 32;
         const int col = n0 + c;
         if (col >= p.N) break;                             // uniform across the warp
         float v[32];
         tc_ld16(taddr + c, v);
         tc_ld16(taddr + c + 16, v + 16);
-        if (u + 1 < UNITS) fetch(u + 1, hnxt);
+        const int un = u + ((u & 1) ? 3 : 1);
+        if (un < UNITS) fetch(un, hnxt);
         tc_wait_ld();
         if (row_ok) {
 #pragma unroll
@@ -546,9 +545,24 @@ pt_status make_map_bf16_strided(CUtensorMap* out, const void* base, int64_t k, i
     return PT_OK;
 }
 
-int gemm_bn(int N, int M, int T) {
-    // wide tiles when there are enough of them to fill the machine
-    if (N % 256 == 0 && (int64_t)((M + BM - 1) / BM) * (N / 256) * T >= 148) return 256;
+int gemm_bn(int N, int M, int T, int epi) {
+    // Tile width by wave efficiency: a launch runs ceil(tiles / SMs) rounds, and a round costs about
+    // the tile's width (bytes streamed per tile when M is small, MMA cycles when it is large).  Take
+    // the widest tile (fewest re-reads of A) within 3 % of the best fill.  The QKV epilogue needs
+    // whole heads (rotary partners) in a tile, so it never goes below 128.
+    const int widths[3] = {256, 128, 64};
+    const int tiles_m = (M + BM - 1) / BM;
+    double eff[3], best = 0.0;
+    for (int i = 0; i < 3; ++i) {
+        const int bn = widths[i];
+        eff[i] = 0.0;
+        if (bn == 64 && epi == EPI_QKV) continue;
+        const int64_t tiles = (int64_t)tiles_m * ((N + bn - 1) / bn) * T;
+        const int64_t rounds = (tiles + 147) / 148;
+        eff[i] = (double)N * T * tiles_m / ((double)rounds * 148 * bn);     // useful columns over columns paid for
+        best = std::max(best, eff[i]);
+    }
+    for (int i = 0; i < 3; ++i) if (eff[i] >= best - 0.03) return widths[i];
     return 128;
 }
 
@@ -563,6 +577,7 @@ pt_status launch_gemm(int epi, int bn, const CUtensorMap& ta, const CUtensorMap&
     int box_a = std::min(BM, p.M), box_b = std::min(bn, p.kt > 1 ? p.N : p.N);
     p.tx_bytes = (uint32_t)(box_a + box_b) * BK * 2;
 #define CASE(BN_, E_) if (bn == BN_ && epi == E_) return launch_t<BN_, E_>(ta, tb, p, st, sms)
+    CASE(64, EPI_PLAIN); CASE(64, EPI_SWIGLU); CASE(64, EPI_RESID);
     CASE(128, EPI_PLAIN); CASE(128, EPI_QKV); CASE(128, EPI_SWIGLU); CASE(128, EPI_RESID);
     CASE(256, EPI_PLAIN); CASE(256, EPI_QKV); CASE(256, EPI_SWIGLU); CASE(256, EPI_RESID);
 #undef CASE

@@ -23,6 +23,8 @@ def _operands(T, M, N, K, seed):
     (2, 300, 128, 1376, 128, False),      # K tail (1376 = 21.5 x 64)
     (4, 130, 512, 1376, 256, True),       # tracks folded into K (track-sync contraction)
     (2, 1024, 1024, 1024, 0, False),      # enough tiles for several per CTA, library-chosen width
+    (3, 64, 1024, 320, 64, False),        # narrow tiles (decode shapes), few rows
+    (2, 200, 160, 192, 64, True),         # narrow tiles, N tail, tracks folded into K
 ])
 def test_gemm_bf16_matches_definition(T, M, N, K, bn, fold):
     import torch
