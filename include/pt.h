@@ -195,7 +195,10 @@ pt_status pt_device_status(pt_model* m, void* stream, int32_t* code, int32_t* de
  * with CUDA events on the call's stream.  pt_profile_read waits for those events, ADDS device
  * milliseconds and launch counts per category into ms[] and launches[] (host, PT_PROF_CATEGORIES
  * entries each) and forgets the events.  Categories: 0 attention, 1 QKV GEMM, 2 output-projection
- * GEMM, 3 gate/up GEMM, 4 down GEMM, 5 down GEMM with track-sync, 6 everything else. */
+ * GEMM, 3 gate/up GEMM, 4 down GEMM, 5 down GEMM with track-sync, 6 everything else.
+ * on = 0: off; on = 1: every category; any other value: bit (c + 1) selects category c (e.g.
+ * on = 2 times the attention launches only, which keeps the cost of the events themselves -
+ * about 2 us per bracketed launch - out of a measurement of the whole step). */
 #define PT_PROF_CATEGORIES 7
 pt_status pt_profile_enable(pt_model* m, int32_t on);
 pt_status pt_profile_read(pt_model* m, float* ms, int64_t* launches);

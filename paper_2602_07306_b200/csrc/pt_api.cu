@@ -153,7 +153,7 @@ void pt_model_destroy(pt_model* m) {
 
 pt_status pt_profile_enable(pt_model* m, int32_t on) {
     if (!m) PT_FAIL(PT_ERR_INVALID_ARG, "null argument");
-    m->prof_on = on != 0;
+    m->prof_mask = on == 1 ? 0xffffffffu : (on < 0 ? 0u : ((uint32_t)on >> 1));
     if (!on) m->prof_used = 0;
     return PT_OK;
 }

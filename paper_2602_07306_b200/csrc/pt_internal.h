@@ -53,7 +53,7 @@ struct pt_model {
     std::vector<char> meta_host;          // staging for the per-call metadata upload
     // optional per-kernel timing (pt_profile_enable)
     struct ProfEv { cudaEvent_t a, b; int cat; };
-    bool prof_on = false;
+    uint32_t prof_mask = 0;               // bit c set: launches of category c are bracketed with events
     std::vector<ProfEv> prof_ev;
     size_t prof_used = 0;
 
@@ -127,7 +127,7 @@ struct Call {
 struct ProfScope {
     pt_model* m; cudaStream_t st; int idx = -1;
     ProfScope(pt_model* m_, cudaStream_t st_, int cat) : m(m_), st(st_) {
-        if (!m->prof_on) return;
+        if (!((m->prof_mask >> cat) & 1u)) return;
         if (m->prof_used == m->prof_ev.size()) {
             pt_model::ProfEv e{};
             if (cudaEventCreate(&e.a) != cudaSuccess || cudaEventCreate(&e.b) != cudaSuccess) return;

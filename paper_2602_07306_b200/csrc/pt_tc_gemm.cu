@@ -546,24 +546,22 @@ pt_status make_map_bf16_strided(CUtensorMap* out, const void* base, int64_t k, i
 }
 
 int gemm_bn(int N, int M, int T, int epi) {
-    // Tile width by wave efficiency: a launch runs ceil(tiles / SMs) rounds, and a round costs about
-    // the tile's width (bytes streamed per tile when M is small, MMA cycles when it is large).  Take
-    // the widest tile (fewest re-reads of A) within 3 % of the best fill.  The QKV epilogue needs
-    // whole heads (rotary partners) in a tile, so it never goes below 128.
+    // Tile width by a round model: a launch runs ceil(tiles / SMs) rounds and a round costs about
+    // bn + min(M, 128) (bytes of B and A streamed per k-block when M is small, and near enough the MMA
+    // and A-reload cost when it is large).  Ties go to the wider tile.  The QKV epilogue needs whole
+    // heads (rotary partners) in a tile, so it never goes below 128.
     const int widths[3] = {256, 128, 64};
     const int tiles_m = (M + BM - 1) / BM;
-    double eff[3], best = 0.0;
+    int best_bn = 128;
+    int64_t best = -1;
     for (int i = 0; i < 3; ++i) {
         const int bn = widths[i];
-        eff[i] = 0.0;
         if (bn == 64 && epi == EPI_QKV) continue;
         const int64_t tiles = (int64_t)tiles_m * ((N + bn - 1) / bn) * T;
-        const int64_t rounds = (tiles + 147) / 148;
-        eff[i] = (double)N * T * tiles_m / ((double)rounds * 148 * bn);     // useful columns over columns paid for
-        best = std::max(best, eff[i]);
+        const int64_t cost = ((tiles + 147) / 148) * (bn + std::min(M, BM));
+        if (best < 0 || cost < best) { best = cost; best_bn = bn; }
     }
-    for (int i = 0; i < 3; ++i) if (eff[i] >= best - 0.03) return widths[i];
-    return 128;
+    return best_bn;
 }
 
 pt_status launch_gemm(int epi, int bn, const CUtensorMap& ta, const CUtensorMap& tb, GemmP p, cudaStream_t st) {

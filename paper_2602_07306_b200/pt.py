@@ -239,8 +239,13 @@ class Model:
 
     PROF_NAMES = ("attention", "gemm_qkv", "gemm_out", "gemm_gate_up", "gemm_down", "gemm_down_sync", "other")
 
-    def profile(self, on: bool) -> None:
-        check(lib().pt_profile_enable(self.h, int(on)))
+    def profile(self, on, only=None) -> None:
+        """on False / True: no launch / every launch bracketed with events; only=("attention", ...) brackets
+        the launches of those categories alone."""
+        code = int(bool(on))
+        if on and only:
+            code = sum(2 << self.PROF_NAMES.index(n) for n in only)
+        check(lib().pt_profile_enable(self.h, code))
 
     def profile_read(self) -> dict:
         """Device milliseconds and launches per kernel category since the last read."""
