@@ -45,9 +45,12 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
                  : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+// `relaxed` waits (the copy warp's, which run stages ahead of their consumers) back off between polls:
+// a spinning warp costs issue slots and power; the softmax and MMA hand-offs poll at full rate.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, bool relaxed = false) {
     for (uint32_t i = 0; i < kSpin; ++i) {
         if (mbar_try(bar, parity)) return true;
+        if (relaxed && i >= 2) __nanosleep(128);
         if ((i & 1023) == 1023 && *abort_flag) return false;
     }
     return false;
@@ -270,7 +273,7 @@ k_flash_prefill_tc(const __grid_constant__ CUtensorMap qmap, const __grid_consta
                 row_k = (page * 2 * p.nkv + kvh) * p.ps + key % p.ps;
             }
             const uint32_t bytes = (uint32_t)ng * 16u * DH * 2u;
-            if (!mbar_wait(&bars[B_KEMPTY + s], ph ^ 1u, abort_flag)) { if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_FLASH_KEMPTY); *abort_flag = 1; } break; }
+            if (!mbar_wait(&bars[B_KEMPTY + s], ph ^ 1u, abort_flag, true)) { if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_FLASH_KEMPTY); *abort_flag = 1; } break; }
             if (lane == 0) mbar_expect_tx(&bars[B_KFULL + s], bytes);
             __syncwarp();
             if (lane < ng) {
@@ -278,7 +281,7 @@ k_flash_prefill_tc(const __grid_constant__ CUtensorMap qmap, const __grid_consta
                 for (int h = 0; h < HALVES; ++h)
                     tma_load_3d(smem_u32(sk + s * TILE + h * kHalfBytes + lane * 2048), &kvmap, &bars[B_KFULL + s], h * 64, row_k, t);
             }
-            if (!mbar_wait(&bars[B_VEMPTY + s], ph ^ 1u, abort_flag)) { if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_FLASH_VEMPTY); *abort_flag = 1; } break; }
+            if (!mbar_wait(&bars[B_VEMPTY + s], ph ^ 1u, abort_flag, true)) { if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_FLASH_VEMPTY); *abort_flag = 1; } break; }
             const bool partial = key0 + 128 > key_end;             // rows past the last key must read as zero
             uint64_t* vbar = partial ? &bars[B_VRAW] : &bars[B_VFULL + s];
             if (lane == 0) mbar_expect_tx(vbar, bytes);

@@ -50,6 +50,7 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         if (mbar_try(bar, parity)) return true;
+        if (i >= 4) __nanosleep(64);                       // back off: a spinning warp costs issue slots and power
         if ((i & 1023) == 1023 && *abort_flag) return false;
     }
     return false;
