@@ -169,7 +169,7 @@ def run_decode(wl, dev, steps, warmup, barrier, rank):
     while i < B:
         n = int(lens[order[i]])
         j = i
-        while j < B and int(lens[order[j]]) == n and (j - i + 1) * n <= 16384:
+        while j < B and int(lens[order[j]]) == n and (j == i or (j - i + 1) * n <= 16384):
             j += 1
         ids = [int(s) for s in order[i:j]]
         x = torch.randn((wl.T, len(ids), n, wl.hidden), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
@@ -424,9 +424,16 @@ def main():
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--extra", default="cfg3", help="comma-separated workloads reported under 'extra' (N=1 only); '' for none")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--seq", type=int, default=0, help="override the workload's sequence / KV length")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch")
+    ap.add_argument("--depth", type=int, default=0, help="override the track-block depth D (must divide L)")
     a = ap.parse_args()
     a.warmup = max(a.warmup, 3) if a.impl == "ours" else a.warmup
     wl = I.WORKLOADS[a.workload]
+    import dataclasses
+    over = {k: v for k, v in (("seq", a.seq), ("batch", a.batch), ("D", a.depth)) if v}
+    if over:
+        wl = dataclasses.replace(wl, **over)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     metric = "decode tokens/s" if wl.mode == "decode" else "prefill tokens/s"

@@ -105,7 +105,7 @@ def _decode_equals_prefill_row(model, wl, lens, seed, sub_tokens=16384):
     while i < B:
         n = int(lens[order[i]]) + 1
         j = i
-        while j < B and int(lens[order[j]]) + 1 == n and (j - i + 1) * n <= sub_tokens:
+        while j < B and int(lens[order[j]]) + 1 == n and (j == i or (j - i + 1) * n <= sub_tokens):
             j += 1
         ids = [int(s) for s in order[i:j]]
         x = torch.randn((T, len(ids), n, H), generator=g, device=model.device, dtype=torch.float32).to(torch.bfloat16)

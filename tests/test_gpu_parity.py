@@ -155,3 +155,11 @@ def test_bf16_decode_split_kv_long_context(H, nq, nkv):
     via an extra prefill chunk on one sequence only is covered by the decode steps below."""
     wl = small("bf16", T=2, L=2, D=1, H=H, nq=nq, nkv=nkv, F=128)
     run_case(wl, B=2, S=700, decode_steps=2, shuffle=True, std=0.05, gain_jitter=0.1)
+
+
+@pytest.mark.parametrize("D", [2, 4])
+def test_bf16_table1_head_layout_eight_query_heads_one_kv_head(D):
+    """Table 1's per-track head partition (8 query heads sharing 1 KV head) with block depths 2 and 4;
+    prefill in chunks, then decode steps over split key ranges."""
+    wl = small("bf16", T=2, L=4, D=D, H=512, nq=8, nkv=1, F=256)
+    run_case(wl, B=2, S=300, chunks=[290, 10], decode_steps=2, shuffle=True, gain_jitter=0.1)
