@@ -138,6 +138,7 @@ pt_status pt_model_create(const pt_config* cfg, pt_model** out) {
     m->off_g2 = take((size_t)c.L * c.T * c.hidden * 4);
     m->off_cos = take((size_t)c.max_pos * (dh / 2) * 4);
     m->off_sin = take((size_t)c.max_pos * (dh / 2) * 4);
+    m->off_cs16 = take((size_t)c.max_pos * (dh / 2) * 4);
     m->off_status = take(kStatusWords * 4);
     m->total_bytes = off;
     *out = m;
@@ -197,6 +198,12 @@ pt_status pt_model_bind_weights(pt_model* m, void* dev_buf, size_t bytes) {
     char* b = (char*)dev_buf;
     PT_CUDA(cudaMemcpy(b + m->off_cos, cs.data(), cs.size() * 4, cudaMemcpyHostToDevice));
     PT_CUDA(cudaMemcpy(b + m->off_sin, sn.data(), sn.size() * 4, cudaMemcpyHostToDevice));
+    {   // the tensor-core path reads (cos, sin) as fp16 pairs: 2^-12 absolute error, an eighth of the bf16
+        // rounding q and k receive right after the rotation, for half the table bytes per token
+        std::vector<__half2> cs16(cs.size());
+        for (size_t i = 0; i < cs.size(); ++i) cs16[i] = __halves2half2(__float2half_rn(cs[i]), __float2half_rn(sn[i]));
+        PT_CUDA(cudaMemcpy(b + m->off_cs16, cs16.data(), cs16.size() * 4, cudaMemcpyHostToDevice));
+    }
     PT_CUDA(cudaMemset(b + m->off_g1, 0, (size_t)c.L * c.T * c.hidden * 4));
     PT_CUDA(cudaMemset(b + m->off_g2, 0, (size_t)c.L * c.T * c.hidden * 4));
     PT_CUDA(cudaMemset(b + m->off_status, 0, kStatusWords * 4));

@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda.h>
 
 #include <atomic>
@@ -46,7 +47,7 @@ struct pt_model {
     size_t esz;                           // bytes per element of the model dtype
     bool tc;                              // bf16 tensor-core path (else SIMT)
     // byte offsets inside the bound weight buffer; matrices are [L][T][rows][cols]
-    size_t off_wqkv, off_wo, off_wgu, off_wd, off_g1, off_g2, off_cos, off_sin, off_status, total_bytes;
+    size_t off_wqkv, off_wo, off_wgu, off_wd, off_g1, off_g2, off_cos, off_sin, off_cs16, off_status, total_bytes;
     char* wbuf = nullptr;
     int tap_layer = -2;
     float* tap_buf = nullptr;
@@ -67,6 +68,7 @@ struct pt_model {
     }
     const float* rope_cos() const { return (const float*)(wbuf + off_cos); }
     const float* rope_sin() const { return (const float*)(wbuf + off_sin); }
+    const uint32_t* rope_cs16() const { return (const uint32_t*)(wbuf + off_cs16); }   // [max_pos][dh/2] (cos, sin) as fp16 pairs
 };
 
 struct pt_kv_cache {

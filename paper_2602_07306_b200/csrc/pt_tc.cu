@@ -148,7 +148,7 @@ pt_status tc_forward(Call& k) {
             p.N = m->Nqkv; p.K = H;
             p.ssq_in = w.ssq; p.ssq_in_tstride = ssq_tstride; p.ssq_tiles = tiles;
             p.q_out = q; p.pool_l = pool_l; p.pool_tstride = pool_tstride; p.slab_elems = c->slab_elems;
-            p.row_kvoff = w.meta.row_kvoff; p.row_pos = w.meta.row_pos; p.cs = m->rope_cos(); p.sn = m->rope_sin();
+            p.row_kvoff = w.meta.row_kvoff; p.row_pos = w.meta.row_pos; p.cs = m->rope_cos(); p.sn = m->rope_sin(); p.cs16 = m->rope_cs16();
             p.nq = g.heads; p.nkv = g.kv_heads; p.dh = m->dh; p.ps = c->ps;
             int bn = gemm_bn(p.N, M, T, EPI_QKV);
             ProfScope ps(m, st, 1);

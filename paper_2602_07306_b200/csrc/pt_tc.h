@@ -26,6 +26,7 @@ struct GemmP {
     int64_t pool_tstride, slab_elems;
     const int64_t* row_kvoff; const int32_t* row_pos;
     const float* cs; const float* sn;
+    const uint32_t* cs16;   // [max_pos][dh/2] (cos, sin) fp16 pairs
     int nq, nkv, dh, ps;
     // EPI_SWIGLU
     __nv_bfloat16* z_out;   // [T][M][N/2]

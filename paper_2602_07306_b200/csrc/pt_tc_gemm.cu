@@ -212,8 +212,8 @@ __device__ __forceinline__ bool epi_swiglu(const GemmP& p, uint32_t taddr, int t
 }
 
 // A unit is 32 accumulator columns of one head: for q and k heads the 16 columns j0..j0+15 and
-// their rotary partners j0+dh/2.., for v heads 32 consecutive columns.  The 16 cos and 16 sin
-// values of the row's position are fetched one unit ahead.
+// their rotary partners j0+dh/2.., for v heads 32 consecutive columns.  The 16 (cos, sin) pairs
+// of the row's position (fp16, 64 bytes) are fetched one unit ahead.
 template <int BN, class Wait>
 __device__ __forceinline__ bool epi_qkv(const GemmP& p, uint32_t taddr, int t, int row, bool row_ok, int n0, int half, Wait wait) {
     constexpr int UNITS = BN / 32;                        // units of the tile, alternating between the two warps
@@ -224,16 +224,14 @@ __device__ __forceinline__ bool epi_qkv(const GemmP& p, uint32_t taddr, int t, i
     const float rinv = row_rinv(p, t, row, row_ok);
     const bool slot_ok = row_ok && kvoff >= 0 && kvoff + (int64_t)(2 * p.nkv - 1) * p.ps * dh + dh <= p.slab_elems;
     if (row_ok && !slot_ok) report(p.status, PT_ERR_DEVICE_BOUNDS, LOC_ROPE_PAGE);
-    const float* csr = p.cs + (size_t)pos * halfdh;
-    const float* snr = p.sn + (size_t)pos * halfdh;
-    auto fetch = [&](int u, float* tab) {                 // tab[0..15] = cos, tab[16..31] = sin of columns j0..j0+15
+    const float* csr = reinterpret_cast<const float*>(p.cs16 + (size_t)pos * halfdh);   // (cos, sin) fp16 pairs, moved as 32-bit words
+    auto fetch = [&](int u, float* tab) {                 // tab[i] = packed (cos, sin) of column j0 + i
         const int hs = n0 / dh + u / upd;
         if (hs >= p.nq + p.nkv || !row_ok) return;         // v heads, columns past N, rows past M: no rotation
         const int j0 = (u % upd) * 16;
         ld256(csr + j0, tab); ld256(csr + j0 + 8, tab + 8);
-        ld256(snr + j0, tab + 16); ld256(snr + j0 + 8, tab + 24);
     };
-    float tab[32], nxt[32];
+    float tab[16], nxt[16];
     fetch(half, tab);
     if (!wait()) return false;
 #pragma unroll 1
@@ -264,8 +262,10 @@ __device__ __forceinline__ bool epi_qkv(const GemmP& p, uint32_t taddr, int t, i
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
                     const float l = lo[i] * rinv, h = hi[i] * rinv;
-                    lo[i] = l * tab[i] - h * tab[16 + i];
-                    hi[i] = h * tab[i] + l * tab[16 + i];
+                    const uint32_t w = __float_as_uint(tab[i]);
+                    const float2 cs = __half22float2(*reinterpret_cast<const __half2*>(&w));
+                    lo[i] = l * cs.x - h * cs.y;
+                    hi[i] = h * cs.x + l * cs.y;
                 }
                 store16_bf16(dst + sub * 16, lo);
                 store16_bf16(dst + halfdh + sub * 16, hi);
@@ -277,7 +277,7 @@ __device__ __forceinline__ bool epi_qkv(const GemmP& p, uint32_t taddr, int t, i
             }
         }
 #pragma unroll
-        for (int i = 0; i < 32; ++i) tab[i] = nxt[i];      // last: the fetch stays in flight until here
+        for (int i = 0; i < 16; ++i) tab[i] = nxt[i];      // last: the fetch stays in flight until here
     }
     return true;
 }
