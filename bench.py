@@ -172,14 +172,14 @@ def run_decode(wl, dev, steps, warmup, barrier, rank):
         while j < B and int(lens[order[j]]) == n and (j == i or (j - i + 1) * n <= 16384):
             j += 1
         ids = [int(s) for s in order[i:j]]
-        x = torch.randn((wl.T, len(ids), n, wl.hidden), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        x = torch.randn((wl.T, len(ids), n, wl.hidden), generator=g, device=dev, dtype=torch.float32).to(model.tdtype)
         model.prefill(cache, x, ids)
         i = j
     torch.cuda.synchronize()
     t_fill = time.time() - t_fill
     code = model.device_status()
     assert code == (0, 0), f"device status after cache fill: {code}"
-    xd = torch.randn((wl.T, B, wl.hidden), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    xd = torch.randn((wl.T, B, wl.hidden), generator=g, device=dev, dtype=torch.float32).to(model.tdtype)
     out = torch.empty((B, wl.hidden), dtype=torch.float32, device=dev)
 
     def step():
@@ -270,7 +270,7 @@ def run_prefill(wl, dev, steps, warmup, barrier, rank):
     cache = model.new_cache(pages, ps)
     seq_ids = list(range(B))
     g = torch.Generator(device=dev).manual_seed(rank_batch_seed(wl.seed, rank))
-    x = torch.randn((wl.T, B, S, wl.hidden), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    x = torch.randn((wl.T, B, S, wl.hidden), generator=g, device=dev, dtype=torch.float32).to(model.tdtype)
     out = torch.empty((B, S, wl.hidden), dtype=torch.float32, device=dev)
 
     def step():
@@ -300,10 +300,17 @@ def run_prefill(wl, dev, steps, warmup, barrier, rank):
     gemm_ms = sum(prof[k][0] for k in ("gemm_qkv", "gemm_out", "gemm_gate_up", "gemm_down", "gemm_down_sync")) / steps
     gemm_n = sum(prof[k][1] for k in ("gemm_qkv", "gemm_out", "gemm_gate_up", "gemm_down", "gemm_down_sync"))
     attn_ms = prof["attention"][0] / steps
+    if gemm_n == 0:        # the fp32 workload runs the plain kernels, which are not bracketed per category
+        gemm_ms, attn_ms = float("nan"), float("nan")
     gemm_tf = alg["gemm_flops"] / (gemm_ms * 1e-3) / 1e12
     attn_tf = alg["attn_flops"] / (attn_ms * 1e-3) / 1e12
     peak = pk["bf16_tflops_sustained"] if ms * steps > 1000 else pk["bf16_tflops"]
-    roof = {"bound": "tensor", "kernel": "gemm_tc (QKV, out, gate/up, down, down+sync)", "achieved": gemm_tf, "peak": peak,
+    if gemm_n == 0:
+        step_tf = alg["flops"] / (ms * 1e-3) / 1e12
+        roof = {"bound": "alu", "kernel": "plain fp32 kernels (launch-bound workload: absolute numbers only)", "achieved": step_tf,
+                "peak": None, "unit": "TFLOP/s", "frac": None, "traffic": None, "peak_kind": "not applicable"}
+    else:
+      roof = {"bound": "tensor", "kernel": "gemm_tc (QKV, out, gate/up, down, down+sync)", "achieved": gemm_tf, "peak": peak,
             "unit": "TFLOP/s", "frac": gemm_tf / peak, "traffic": None, "peak_kind": f"of {pk_kind}",
             "avg_launch_ms": gemm_ms * steps / max(gemm_n, 1), "launches": gemm_n,
             "frac_of_nominal_2250": gemm_tf / 2250.0, "attention_tflops": attn_tf,
