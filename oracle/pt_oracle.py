@@ -270,3 +270,50 @@ def pt_decode_step(cfg: PTConfig, weights, x: np.ndarray, cache: PagedKVCache, s
     written at position length[seq] and attends positions 0..length[seq]."""
     x = np.asarray(x, np.float64)
     return pt_prefill(cfg, weights, x[:, :, None, :], cache, seq_ids, taps)[:, 0, :]
+
+
+# ----------------------------------------------------------------------------- ends of the model
+# Algorithm 1 starts from the embedding output x and returns h; the paper measures time to first
+# token and time per output token (Tables 6-10), which need the two ends it does not spell out.
+# Declared conventions (nothing in the paper fixes them): one embedding table shared by all
+# tracks (Algorithm 1's "Set h_i = x"), a final RMSNorm with its own gain on h, an untied
+# LM-head matrix, greedy decoding that takes the lowest index among equal maxima.
+
+def embed(table: np.ndarray, tokens: np.ndarray) -> np.ndarray:
+    """Row tokens[...] of the embedding table [vocab, H] -> [..., H]."""
+    return np.asarray(table, np.float64)[np.asarray(tokens, np.int64)]
+
+
+def lm_head(h: np.ndarray, gain: np.ndarray, w_out: np.ndarray, eps: float) -> np.ndarray:
+    """logits = rmsnorm(h; gain) @ w_out.T with w_out [vocab, H]."""
+    return rmsnorm(np.asarray(h, np.float64), np.asarray(gain, np.float64), eps) @ np.asarray(w_out, np.float64).T
+
+
+def greedy(logits: np.ndarray) -> np.ndarray:
+    """Index of the largest logit per row (the lowest index when several are equal)."""
+    return np.argmax(logits, axis=-1).astype(np.int64)
+
+
+def pt_generate(cfg: PTConfig, weights, table, gain, w_out, prompt: np.ndarray, n_new: int,
+                cache: PagedKVCache, seq_ids, round_x=None):
+    """Greedy generation: prefill the prompt [B, S] (token ids), take the next token from the last
+    position's logits, then one decode step per further token.  Every track starts from the same
+    embedding (Algorithm 1).  ``round_x`` (optional) is applied to the embedded inputs, for callers
+    whose model consumes them in a narrower type.  Returns (tokens [B, n_new], logits [B, n_new, V])."""
+    prompt = np.asarray(prompt, np.int64)
+    B, S = prompt.shape
+    fix = round_x if round_x is not None else (lambda a: a)
+    x = fix(embed(table, prompt))                                       # [B, S, H]
+    h = pt_prefill(cfg, weights, np.broadcast_to(x, (cfg.T,) + x.shape), cache, seq_ids)
+    out_tok = np.zeros((B, n_new), np.int64)
+    out_logits = []
+    logits = lm_head(h[:, -1, :], gain, w_out, cfg.rms_eps)              # [B, V]
+    for i in range(n_new):
+        out_logits.append(logits)
+        out_tok[:, i] = greedy(logits)
+        if i + 1 == n_new:
+            break
+        x = fix(embed(table, out_tok[:, i]))                              # [B, H]
+        h = pt_decode_step(cfg, weights, np.broadcast_to(x, (cfg.T,) + x.shape), cache, seq_ids)
+        logits = lm_head(h, gain, w_out, cfg.rms_eps)
+    return out_tok, np.stack(out_logits, axis=1)

@@ -376,3 +376,50 @@ def test_workload_recipe():
     assert w["wq"].shape == (128, 128) and w["wg"].shape == (512, 128) and w["wd"].shape == (128, 512)
     assert abs(float(w["wg"].std()) - 0.02) < 1e-3 and np.all(w["g1"] == 1)
     np.testing.assert_array_equal(w["wq"], I.WeightSource(I.WORKLOADS["cfg0"]).get(1, 2)["wq"])
+
+
+# ----------------------------------------------------------------------------- ends of the model
+
+def test_embedding_is_a_one_hot_product():
+    rng = np.random.default_rng(0)
+    table = rng.standard_normal((11, 6))
+    tokens = np.array([[3, 0, 10], [7, 7, 1]])
+    onehot = np.zeros(tokens.shape + (11,))
+    for idx in np.ndindex(tokens.shape):
+        onehot[idx + (tokens[idx],)] = 1.0
+    assert np.array_equal(O.embed(table, tokens), onehot @ table)
+
+
+def test_lm_head_against_torch_rms_norm_and_linear():
+    import torch
+    rng = np.random.default_rng(1)
+    h, g, w = rng.standard_normal((5, 16)), 1 + 0.1 * rng.standard_normal(16), rng.standard_normal((9, 16))
+    want = torch.nn.functional.linear(torch.nn.functional.rms_norm(torch.from_numpy(h), (16,), torch.from_numpy(g), 1e-6),
+                                      torch.from_numpy(w)).numpy()
+    assert np.allclose(O.lm_head(h, g, w, 1e-6), want, rtol=1e-12, atol=1e-12)
+
+
+def test_greedy_takes_the_lowest_index_among_equal_maxima():
+    assert O.greedy(np.array([[1.0, 5.0, 5.0, 2.0], [7.0, 7.0, 7.0, 7.0], [0.0, -1.0, 3.0, 3.0]])).tolist() == [1, 0, 2]
+
+
+def test_generation_equals_teacher_forced_prefill():
+    """Feeding the generated tokens back one at a time (decode steps) gives the same logits as one
+    prefill over prompt + generated tokens: the cache and the positions line up at both ends."""
+    wl = I.Workload("gen", T=2, L=4, D=2, hidden=32, heads=2, kv_heads=1, ffn=48, dtype="f32", mode="prefill", batch=2, seq=5)
+    cfg = O.PTConfig(T=wl.T, D=wl.D, L=wl.L, hidden=wl.hidden, heads=wl.heads, kv_heads=wl.kv_heads, ffn=wl.ffn)
+    ws = I.WeightSource(wl, std=0.3)
+    rng = np.random.default_rng(2)
+    V = 13
+    table, gain, w_out = rng.standard_normal((V, wl.hidden)), 1 + 0.1 * rng.standard_normal(wl.hidden), rng.standard_normal((V, wl.hidden))
+    prompt = rng.integers(0, V, (2, 5))
+    cache = O.PagedKVCache(cfg, 8, 4)
+    toks, logits = O.pt_generate(cfg, ws, table, gain, w_out, prompt, 4, cache, [0, 1])
+    full = np.concatenate([prompt, toks[:, :3]], axis=1)                  # the last token is never fed back
+    cache2 = O.PagedKVCache(cfg, 8, 4)
+    x = O.embed(table, full)
+    h = O.pt_prefill(cfg, ws, np.broadcast_to(x, (cfg.T,) + x.shape), cache2, [0, 1])
+    want = O.lm_head(h[:, 4:], gain, w_out, cfg.rms_eps)                  # logits after positions 4..7
+    assert np.allclose(logits, want, rtol=1e-9, atol=1e-9)
+    assert np.array_equal(toks, O.greedy(want))
+    assert cache.length[0] == cache.length[1] == 8
