@@ -178,6 +178,47 @@ pt_status pt_decode_step(pt_model* m, pt_kv_cache* c, const void* x, int64_t x_t
                          int32_t B, const int32_t* seq_ids, void* out_h,
                          void* workspace, size_t ws_bytes, void* stream);
 
+/* ---- ends of the model (bf16 models) -----------------------------------------------------------
+ * Algorithm 1 takes the embedding output x and returns h; the paper's latency tables (time to first
+ * token, time per output token: Tables 6-10) need the two ends it leaves to "standard" practice.
+ * Conventions of this library: one embedding table [vocab][hidden] shared by every track (Algorithm 1,
+ * "Set h_i = x"), a final RMSNorm with its own gain, an untied LM head [vocab][hidden], greedy choice =
+ * lowest index among the largest logits.  vocab must be a multiple of 16. */
+
+/* Bytes of, and binding of, the caller-owned device buffer (256-byte aligned) that holds the embedding
+ * table, the LM head (both in the model dtype) and the final gain (fp32). */
+pt_status pt_lm_bytes(const pt_model* m, int32_t vocab, size_t* bytes);
+pt_status pt_lm_bind(pt_model* m, int32_t vocab, void* dev_buf, size_t bytes);
+/* Copy one of them from `dev_src` (device, row-major): kind 0 = embedding table, 1 = LM head,
+ * 2 = final gain [hidden] fp32. */
+pt_status pt_lm_set(pt_model* m, int32_t kind, const void* dev_src, void* stream);
+
+/* x_out[r][:] = table[dev_tokens[r]][:] for r < n (device int32 ids; x_out device, 16-byte aligned,
+ * [n][hidden]).  Pass x_out to pt_prefill / pt_decode_step with x_track_stride = 0.  An id outside
+ * [0, vocab) is reported through pt_device_status (PT_ERR_DEVICE_BOUNDS) and read as id 0. */
+pt_status pt_embed(pt_model* m, const int32_t* dev_tokens, int64_t n, void* x_out, void* stream);
+
+/* logits[r][:] = rmsnorm(h_r; final gain) . head^T for the n rows h_r = h + r*row_stride (fp32, device,
+ * 16-byte aligned; row_stride in elements, a multiple of 4 - use S*hidden with h pointing at the last
+ * position to take one row per sequence of a prefill output).  logits: device fp32 [n][vocab];
+ * next_token (device int32 [n], may be NULL) receives the greedy choice; workspace: device, 256-byte
+ * aligned, >= pt_lm_workspace_bytes(n). */
+pt_status pt_lm_workspace_bytes(const pt_model* m, int64_t n, size_t* bytes);
+pt_status pt_lm_head(pt_model* m, const float* h, int64_t row_stride, int64_t n, float* logits, int32_t* next_token,
+                     void* workspace, size_t ws_bytes, void* stream);
+
+/* Greedy generation for B sequences: embed and prefill the prompts (dev_prompt: device int32 [B][S]),
+ * take each sequence's next token from its last position, then one decode step per further token, n_new
+ * tokens in all.  Token ids never leave the device, so the whole loop is asynchronous on `stream`.
+ *   dev_tokens_out  device int32 [B][n_new]
+ *   dev_logits_out  device fp32 [B][n_new][vocab] or NULL: the logits each token was chosen from
+ *   workspace       device, 256-byte aligned, >= pt_generate_workspace_bytes(B, S, page_size)
+ * The sequences seq_ids[b] grow by S + n_new - 1 positions (the last token is not fed back). */
+pt_status pt_generate_workspace_bytes(const pt_model* m, int32_t B, int32_t S, int32_t page_size, size_t* bytes);
+pt_status pt_generate(pt_model* m, pt_kv_cache* c, const int32_t* dev_prompt, int32_t B, int32_t S, int32_t n_new,
+                      const int32_t* seq_ids, int32_t* dev_tokens_out, float* dev_logits_out,
+                      void* workspace, size_t ws_bytes, void* stream);
+
 /* Debug tap.  `dev_buf` (device, fp32) receives the residual stream of the following forward
  * calls: for each tapped layer two [T][tokens][hidden] blocks, the first after the attention
  * residual add, the second after the whole layer (after the sync when the layer closes a

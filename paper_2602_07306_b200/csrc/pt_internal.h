@@ -26,6 +26,7 @@ enum : int {
     LOC_GEMM_EPI_WAIT = 5, LOC_GEMM_EMPTY_WAIT = 6, LOC_DECODE_PAGE = 7, LOC_FLASH_PAGE = 8,
     LOC_GEMM_ACC_WAIT = 9,
     LOC_FLASH_KEMPTY = 10, LOC_FLASH_VEMPTY = 11, LOC_FLASH_VRAW = 12, LOC_FLASH_KFULL = 13, LOC_FLASH_QFULL = 14,
+    LOC_EMBED_TOKEN = 19,
     LOC_FLASH_PFULL = 15, LOC_FLASH_VFULL = 16, LOC_FLASH_SFULL = 17, LOC_FLASH_OREADY = 18,
 };
 
@@ -49,6 +50,8 @@ struct pt_model {
     // byte offsets inside the bound weight buffer; matrices are [L][T][rows][cols]
     size_t off_wqkv, off_wo, off_wgu, off_wd, off_g1, off_g2, off_cos, off_sin, off_cs16, off_status, total_bytes;
     char* wbuf = nullptr;
+    char* lm_buf = nullptr;                // embedding table, LM head, final gain (pt_lm_bind)
+    int lm_vocab = 0;
     int tap_layer = -2;
     float* tap_buf = nullptr;
     std::vector<char> meta_host;          // staging for the per-call metadata upload

@@ -57,6 +57,14 @@ _PROTOS = {
     "pt_workspace_bytes": (_I32, [_P, _I64, _I32, _I32, C.POINTER(_SZ)]),
     "pt_prefill": (_I32, [_P, _P, _P, _I64, _I32, _I32, C.POINTER(_I32), _P, _P, _SZ, _P]),
     "pt_decode_step": (_I32, [_P, _P, _P, _I64, _I32, C.POINTER(_I32), _P, _P, _SZ, _P]),
+    "pt_lm_bytes": (_I32, [_P, _I32, C.POINTER(_SZ)]),
+    "pt_lm_bind": (_I32, [_P, _I32, _P, _SZ]),
+    "pt_lm_set": (_I32, [_P, _I32, _P, _P]),
+    "pt_embed": (_I32, [_P, _P, _I64, _P, _P]),
+    "pt_lm_workspace_bytes": (_I32, [_P, _I64, C.POINTER(_SZ)]),
+    "pt_lm_head": (_I32, [_P, _P, _I64, _I64, _P, _P, _P, _SZ, _P]),
+    "pt_generate_workspace_bytes": (_I32, [_P, _I32, _I32, _I32, C.POINTER(_SZ)]),
+    "pt_generate": (_I32, [_P, _P, _P, _I32, _I32, _I32, C.POINTER(_I32), _P, _P, _P, _SZ, _P]),
     "pt_set_debug_tap": (_I32, [_P, _I32, _P]),
     "pt_device_status": (_I32, [_P, _P, C.POINTER(_I32), C.POINTER(_I32)]),
     "pt_profile_enable": (_I32, [_P, _I32]),
@@ -236,6 +244,65 @@ class Model:
             check(lib().pt_decode_step(self.h, cache.h, x.data_ptr(), stride, B, pids, out.data_ptr(),
                                        ws.data_ptr(), ws.numel(), self._stream()))
         return out
+
+    # ---- ends of the model -------------------------------------------------------------------
+    def load_lm(self, table, head, gain) -> None:
+        """table, head: [vocab, hidden]; gain: [hidden] (numpy or torch); stored in the model dtype / fp32."""
+        torch = self.torch
+        as_t = lambda a: torch.from_numpy(np.ascontiguousarray(a)) if isinstance(a, np.ndarray) else a
+        table, head, gain = as_t(table), as_t(head), as_t(gain)
+        self.vocab = table.shape[0]
+        n = _SZ()
+        check(lib().pt_lm_bytes(self.h, self.vocab, C.byref(n)))
+        with torch.cuda.device(self.device):
+            self.lm_buf = torch.empty(n.value, dtype=torch.uint8, device=self.device)
+            check(lib().pt_lm_bind(self.h, self.vocab, self.lm_buf.data_ptr(), n.value))
+            for kind, w, dt in ((0, table, self.tdtype), (1, head, self.tdtype), (2, gain, torch.float32)):
+                w = w.to(device=self.device, dtype=dt).contiguous()
+                check(lib().pt_lm_set(self.h, kind, w.data_ptr(), self._stream()))
+                torch.cuda.current_stream().synchronize()
+
+    def embed(self, tokens):
+        """tokens: int32 CUDA tensor of any shape -> [..., hidden] in the model dtype."""
+        torch = self.torch
+        assert tokens.is_cuda and tokens.dtype == torch.int32 and tokens.is_contiguous()
+        x = torch.empty(tuple(tokens.shape) + (self.cfg.hidden,), dtype=self.tdtype, device=self.device)
+        with torch.cuda.device(self.device):
+            check(lib().pt_embed(self.h, tokens.data_ptr(), tokens.numel(), x.data_ptr(), self._stream()))
+        return x
+
+    def lm_head(self, h, want_tokens=True):
+        """h: fp32 CUDA [n, hidden] (contiguous) -> (logits fp32 [n, vocab], greedy tokens int32 [n] or None)."""
+        torch = self.torch
+        assert h.is_cuda and h.dtype == torch.float32 and h.is_contiguous() and h.dim() == 2
+        n = h.shape[0]
+        logits = torch.empty((n, self.vocab), dtype=torch.float32, device=self.device)
+        tok = torch.empty(n, dtype=torch.int32, device=self.device) if want_tokens else None
+        nb = _SZ()
+        check(lib().pt_lm_workspace_bytes(self.h, n, C.byref(nb)))
+        ws = torch.empty(nb.value, dtype=torch.uint8, device=self.device)
+        with torch.cuda.device(self.device):
+            check(lib().pt_lm_head(self.h, h.data_ptr(), h.shape[1], n, logits.data_ptr(), tok.data_ptr() if want_tokens else None,
+                                   ws.data_ptr(), ws.numel(), self._stream()))
+        return logits, tok
+
+    def generate(self, cache: "Cache", prompt, n_new: int, seq_ids, want_logits=False):
+        """prompt: int32 CUDA [B, S] -> (tokens int32 [B, n_new], logits fp32 [B, n_new, vocab] or None)."""
+        torch = self.torch
+        assert prompt.is_cuda and prompt.dtype == torch.int32 and prompt.is_contiguous()
+        B, S = prompt.shape
+        out = torch.empty((B, n_new), dtype=torch.int32, device=self.device)
+        logits = torch.empty((B, n_new, self.vocab), dtype=torch.float32, device=self.device) if want_logits else None
+        nb = _SZ()
+        check(lib().pt_generate_workspace_bytes(self.h, B, S, cache.page_size, C.byref(nb)))
+        if getattr(self, "gen_ws", None) is None or self.gen_ws.numel() < nb.value:
+            self.gen_ws = None
+            self.gen_ws = torch.empty(nb.value, dtype=torch.uint8, device=self.device)
+        ids, pids = _i32arr(seq_ids)
+        with torch.cuda.device(self.device):
+            check(lib().pt_generate(self.h, cache.h, prompt.data_ptr(), B, S, n_new, pids, out.data_ptr(),
+                                    logits.data_ptr() if want_logits else None, self.gen_ws.data_ptr(), self.gen_ws.numel(), self._stream()))
+        return out, logits
 
     PROF_NAMES = ("attention", "gemm_qkv", "gemm_out", "gemm_gate_up", "gemm_down", "gemm_down_sync", "other")
 
