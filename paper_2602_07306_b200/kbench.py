@@ -3,6 +3,7 @@
     python -m paper_2602_07306_b200.kbench decode --T 8 --B 64 --nq 8 --nkv 8 --dh 128 --len 2048
     python -m paper_2602_07306_b200.kbench prefill --T 8 --B 8 --S 4096 --nq 8 --nkv 8 --dh 128 [--impl 1]
     python -m paper_2602_07306_b200.kbench layer --T 8 --B 2 --S 4096 --H 1024 --nq 8 --nkv 8 --F 2816
+    python -m paper_2602_07306_b200.kbench generate --B 1 --S 1024 --new 64 [--depth 2|4|8]
     python -m paper_2602_07306_b200.kbench gemm --T 8 --M 32768 --N 3072 --K 1024 [--bn 256] [--fold]
 
 Prints one JSON line: average device time per launch (CUDA events on the launching stream,
@@ -119,6 +120,46 @@ def layer(a):
     print(json.dumps({"kernel": "layer", "per_launch": res, "args": vars(a)}))
 
 
+def generate(a):
+    """Greedy generation at the head layout of the paper's 30B model (inputs.WORKLOADS["pt30b_prefill"]): time
+    to the first token (embed + prefill + LM head + choice) and time per further token, batch a.B."""
+    from paper_2602_07306_b200 import inputs as I
+    import dataclasses
+    wl = I.WORKLOADS["pt30b_prefill"]
+    if a.depth:
+        wl = dataclasses.replace(wl, D=a.depth)
+    dev = torch.device("cuda:0")
+    m = pt.Model(T=wl.T, D=wl.D, L=wl.L, hidden=wl.hidden, heads=wl.heads, kv_heads=wl.kv_heads, ffn=wl.ffn,
+                 dtype="bf16", max_pos=a.S + a.new + 16, device=dev)
+    m.init_random(0)
+    g = torch.Generator(device=dev).manual_seed(0)
+    H = wl.hidden
+    m.load_lm(torch.randn((a.vocab, H), generator=g, device=dev), torch.randn((a.vocab, H), generator=g, device=dev) * 0.05,
+              torch.ones(H, device=dev))
+    pages = a.B * (-(-(a.S + a.new) // 16))
+    cache = m.new_cache(pages, 16)
+    prompt = torch.randint(0, a.vocab, (a.B, a.S), generator=g, device=dev, dtype=torch.int32)
+    ids = list(range(a.B))
+
+    def run(n_new):
+        for s_ in ids:
+            if cache.length(s_):
+                cache.truncate(s_, 0)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        toks, _ = m.generate(cache, prompt, n_new, ids)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+    for _ in range(a.warmup):
+        run(2)
+    ttft = min(run(1) for _ in range(a.iters))
+    full = min(run(1 + a.new) for _ in range(a.iters))
+    assert m.device_status() == (0, 0)
+    print(json.dumps({"kernel": "generate", "ttft_ms": ttft, "tpot_ms": (full - ttft) / a.new, "tokens_per_s": a.B * a.new / ((full - ttft) * 1e-3),
+                      "model": f"T={wl.T} L={wl.L} D={wl.D} H={wl.hidden} heads={wl.heads}/{wl.kv_heads} F={wl.ffn} vocab={a.vocab}", "args": vars(a)}))
+
+
 def gemm(a):
     dev = torch.device("cuda:0")
     g = torch.Generator(device=dev).manual_seed(0)
@@ -151,12 +192,15 @@ def main():
     ly = sub.add_parser("layer")
     for k, v in dict(T=8, B=2, S=4096, H=1024, nq=8, nkv=8, F=2816, ps=16, iters=3, warmup=1).items():
         ly.add_argument("--" + k, type=int, default=v)
+    gn = sub.add_parser("generate")
+    for k, v in dict(B=1, S=1024, new=64, vocab=32000, depth=0, iters=3, warmup=1).items():
+        gn.add_argument("--" + k, type=int, default=v)
     gm = sub.add_parser("gemm")
     for k, v in dict(T=8, M=4096, N=3072, K=1024, bn=0, iters=20, warmup=3).items():
         gm.add_argument("--" + k, type=int, default=v)
     gm.add_argument("--fold", action="store_true")
     a = ap.parse_args()
-    {"decode": decode, "gemm": gemm, "prefill": prefill, "layer": layer}[a.cmd](a)
+    {"decode": decode, "gemm": gemm, "prefill": prefill, "layer": layer, "generate": generate}[a.cmd](a)
 
 
 if __name__ == "__main__":
