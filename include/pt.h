@@ -41,7 +41,7 @@ typedef enum {
     PT_OK = 0,
     PT_ERR_INVALID_ARG = 1,      /* null pointer, negative size, index out of range            */
     PT_ERR_BAD_CONFIG = 2,       /* L % D != 0, hidden % heads != 0, heads % kv_heads != 0 ... */
-    PT_ERR_UNSUPPORTED = 3,      /* valid architecture this build has no kernel for            */
+    PT_ERR_UNSUPPORTED = 3,      /* valid architecture the library has no kernel for          */
     PT_ERR_BUFFER_TOO_SMALL = 4, /* caller buffer smaller than the matching *_bytes query      */
     PT_ERR_CACHE_FULL = 5,       /* no free page left                                          */
     PT_ERR_MISALIGNED = 6,       /* device pointer not aligned as documented                   */
