@@ -23,7 +23,6 @@ namespace {
 constexpr int kFlashThreads = 384;
 constexpr int kStages = 2;                 // K ring and V ring depth
 constexpr uint32_t kSpin = 1u << 26;
-constexpr int kPolyOf8 = 0;                // of every 8 scores, 2 (value 4) or 4 (value 8) take the polynomial exp2
 constexpr int kHalfBytes = 128 * 128;      // 128 rows x 64 bf16: one swizzled column block of a tile
 
 enum { B_QFULL = 0, B_KFULL = 2, B_KEMPTY = 4, B_VFULL = 6, B_VEMPTY = 8, B_SFULL = 10, B_PFULL = 12,
@@ -128,29 +127,6 @@ __device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, f
 __device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1) {                    // d += a
     asm("{\n .reg .b64 ra, rd;\n mov.b64 ra, {%2, %3};\n mov.b64 rd, {%0, %1};\n add.rn.f32x2 rd, rd, ra;\n mov.b64 {%0, %1}, rd;\n}"
         : "+f"(d0), "+f"(d1) : "f"(a0), "f"(a1));
-}
-// (a0, a1) * (b0, b1) + (c0, c1)
-__device__ __forceinline__ void fma2v(float& d0, float& d1, float a0, float a1, float b0, float b1, float c0, float c1) {
-    asm("{\n .reg .b64 ra, rb, rc, rd;\n mov.b64 ra, {%2, %3};\n mov.b64 rb, {%4, %5};\n mov.b64 rc, {%6, %7};\n"
-        " fma.rn.f32x2 rd, ra, rb, rc;\n mov.b64 {%0, %1}, rd;\n}"
-        : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1), "f"(c0), "f"(c1));
-}
-// 2^x for a pair of x <= 0 without the special-function unit: x = r + f with r = round(x) taken
-// from the low mantissa bits of x + 1.5*2^23, 2^f from a cubic fitted on [-0.5, 0.5] (relative
-// error below 8e-5, far inside the bf16 rounding P receives), 2^r added into the exponent field.
-__device__ __forceinline__ void ex2_poly2(float& x0, float& x1) {
-    constexpr float kMagic = 12582912.0f;
-    constexpr float k0 = 0.99992895f, k1 = 0.69327623f, k2 = 0.24260405f, k3 = 0.05508868f;
-    x0 = fmaxf(x0, -126.0f); x1 = fmaxf(x1, -126.0f);
-    float t0, t1, r0, r1, f0, f1, p0, p1;
-    fma2v(t0, t1, x0, x1, 1.0f, 1.0f, kMagic, kMagic);
-    fma2v(r0, r1, t0, t1, 1.0f, 1.0f, -kMagic, -kMagic);
-    fma2v(f0, f1, r0, r1, -1.0f, -1.0f, x0, x1);
-    fma2v(p0, p1, f0, f1, k3, k3, k2, k2);
-    fma2v(p0, p1, p0, p1, f0, f1, k1, k1);
-    fma2v(p0, p1, p0, p1, f0, f1, k0, k0);
-    x0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(t0) << 23));
-    x1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
 }
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float d;
@@ -432,8 +408,7 @@ k_flash_prefill_tc(const __grid_constant__ CUtensorMap qmap, const __grid_consta
                     float x0, x1, x2, x3;
                     fma2(x0, x1, v[cc * 32 + e], v[cc * 32 + e + 1], c, nmc);
                     fma2(x2, x3, v[cc * 32 + e + 2], v[cc * 32 + e + 3], c, nmc);
-                    x0 = ex2(x0); x1 = ex2(x1);
-                    if ((e & 7) < kPolyOf8) ex2_poly2(x2, x3); else { x2 = ex2(x2); x3 = ex2(x3); }
+                    x0 = ex2(x0); x1 = ex2(x1); x2 = ex2(x2); x3 = ex2(x3);
                     add2(l0, l1, x0, x1);
                     add2(l2, l3, x2, x3);
                     pk[e >> 1] = pack_bf16(x0, x1);
