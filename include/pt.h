@@ -219,6 +219,20 @@ pt_status pt_generate(pt_model* m, pt_kv_cache* c, const int32_t* dev_prompt, in
                       const int32_t* seq_ids, int32_t* dev_tokens_out, float* dev_logits_out,
                       void* workspace, size_t ws_bytes, void* stream);
 
+/* ---- track parallelism across GPUs ---------------------------------------------------------------
+ * The paper's deployment (Sections 2.2 and 3.3): each GPU holds some of the tracks and the track-sync is
+ * one all-reduce per track block, L/D per forward against tensor parallelism's 2L.  A model created
+ * with cfg.T = the tracks of THIS rank can be told that it is part of a larger stack of `world_tracks`
+ * tracks; at every sync it then sums its own tracks into one fp32 [tokens][hidden] buffer, calls `fn`
+ * once, and continues from the result.  `fn(user, dev_buf, count, stream)` must replace the `count`
+ * fp32 values at `dev_buf` (device) by their sum over all ranks, enqueued on `stream` (e.g. an NCCL
+ * all-reduce), and return 0; any other return value fails the forward call with PT_ERR_CUDA.  With
+ * sync_op = MEAN the mean is taken over world_tracks.  Every rank passes the same batch; x holds the
+ * rank's own tracks.  fn == NULL or world_tracks == 0 returns the model to the single-GPU schedule.
+ * bf16 models on the tensor-core path only. */
+typedef int32_t (*pt_allreduce_fn)(void* user, void* dev_buf, int64_t count, void* stream);
+pt_status pt_model_set_track_group(pt_model* m, int32_t world_tracks, pt_allreduce_fn fn, void* user);
+
 /* Debug tap.  `dev_buf` (device, fp32) receives the residual stream of the following forward
  * calls: for each tapped layer two [T][tokens][hidden] blocks, the first after the attention
  * residual add, the second after the whole layer (after the sync when the layer closes a

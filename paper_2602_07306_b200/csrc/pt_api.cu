@@ -172,6 +172,15 @@ pt_status pt_profile_read(pt_model* m, float* ms, int64_t* launches) {
     return PT_OK;
 }
 
+pt_status pt_model_set_track_group(pt_model* m, int32_t world_tracks, pt_allreduce_fn fn, void* user) {
+    if (!m) PT_FAIL(PT_ERR_INVALID_ARG, "null argument");
+    if (!fn || world_tracks == 0) { m->world_tracks = 0; m->ar_fn = nullptr; m->ar_user = nullptr; return PT_OK; }
+    if (!m->tc) PT_FAIL(PT_ERR_UNSUPPORTED, "track groups are built for bf16 models on the tensor-core path");
+    if (world_tracks < m->cfg.T) PT_FAIL(PT_ERR_INVALID_ARG, "world_tracks %d is smaller than this rank's %d tracks", world_tracks, m->cfg.T);
+    m->world_tracks = world_tracks; m->ar_fn = fn; m->ar_user = user;
+    return PT_OK;
+}
+
 int32_t pt_sync_count(const pt_model* m) { return m ? m->cfg.L / m->cfg.D : -1; }
 
 pt_status pt_model_weight_bytes(const pt_model* m, size_t* bytes) {

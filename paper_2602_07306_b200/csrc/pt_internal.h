@@ -52,6 +52,9 @@ struct pt_model {
     char* wbuf = nullptr;
     char* lm_buf = nullptr;                // embedding table, LM head, final gain (pt_lm_bind)
     int lm_vocab = 0;
+    int world_tracks = 0;                  // > 0: this model holds cfg.T of world_tracks tracks (pt_model_set_track_group)
+    pt_allreduce_fn ar_fn = nullptr;
+    void* ar_user = nullptr;
     int tap_layer = -2;
     float* tap_buf = nullptr;
     std::vector<char> meta_host;          // staging for the per-call metadata upload

@@ -190,11 +190,14 @@ pt_status tc_forward(Call& k) {
             // a decode step (few rows): per-track down GEMM on the whole machine, then a small reduction kernel;
             // many rows (prefill): one GEMM whose K loop runs over (track, k) and whose epilogue is the sync
             const bool split_sync = sync && k.decode && M <= 256;
+            const bool grouped = sync && m->ar_fn != nullptr;          // tracks of other ranks join through an all-reduce
+            const float sync_scale = g.sync_op ? 1.0f / (float)(grouped ? m->world_tracks : T) : 1.0f;
             if (sync && !split_sync) {
                 p.T = 1; p.kt = T; p.n_sum = T; p.n_out = T;
-                p.scale = g.sync_op ? 1.0f / T : 1.0f;
-                p.h_out = last ? k.out : w.hS; p.h_out_tstride = 0;
+                p.scale = grouped ? 1.0f : sync_scale;
+                p.h_out = (last && !grouped) ? k.out : w.hS; p.h_out_tstride = 0;
                 p.ssq_out_tstride = 0;
+                if (grouped) { p.hb_out = nullptr; p.ssq_out = nullptr; }
             } else {
                 p.h_out = w.hT; p.h_out_tstride = MH;
                 p.ssq_out_tstride = (size_t)M * tiles;
@@ -203,14 +206,25 @@ pt_status tc_forward(Call& k) {
             int bn = gemm_bn(p.N, M, p.T, EPI_RESID);
             ProfScope ps(m, st, sync ? 5 : 4);
             if ((s = launch_gemm(EPI_RESID, bn, ta_z, wm[l].m[3][bn_index(bn)], p, st)) != PT_OK) return s;
-            if (split_sync) {
-                float* ho = last ? k.out : w.hS;
-                k_track_sync<<<(M * 32 + 255) / 256, 256, 0, st>>>(w.hT, MH, T, g.sync_op ? 1.0f / T : 1.0f, ho,
-                                                                   last ? nullptr : hb, last ? nullptr : m->gain(0, l + 1),
-                                                                   last ? nullptr : w.ssq, M, H, tiles);
+            float* ho = last ? k.out : w.hS;
+            __nv_bfloat16* hb_next = last ? nullptr : hb;
+            const float* gain_next = last ? nullptr : m->gain(0, l + 1);
+            float* ssq_next = last ? nullptr : w.ssq;
+            const unsigned sync_grid = (unsigned)((M * 32 + 255) / 256);
+            if (split_sync) {       // local tracks -> one stream (the final one unless other ranks still have to join)
+                k_track_sync<<<sync_grid, 256, 0, st>>>(w.hT, MH, T, grouped ? 1.0f : sync_scale, grouped ? w.hS : ho,
+                                                        grouped ? nullptr : hb_next, grouped ? nullptr : gain_next,
+                                                        grouped ? nullptr : ssq_next, M, H, tiles);
                 g_launches.fetch_add(1, std::memory_order_relaxed);
             }
-            if (sync) { ssq_tstride = 0; hin = last ? k.out : w.hS; hin_stride = 0; }
+            if (grouped) {
+                // w.hS holds this rank's partial sum: one all-reduce per track block, then every local track's
+                // next operand from the total
+                if (m->ar_fn(m->ar_user, w.hS, (int64_t)M * H, (void*)st) != 0) { set_error("the all-reduce hook failed at layer %d", l); return PT_ERR_CUDA; }
+                k_track_sync<<<sync_grid, 256, 0, st>>>(w.hS, 0, 1, sync_scale, ho, hb_next, gain_next, ssq_next, M, H, tiles);
+                g_launches.fetch_add(1, std::memory_order_relaxed);
+            }
+            if (sync) { ssq_tstride = 0; hin = ho; hin_stride = 0; }
             else { ssq_tstride = (size_t)M * tiles; hin = w.hT; hin_stride = MH; }
         }
         tap_copy(k, l, 1, hin, hin_stride);

@@ -44,6 +44,7 @@ _PROTOS = {
     "pt_model_bind_weights": (_I32, [_P, _P, _SZ]),
     "pt_model_set_weight": (_I32, [_P, _I32, _I32, _I32, _P, _P]),
     "pt_sync_count": (_I32, [_P]),
+    "pt_model_set_track_group": (_I32, [_P, _I32, _P, _P]),
     "pt_kv_cache_bytes": (_I32, [_P, _I32, _I32, C.POINTER(_SZ)]),
     "pt_kv_cache_alloc": (_I32, [_P, _I32, _I32, _P, _SZ, C.POINTER(_P)]),
     "pt_kv_cache_free": (None, [_P]),
@@ -185,6 +186,27 @@ class Model:
                     for k in ("g1", "g2"):
                         check(lib().pt_model_set_weight(self.h, t, l, KIND[k], ones.data_ptr(), self._stream()))
             torch.cuda.synchronize()
+
+    def set_track_group(self, world_tracks: int, allreduce) -> None:
+        """This model holds cfg.T of `world_tracks` tracks; `allreduce(t)` must sum the fp32 CUDA tensor t in
+        place over all ranks on the current stream (e.g. torch.distributed.all_reduce).  None clears it."""
+        if allreduce is None:
+            check(lib().pt_model_set_track_group(self.h, 0, None, None))
+            self._ar_cb = None
+            return
+        torch = self.torch
+
+        def hook(user, ptr, count, stream):
+            try:
+                off = ptr - self.ws.data_ptr()
+                assert 0 <= off and off + 4 * count <= self.ws.numel(), "buffer outside the workspace"
+                allreduce(self.ws[off:off + 4 * count].view(torch.float32))
+                return 0
+            except Exception as e:      # never let an exception cross the C boundary
+                self._ar_error = e
+                return 1
+        self._ar_cb = C.CFUNCTYPE(_I32, _P, _P, _I64, _P)(hook)
+        check(lib().pt_model_set_track_group(self.h, world_tracks, C.cast(self._ar_cb, _P), None))
 
     def sync_count(self) -> int:
         return lib().pt_sync_count(self.h)
