@@ -121,11 +121,23 @@ def algorithmic(wl, B, lens=None, S=None):
     return {"flops": gemm + attn, "gemm_flops": gemm, "attn_flops": attn}
 
 
+TRACK_PARALLEL = {"on": False, "world": 1, "rank": 0, "tracks": 0}
+
+
 def make_model(wl, dev, max_pos):
+    """With --parallel tracks `wl` is one rank's share (T / N tracks, the paper's placement) of a
+    model of TRACK_PARALLEL["tracks"] tracks and the track-sync is one NCCL all-reduce per track
+    block; otherwise every rank holds the whole model."""
     from paper_2602_07306_b200 import pt
     m = pt.Model(T=wl.T, D=wl.D, L=wl.L, hidden=wl.hidden, heads=wl.heads, kv_heads=wl.kv_heads, ffn=wl.ffn,
                  dtype=wl.dtype, rope_base=wl.rope_base, rms_eps=wl.rms_eps, max_pos=max_pos, device=dev)
-    m.init_random(seed=wl.seed)
+    if TRACK_PARALLEL["on"]:
+        import torch.distributed as dist
+        m.init_random(seed=wl.seed + 100 * TRACK_PARALLEL["rank"])          # every rank its own tracks' weights
+        m.set_track_group(TRACK_PARALLEL["tracks"],
+                          (lambda t: dist.all_reduce(t)) if TRACK_PARALLEL["world"] > 1 else (lambda t: None))
+    else:
+        m.init_random(seed=wl.seed)
     return m
 
 
@@ -431,6 +443,10 @@ def main():
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--extra", default="cfg3", help="comma-separated workloads reported under 'extra' (N=1 only); '' for none")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--parallel", default="replicas", choices=["replicas", "tracks"],
+                    help="N > 1: 'replicas' = every rank runs the whole model on its own batch (weak scaling, no collective); "
+                         "'tracks' = every rank holds T/N tracks of one model and all ranks share the batch (strong scaling, "
+                         "one all-reduce per track block)")
     ap.add_argument("--seq", type=int, default=0, help="override the workload's sequence / KV length")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch")
     ap.add_argument("--depth", type=int, default=0, help="override the track-block depth D (must divide L)")
@@ -479,11 +495,22 @@ def main():
         torch.cuda.synchronize()
 
     run = run_decode if wl.mode == "decode" else run_prefill
-    r = run(wl, dev, a.steps, a.warmup, barrier, rank)
-    ms, total_tokens, e2e_value = aggregate_over_ranks(r["ms"], r["tokens"], r["e2e"]["value"], world, dev)
+    tracks_mode = a.parallel == "tracks"
+    if tracks_mode:
+        # one model over all ranks: each holds T / N tracks, all see the same batch (same input seed),
+        # so the job's tokens are one rank's and the step time is the slowest rank's
+        assert wl.T % world == 0, "the number of ranks must divide the number of tracks"
+        TRACK_PARALLEL.update(on=True, world=world, rank=rank, tracks=wl.T)
+        r = run(dataclasses.replace(wl, T=wl.T // world), dev, a.steps, a.warmup, barrier, 0)
+        ms, _, e2e_value = aggregate_over_ranks(r["ms"], r["tokens"], r["e2e"]["value"], world, dev)
+        total_tokens, e2e_value = float(r["tokens"]), e2e_value / world
+        r["config"]["parallelism"] = f"tracks: {wl.T} tracks over {world} rank(s), one all-reduce per track block"
+    else:
+        r = run(wl, dev, a.steps, a.warmup, barrier, rank)
+        ms, total_tokens, e2e_value = aggregate_over_ranks(r["ms"], r["tokens"], r["e2e"]["value"], world, dev)
     r["e2e"]["value"] = e2e_value
     extra = {}
-    if world == 1 and a.extra:
+    if world == 1 and a.extra and not tracks_mode:
         for name in [n for n in a.extra.split(",") if n and n != a.workload]:
             w2 = I.WORKLOADS[name]
             try:
@@ -500,7 +527,8 @@ def main():
         cpu = {"value": v, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample, "seconds": round(dt, 2)}
     if rank == 0:
         line = {"metric": f"PT {metric} on B200", "value": total_tokens / (ms * 1e-3), "unit": "tokens/s", "n_gpus": world,
-                "steps": a.steps, "warmup": a.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+                "steps": a.steps, "warmup": a.warmup, "ms_per_step": ms, "higher_is_better": True,
+                "scaling": "strong" if tracks_mode else "weak",
                 "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
                 "config": r["config"], "clocks": r["clocks"], "e2e": r["e2e"], "gpu_launches": int(r["launches"]),
                 "roofline": r["roofline"], "cpu_baseline": cpu, "kernels_ms_per_step": r["kernels_ms_per_step"],

@@ -39,11 +39,12 @@ __global__ void k_tc_prep(const __nv_bfloat16* __restrict__ x, int64_t x_stride,
     }
 }
 
-// Track-sync of a small batch (decode): h = scale * sum_t h_t in track order, the synced stream, every
-// track's gain-scaled bf16 operand for the next layer and the partial sums of squares.  One warp per row.
+// Track-sync outside a GEMM epilogue: h = scale * sum of T input streams in order, the synced stream, the
+// gain-scaled bf16 operand of each of the T_out tracks that continue from it and the partial sums of
+// squares.  One warp per row.  Used for a decode step's few rows and after the all-reduce of a track group.
 // (With few rows the K-concatenated sync GEMM would run on N/128 CTAs only; the per-track down GEMM fills
 // the machine and this kernel finishes the reduction.)
-__global__ void k_track_sync(const float* __restrict__ hT, size_t tstride, int T, float scale,
+__global__ void k_track_sync(const float* __restrict__ hT, size_t tstride, int T, int T_out, float scale,
                              float* __restrict__ h_out, __nv_bfloat16* __restrict__ hb, const float* __restrict__ gain,
                              float* __restrict__ ssq, int M, int H, int tiles) {
     int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
@@ -62,7 +63,7 @@ __global__ void k_track_sync(const float* __restrict__ hT, size_t tstride, int T
             *reinterpret_cast<float4*>(h_out + ro + c) = a;
             s = a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
             if (hb) {
-                for (int t = 0; t < T; ++t) {
+                for (int t = 0; t < T_out; ++t) {
                     float4 gn = *reinterpret_cast<const float4*>(gain + (size_t)t * H + c);
                     __nv_bfloat162 o0 = __floats2bfloat162_rn(a.x * gn.x, a.y * gn.y), o1 = __floats2bfloat162_rn(a.z * gn.z, a.w * gn.w);
                     uint2 ov;
@@ -212,7 +213,7 @@ pt_status tc_forward(Call& k) {
             float* ssq_next = last ? nullptr : w.ssq;
             const unsigned sync_grid = (unsigned)((M * 32 + 255) / 256);
             if (split_sync) {       // local tracks -> one stream (the final one unless other ranks still have to join)
-                k_track_sync<<<sync_grid, 256, 0, st>>>(w.hT, MH, T, grouped ? 1.0f : sync_scale, grouped ? w.hS : ho,
+                k_track_sync<<<sync_grid, 256, 0, st>>>(w.hT, MH, T, T, grouped ? 1.0f : sync_scale, grouped ? w.hS : ho,
                                                         grouped ? nullptr : hb_next, grouped ? nullptr : gain_next,
                                                         grouped ? nullptr : ssq_next, M, H, tiles);
                 g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -221,7 +222,7 @@ pt_status tc_forward(Call& k) {
                 // w.hS holds this rank's partial sum: one all-reduce per track block, then every local track's
                 // next operand from the total
                 if (m->ar_fn(m->ar_user, w.hS, (int64_t)M * H, (void*)st) != 0) { set_error("the all-reduce hook failed at layer %d", l); return PT_ERR_CUDA; }
-                k_track_sync<<<sync_grid, 256, 0, st>>>(w.hS, 0, 1, sync_scale, ho, hb_next, gain_next, ssq_next, M, H, tiles);
+                k_track_sync<<<sync_grid, 256, 0, st>>>(w.hS, 0, 1, T, sync_scale, ho, hb_next, gain_next, ssq_next, M, H, tiles);
                 g_launches.fetch_add(1, std::memory_order_relaxed);
             }
             if (sync) { ssq_tstride = 0; hin = ho; hin_stride = 0; }

@@ -24,7 +24,7 @@ class _Tracks:
 
 def _full_and_inputs(sync_op, L=4, D=2):
     wl = I.Workload("tp", T=4, L=L, D=D, hidden=256, heads=4, kv_heads=2, ffn=352, dtype="bf16", mode="prefill", batch=2, seq=300)
-    ws = I.WeightSource(wl, std=0.05, gain_jitter=0.1)
+    ws = I.WeightSource(wl, gain_jitter=0.1)
     x = I.prefill_inputs(wl)
     xd = I.decode_inputs(wl)
     return wl, ws, x, xd
@@ -51,8 +51,11 @@ def test_one_rank_with_identity_hook_equals_the_plain_schedule_and_syncs_L_over_
     # one all-reduce per track block: L/D per forward, against 2L for tensor parallelism
     assert n_prefill == wl.L // wl.D and len(calls) == 2 * (wl.L // wl.D)
     assert calls[0] == 2 * 300 * wl.hidden and calls[-1] == 2 * wl.hidden
+    # the two schedules add the partial sums of squares in a different order, which moves a few bf16
+    # roundings of the next layer's operands: equal to well inside the bf16 bounds, not bit for bit
     for a, b in zip(outs[0], outs[1]):
-        assert np.allclose(a, b, rtol=1e-6, atol=1e-6 * np.abs(a).max())
+        mx, mean = Hp.rel_errs(a, b)
+        assert mx <= 1e-2 and mean <= 2.5e-3, (mx, mean)
 
 
 @pytest.mark.parametrize("sync_op", ["sum", "mean"])
@@ -104,9 +107,17 @@ def test_two_ranks_holding_half_the_tracks_each_match_the_single_model(sync_op):
     for rank in range(2):
         p, d = results[rank]
         # the ranks add (t0 + t1) + (t2 + t3), the single model ((t0 + t1) + t2) + t3: fp32 rounding only
-        assert np.allclose(p, want_p, rtol=0, atol=2e-5 * np.abs(want_p).max()), np.abs(p - want_p).max() / np.abs(want_p).max()
-        assert np.allclose(d, want_d, rtol=0, atol=2e-5 * np.abs(want_d).max())
+        # (and a few bf16 roundings downstream of it, as above)
+        for got, want in ((p, want_p), (d, want_d)):
+            mx, mean = Hp.rel_errs(got, want)
+            assert mx <= 1e-2 and mean <= 2.5e-3, (rank, mx, mean)
     assert np.array_equal(results[0][0], results[1][0]) and np.array_equal(results[0][1], results[1][1])
+    # and the two-rank result stands on its own against the oracle
+    from oracle import pt_oracle as O
+    cfg = Hp.oracle_cfg(wl, sync_op)
+    ocache = O.PagedKVCache(cfg, 40, 16)
+    Hp.assert_close(results[0][0], O.pt_prefill(cfg, ws, x, ocache, [0, 1]), "bf16", "two-rank prefill")
+    Hp.assert_close(results[0][1], O.pt_decode_step(cfg, ws, xd, ocache, [0, 1]), "bf16", "two-rank decode")
 
 
 def test_nccl_all_reduce_as_the_hook_on_a_single_rank_group():
@@ -132,7 +143,8 @@ def test_nccl_all_reduce_as_the_hook_on_a_single_rank_group():
         got = m.prefill(c, Hp.to_dev(m, x), [0, 1]).cpu().numpy()
         torch.cuda.synchronize()
         assert m.device_status() == (0, 0)
-        assert np.allclose(got, want, rtol=1e-6, atol=1e-6 * np.abs(want).max())
+        mx, mean = Hp.rel_errs(got, want)
+        assert mx <= 1e-2 and mean <= 2.5e-3, (mx, mean)
         m.close()
     finally:
         dist.destroy_process_group()
