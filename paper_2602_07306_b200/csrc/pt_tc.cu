@@ -41,44 +41,48 @@ __global__ void k_tc_prep(const __nv_bfloat16* __restrict__ x, int64_t x_stride,
 
 // Track-sync outside a GEMM epilogue: h = scale * sum of T input streams in order, the synced stream, the
 // gain-scaled bf16 operand of each of the T_out tracks that continue from it and the partial sums of
-// squares.  One warp per row.  Used for a decode step's few rows and after the all-reduce of a track group.
-// (With few rows the K-concatenated sync GEMM would run on N/128 CTAs only; the per-track down GEMM fills
-// the machine and this kernel finishes the reduction.)
+// squares.  One warp per (row, 128-column group), so a single decoded row still spreads over H / 128 warps.
+// Used for a decode step's few rows and after the all-reduce of a track group.  (With few rows the
+// K-concatenated sync GEMM would run on N/128 CTAs only; the per-track down GEMM fills the machine and this
+// kernel finishes the reduction.)
 __global__ void k_track_sync(const float* __restrict__ hT, size_t tstride, int T, int T_out, float scale,
                              float* __restrict__ h_out, __nv_bfloat16* __restrict__ hb, const float* __restrict__ gain,
                              float* __restrict__ ssq, int M, int H, int tiles) {
-    int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-    if (warp >= M) return;
-    size_t ro = (size_t)warp * H;
-    for (int g = 0; g * 128 < H; ++g) {
-        int c = g * 128 + lane * 4;
-        float s = 0.f;
-        if (c < H) {
-            float4 a = *reinterpret_cast<const float4*>(hT + ro + c);
-            for (int t = 1; t < T; ++t) {
-                float4 b = *reinterpret_cast<const float4*>(hT + (size_t)t * tstride + ro + c);
-                a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
-            }
-            a.x *= scale; a.y *= scale; a.z *= scale; a.w *= scale;
-            *reinterpret_cast<float4*>(h_out + ro + c) = a;
-            s = a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
-            if (hb) {
-                for (int t = 0; t < T_out; ++t) {
-                    float4 gn = *reinterpret_cast<const float4*>(gain + (size_t)t * H + c);
-                    __nv_bfloat162 o0 = __floats2bfloat162_rn(a.x * gn.x, a.y * gn.y), o1 = __floats2bfloat162_rn(a.z * gn.z, a.w * gn.w);
-                    uint2 ov;
-                    ov.x = *reinterpret_cast<uint32_t*>(&o0); ov.y = *reinterpret_cast<uint32_t*>(&o1);
-                    *reinterpret_cast<uint2*>(hb + (size_t)t * M * H + ro + c) = ov;
-                }
+    const int groups = (H + 127) / 128;
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (warp >= M * groups) return;
+    const int row = warp / groups, g = warp % groups;
+    const size_t ro = (size_t)row * H;
+    const int c = g * 128 + lane * 4;
+    float s = 0.f;
+    if (c < H) {
+        float4 a = *reinterpret_cast<const float4*>(hT + ro + c);
+#pragma unroll 4
+        for (int t = 1; t < T; ++t) {
+            float4 b = *reinterpret_cast<const float4*>(hT + (size_t)t * tstride + ro + c);
+            a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+        }
+        a.x *= scale; a.y *= scale; a.z *= scale; a.w *= scale;
+        *reinterpret_cast<float4*>(h_out + ro + c) = a;
+        s = a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
+        if (hb) {
+            for (int t = 0; t < T_out; ++t) {
+                float4 gn = *reinterpret_cast<const float4*>(gain + (size_t)t * H + c);
+                __nv_bfloat162 o0 = __floats2bfloat162_rn(a.x * gn.x, a.y * gn.y), o1 = __floats2bfloat162_rn(a.z * gn.z, a.w * gn.w);
+                uint2 ov;
+                ov.x = *reinterpret_cast<uint32_t*>(&o0); ov.y = *reinterpret_cast<uint32_t*>(&o1);
+                *reinterpret_cast<uint2*>(hb + (size_t)t * M * H + ro + c) = ov;
             }
         }
-        for (int o = 8; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-        int tile = g * 2 + (lane >> 4);
-        if (ssq && (lane & 15) == 0 && tile < tiles) ssq[(size_t)warp * tiles + tile] = s;
     }
+    for (int o = 8; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    const int tile = g * 2 + (lane >> 4);
+    if (ssq && (lane & 15) == 0 && tile < tiles) ssq[(size_t)row * tiles + tile] = s;
 }
 
-struct WMaps { CUtensorMap m[4][3]; };   // [qkv, o, gu, d][bn 64, 128, 256]
+// [qkv, o, gu, d][bn 64, 128, 256][k-blocks per copy 1, 2, 4]; combinations gemm_kps never picks stay unset
+struct WMaps { CUtensorMap m[4][3][3]; };
+inline int kps_index(int kps) { return kps == 4 ? 2 : (kps == 2 ? 1 : 0); }
 
 }  // namespace
 
@@ -93,14 +97,19 @@ pt_status tc_build_weight_maps(pt_model* m) {
     const __nv_bfloat16* wgu = (const __nv_bfloat16*)(m->wbuf + m->off_wgu);
     const __nv_bfloat16* wd = (const __nv_bfloat16*)(m->wbuf + m->off_wd);
     for (int l = 0; l < c.L; ++l)
-        for (int b = 0; b < 3; ++b) {
-            int bn = 64 << b;
-            pt_status s;
-            if ((s = make_map_bf16(&v[l].m[0][b], wqkv + (size_t)l * m->wqkv_layer(), c.hidden, m->Nqkv, c.T, bn)) != PT_OK) return s;
-            if ((s = make_map_bf16(&v[l].m[1][b], wo + (size_t)l * m->wo_layer(), m->QD, c.hidden, c.T, bn)) != PT_OK) return s;
-            if ((s = make_map_bf16(&v[l].m[2][b], wgu + (size_t)l * m->wgu_layer(), c.hidden, 2 * c.ffn, c.T, bn)) != PT_OK) return s;
-            if ((s = make_map_bf16(&v[l].m[3][b], wd + (size_t)l * m->wd_layer(), c.ffn, c.hidden, c.T, bn)) != PT_OK) return s;
-        }
+        for (int b = 0; b < 3; ++b)
+            for (int kp = 0; kp < 3; ++kp) {
+                const int bn = 64 << b, kps = 1 << kp;
+                if (bn * kps > 256) continue;
+                const void* base[4] = {wqkv + (size_t)l * m->wqkv_layer(), wo + (size_t)l * m->wo_layer(),
+                                       wgu + (size_t)l * m->wgu_layer(), wd + (size_t)l * m->wd_layer()};
+                const int64_t kk[4] = {c.hidden, m->QD, c.hidden, c.ffn}, nn[4] = {m->Nqkv, c.hidden, 2 * c.ffn, c.hidden};
+                for (int i = 0; i < 4; ++i) {
+                    if (kps > 1 && (kk[i] % 64 || (kk[i] / 64) % kps)) continue;
+                    pt_status s = make_w_map(&v[l].m[i][b][kp], base[i], kk[i], nn[i], c.T, bn, kps);
+                    if (s != PT_OK) return s;
+                }
+            }
     g_wmaps[m] = std::move(v);
     return PT_OK;
 }
@@ -143,7 +152,7 @@ pt_status tc_forward(Call& k) {
         __nv_bfloat16* pool_l = pool + (size_t)l * c->slab_elems;
         GemmP base{};
         base.M = M; base.status = m->status(); base.eps = g.rms_eps; base.kt = 1; base.T = T;
-        base.scale = 1.0f; base.n_sum = 1; base.n_out = 1;
+        base.scale = 1.0f; base.n_sum = 1; base.n_out = 1; base.w_static = 1;
         {   // QKV: RMSNorm-1 scale, RoPE, KV append
             GemmP p = base;
             p.N = m->Nqkv; p.K = H;
@@ -152,8 +161,9 @@ pt_status tc_forward(Call& k) {
             p.row_kvoff = w.meta.row_kvoff; p.row_pos = w.meta.row_pos; p.cs = m->rope_cos(); p.sn = m->rope_sin(); p.cs16 = m->rope_cs16();
             p.nq = g.heads; p.nkv = g.kv_heads; p.dh = m->dh; p.ps = c->ps;
             int bn = gemm_bn(p.N, M, T, EPI_QKV);
+            p.kps = gemm_kps(bn, M, p.K, 1);
             ProfScope ps(m, st, 1);
-            if ((s = launch_gemm(EPI_QKV, bn, ta_h, wm[l].m[0][bn_index(bn)], p, st)) != PT_OK) return s;
+            if ((s = launch_gemm(EPI_QKV, bn, ta_h, wm[l].m[0][bn_index(bn)][kps_index(p.kps)], p, st)) != PT_OK) return s;
         }
         {
             ProfScope ps(m, st, 0);
@@ -168,8 +178,9 @@ pt_status tc_forward(Call& k) {
             p.hb_out = hb; p.gain = m->gain(1, l);
             p.ssq_out = w.ssq; p.ssq_out_tstride = (size_t)M * tiles; p.ssq_out_tiles = tiles;
             int bn = gemm_bn(p.N, M, T, EPI_RESID);
+            p.kps = gemm_kps(bn, M, p.K, 1);
             ProfScope ps(m, st, 2);
-            if ((s = launch_gemm(EPI_RESID, bn, ta_o, wm[l].m[1][bn_index(bn)], p, st)) != PT_OK) return s;
+            if ((s = launch_gemm(EPI_RESID, bn, ta_o, wm[l].m[1][bn_index(bn)][kps_index(p.kps)], p, st)) != PT_OK) return s;
             ssq_tstride = (size_t)M * tiles;
         }
         tap_copy(k, l, 0, w.hT, MH);
@@ -179,8 +190,9 @@ pt_status tc_forward(Call& k) {
             p.ssq_in = w.ssq; p.ssq_in_tstride = ssq_tstride; p.ssq_tiles = tiles;
             p.z_out = z;
             int bn = gemm_bn(p.N, M, T, EPI_SWIGLU);
+            p.kps = gemm_kps(bn, M, p.K, 1);
             ProfScope ps(m, st, 3);
-            if ((s = launch_gemm(EPI_SWIGLU, bn, ta_h, wm[l].m[2][bn_index(bn)], p, st)) != PT_OK) return s;
+            if ((s = launch_gemm(EPI_SWIGLU, bn, ta_h, wm[l].m[2][bn_index(bn)][kps_index(p.kps)], p, st)) != PT_OK) return s;
         }
         {   // down projection + residual (+ track-sync when the layer closes a track block)
             const bool sync = (l + 1) % g.D == 0, last = l + 1 == g.L;
@@ -205,13 +217,14 @@ pt_status tc_forward(Call& k) {
                 if (split_sync) { p.hb_out = nullptr; p.ssq_out = nullptr; }
             }
             int bn = gemm_bn(p.N, M, p.T, EPI_RESID);
+            p.kps = gemm_kps(bn, M, p.K, p.kt);
             ProfScope ps(m, st, sync ? 5 : 4);
-            if ((s = launch_gemm(EPI_RESID, bn, ta_z, wm[l].m[3][bn_index(bn)], p, st)) != PT_OK) return s;
+            if ((s = launch_gemm(EPI_RESID, bn, ta_z, wm[l].m[3][bn_index(bn)][kps_index(p.kps)], p, st)) != PT_OK) return s;
             float* ho = last ? k.out : w.hS;
             __nv_bfloat16* hb_next = last ? nullptr : hb;
             const float* gain_next = last ? nullptr : m->gain(0, l + 1);
             float* ssq_next = last ? nullptr : w.ssq;
-            const unsigned sync_grid = (unsigned)((M * 32 + 255) / 256);
+            const unsigned sync_grid = (unsigned)(((size_t)M * ((H + 127) / 128) * 32 + 255) / 256);
             if (split_sync) {       // local tracks -> one stream (the final one unless other ranks still have to join)
                 k_track_sync<<<sync_grid, 256, 0, st>>>(w.hT, MH, T, T, grouped ? 1.0f : sync_scale, grouped ? w.hS : ho,
                                                         grouped ? nullptr : hb_next, grouped ? nullptr : gain_next,
@@ -249,9 +262,10 @@ extern "C" pt_status pt_kernel_gemm_bf16(const void* a, const void* w, void* c, 
     CUtensorMap ta, tb;
     pt_status s;
     if ((s = make_map_bf16(&ta, a, K, M, T, 128)) != PT_OK) return s;
-    if ((s = make_map_bf16(&tb, w, K, N, T, bn)) != PT_OK) return s;
+    const int kps = gemm_kps(bn, M, K, fold_tracks ? T : 1);
+    if ((s = make_w_map(&tb, w, K, N, T, bn, kps)) != PT_OK) return s;
     GemmP p{};
-    p.M = M; p.N = N; p.K = K; p.T = fold_tracks ? 1 : T; p.kt = fold_tracks ? T : 1;
+    p.M = M; p.N = N; p.K = K; p.T = fold_tracks ? 1 : T; p.kt = fold_tracks ? T : 1; p.kps = kps;
     p.status = (int*)status; p.c_out = (float*)c; p.scale = 1.f; p.n_sum = 1; p.n_out = 1;
     if ((s = launch_gemm(EPI_PLAIN, bn, ta, tb, p, (cudaStream_t)stream)) != PT_OK) return s;
     cudaError_t e = cudaGetLastError();

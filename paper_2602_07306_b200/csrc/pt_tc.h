@@ -2,6 +2,7 @@
 // decode attention).
 #pragma once
 #include <algorithm>
+#include <utility>
 #include "pt_internal.h"
 
 namespace pt {
@@ -14,7 +15,13 @@ struct GemmP {
     int T;                  // tracks folded into the grid
     int kt;                 // tracks folded into the K loop (1, or all tracks for the sync GEMM with T = 1)
     int tiles_m, tiles_n;   // filled by the launcher
-    uint32_t tx_bytes;      // bytes one stage's two TMA loads deliver (filled by the launcher)
+    int kps;                // k-blocks per ring stage (1, or 2 / 4 with a 4-D W map from make_w_map; see gemm_kps)
+    // filled by the launcher:
+    uint32_t a_tx, w_tx;    // bytes one A copy and the stage's W copy deliver
+    uint32_t a_bytes;       // shared-memory bytes reserved per k-block of A; the stage's W part follows its kps A pieces
+    uint32_t w_kb_bytes;    // shared-memory bytes one k-block of W takes
+    int stages;             // ring depth
+    int w_static;           // W is written by no kernel of the stream: its first tiles may be fetched before grid_dep_wait()
     int* status;
     // RMSNorm applied as a per-row scale: rinv = rsqrt(sum(ssq_in[row][:]) / K + eps)
     const float* ssq_in; size_t ssq_in_tstride; int ssq_tiles; float eps;
@@ -54,6 +61,34 @@ struct AttnP {
     const int32_t* items; const int32_t* nsplit; float* part; int max_splits;
 };
 
+// Programmatic dependent launch.  A kernel launched with launch_dependent() may start while the
+// kernel before it in the stream is still running: its blocks get free SMs as the earlier kernel's
+// blocks retire, and run until grid_dep_wait(), which returns once the earlier kernel has completed
+// and its writes are visible.  Before that wait a kernel may only touch memory that no kernel of the
+// stream writes (weights); everything else, reads and writes, comes after it.  Every block calls
+// grid_dep_wait() and only then grid_dep_launch(), so at most two kernels overlap and a kernel past
+// its wait sees the results of every launch before it.  In a kernel launched the ordinary way both
+// calls do nothing.
+#ifdef __CUDACC__
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+#endif
+
 pt_status launch_flash_prefill_p(const AttnP& p, int T, int dh, bool legacy, cudaStream_t st);
 pt_status launch_decode_attn_p(const AttnP& p, int T, int dh, int n_items, int max_splits, cudaStream_t st);
 
@@ -61,6 +96,10 @@ pt_status make_map_bf16(CUtensorMap* out, const void* base, int64_t k, int64_t r
 pt_status make_map_bf16_strided(CUtensorMap* out, const void* base, int64_t k, int64_t rows, int64_t tracks,
                                 int64_t track_stride_bytes, int box_rows);
 int gemm_bn(int N, int M, int T, int epi);
+// k-blocks per ring stage for a launch of M rows: more than one when the rows are few, so that a copy of W is 16-32 KB
+int gemm_kps(int bn, int M, int K, int kt);
+// tensor map of W [tracks][rows][k] for tiles of bn rows: 3-D (k, row, track) for kps = 1, else 4-D (64, row, k-block, track)
+pt_status make_w_map(CUtensorMap* out, const void* base, int64_t k, int64_t rows, int64_t tracks, int bn, int kps);
 inline int bn_index(int bn) { return bn == 64 ? 0 : (bn == 128 ? 1 : 2); }
 pt_status launch_gemm(int epi, int bn, const CUtensorMap& ta, const CUtensorMap& tb, GemmP p, cudaStream_t st);
 

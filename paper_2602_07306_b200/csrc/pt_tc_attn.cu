@@ -326,6 +326,8 @@ k_decode_attn_tma(const __grid_constant__ CUtensorMap kvmap, const AttnP p) {
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint64_t* bars = (uint64_t*)(smem + 4 * kDecStages * SLOT_BYTES);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    grid_dep_wait();                                          // q and this step's K/V rows come from the QKV GEMM before it
+    grid_dep_launch();
     const int32_t* item = p.items + (size_t)blockIdx.x * 4;
     const int b = item[0], kstart = item[1], kcount = item[2], split = item[3];
     const int kvh = blockIdx.y, t = blockIdx.z;
@@ -542,6 +544,8 @@ k_decode_attn(const AttnP p) {
 // Merge the key ranges of one (track, sequence, head): one warp each.
 template <int DH>
 __global__ void k_decode_combine(const AttnP p) {
+    grid_dep_wait();
+    grid_dep_launch();
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     const int t = blockIdx.y;
     if (warp >= p.B * p.nq) return;
@@ -615,8 +619,9 @@ pt_status launch_decode_attn_p(const AttnP& p, int T, int dh, int n_items, int m
         if (s != PT_OK) return s;
         const int smem = 1024 + 4 * kDecStages * 2 * 16 * dh * 2 + 4 * kDecStages * 8;
 #define GOT(DH_) { static bool done = false; if (!done) { if ((s = set_smem(k_decode_attn_tma<DH_>, smem)) != PT_OK) return s; done = true; } \
-                   k_decode_attn_tma<DH_><<<grid, kThreads, smem, st>>>(kvmap, p); \
-                   if (max_splits > 1) { k_decode_combine<DH_><<<dim3((p.B * p.nq * 32 + 127) / 128, T), 128, 0, st>>>(p); g_launches.fetch_add(1, std::memory_order_relaxed); } }
+                   launch_dependent(k_decode_attn_tma<DH_>, grid, dim3(kThreads), (size_t)smem, st, kvmap, p); \
+                   if (max_splits > 1) { launch_dependent(k_decode_combine<DH_>, dim3((p.B * p.nq * 32 + 127) / 128, T), dim3(128), (size_t)0, st, p); \
+                                         g_launches.fetch_add(1, std::memory_order_relaxed); } }
         if (dh == 64) GOT(64) else GOT(128)
 #undef GOT
         g_launches.fetch_add(1, std::memory_order_relaxed);

@@ -61,6 +61,11 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, u
                  ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar)) : "memory");
 }
 
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2, int c3) {
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+                 ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(bar)) : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -103,14 +108,28 @@ __device__ __forceinline__ void report(int* status, int code, int loc) {
     if (atomicCAS(status, 0, code) == 0) status[1] = loc;
 }
 
+// Shared memory of a CTA: a ring of stages, each one k-block of A (the launch's row box: min(M, 128)
+// rows, rounded up to the 1024-byte swizzle atom) followed by one of W (BN rows).  The fewer rows a
+// launch has, the more stages fit, so a decode step (few rows, weights streamed once) keeps more
+// bytes of W in flight per SM.  tcgen05.mma always reads 128 rows of A from a stage: rows past the box
+// belong to the stages behind it (or to the slack after the last stage) and only feed accumulator rows
+// that nobody stores.  With few rows a stage holds kps k-blocks (A pieces first, then W) and W arrives
+// as one copy of kps k-blocks (a 4-D view of W: 64 columns, rows, k-blocks, tracks): a copy occupies the
+// SM's TMA unit for about a memory latency whatever its size, so W streams from HBM at full rate only
+// with 16 KB or more per copy.
+constexpr int kMaxStages = 24;
+constexpr int kRingBytes = 216 * 1024;                       // stages + the slack behind the last one
+constexpr int kBarBytes = 512;                               // 2 * kMaxStages + 4 mbarriers, TMEM slot, abort flag
+constexpr int kGemmSmem = kRingBytes + 1024 /*alignment*/ + kBarBytes;
+constexpr int kFullA = BM * BK * 2;
+
 template <int BN> struct Cfg {
-    static constexpr int STAGES = BN == 256 ? 4 : (BN == 128 ? 6 : 8);
-    static constexpr int A_BYTES = BM * BK * 2;
     static constexpr int B_BYTES = BN * BK * 2;
-    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int RING_BYTES = STAGES * STAGE_BYTES;
-    static constexpr int SMEM = RING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
+inline int stage_a_bytes(int M) { return (std::min(M, BM) * BK * 2 + 1023) / 1024 * 1024; }
+inline int ring_stages(int a_bytes, int b_bytes, int kps) {
+    return std::min(kMaxStages, (kRingBytes - (kFullA - a_bytes)) / (kps * (a_bytes + b_bytes)));
+}
 
 // ---- epilogue ------------------------------------------------------------------------------
 // tcgen05.ld hands every thread one accumulator row (row0 + lane); a warp works through its share
@@ -374,22 +393,33 @@ __device__ __forceinline__ bool epilogue(const GemmP& p, uint32_t taddr, int t, 
     else return epi_resid<BN>(p, taddr, t, row, row_ok, n0, half, wait);
 }
 
+// Tile index -> (column tile, row tile, track).  With one or two row tiles (a decode step) the row
+// tile runs fastest, so the CTAs that stream the same W tile are neighbours in time and the second one
+// finds it in L2; with many row tiles the column tile runs fastest and neighbours share their A tile.
+__device__ __forceinline__ void tile_coords(const GemmP& p, int tile, int& nt, int& mt, int& t) {
+    if (p.tiles_m <= 2) { mt = tile % p.tiles_m; nt = (tile / p.tiles_m) % p.tiles_n; }
+    else { nt = tile % p.tiles_n; mt = (tile / p.tiles_n) % p.tiles_m; }
+    t = tile / (p.tiles_n * p.tiles_m);
+}
+
 template <int BN, int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_tc(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensorMap tb, const GemmP p) {
     using C = Cfg<BN>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint64_t* full = (uint64_t*)(smem + C::RING_BYTES);
-    uint64_t* empty = full + C::STAGES;
-    uint64_t* acc_full = empty + C::STAGES;
+    uint64_t* full = (uint64_t*)(smem + kRingBytes);
+    uint64_t* empty = full + kMaxStages;
+    uint64_t* acc_full = empty + kMaxStages;
     uint64_t* acc_empty = acc_full + 2;
     uint32_t* tmem_slot = (uint32_t*)(acc_empty + 2);
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+    const int stages = p.stages, kps = p.kps;
+    const uint32_t a_bytes = p.a_bytes, w_off = kps * p.a_bytes, stage_bytes = kps * (p.a_bytes + C::B_BYTES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < C::STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int s = 0; s < stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], kEpiWarps); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -407,28 +437,72 @@ gemm_tc(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensor
     const int num_tiles = p.tiles_m * p.tiles_n * p.T;
     const int kpb = (p.K + BK - 1) / BK;            // k-blocks per track
     const int kblocks = kpb * p.kt;
+    const int nsteps = kblocks / kps;                // ring stages one tile consumes (kps divides kblocks)
+    const uint32_t stage_tx = kps * p.a_tx + p.w_tx;
 
     if (warp == 0) {
         if (lane == 0) {
+            // Model weights are written by no kernel, so the first ring generation of W tiles is requested
+            // before the wait for the previous kernel: their stream is under way when its results arrive.
+            int npre = 0;
+            auto load_w = [&](int s, int it, int nt, int t) {
+                uint8_t* sw = smem + s * stage_bytes + w_off;
+                if (kps > 1) tma_load_4d(sw, &tb, &full[s], 0, nt * BN, it * kps, t);        // kps k-blocks in one copy
+                else tma_load_3d(sw, &tb, &full[s], (p.kt > 1 ? it % kpb : it) * BK, nt * BN, p.kt > 1 ? it / kpb : t);
+            };
+            if (p.w_static && (int)blockIdx.x < num_tiles) {
+                int nt, mt, t;
+                tile_coords(p, blockIdx.x, nt, mt, t);
+                npre = min(stages, nsteps);
+                for (int it = 0; it < npre; ++it) {
+                    mbar_expect_tx(&full[it], stage_tx);
+                    load_w(it, it, nt, t);
+                }
+            }
+            grid_dep_wait();
+            grid_dep_launch();
             int s = 0; uint32_t ph = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                int nt = tile % p.tiles_n, mt = (tile / p.tiles_n) % p.tiles_m, t = tile / (p.tiles_n * p.tiles_m);
-                for (int kb = 0; kb < kblocks; ++kb) {
-                    if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_EMPTY_WAIT); *abort_flag = 1; break; }
-                    int tt = p.kt > 1 ? kb / kpb : t;
-                    int k0 = (p.kt > 1 ? kb % kpb : kb) * BK;
-                    uint8_t* sa = smem + s * C::STAGE_BYTES;
-                    mbar_expect_tx(&full[s], p.tx_bytes);
-                    tma_load_3d(sa, &ta, &full[s], k0, mt * BM, tt);
-                    tma_load_3d(sa + C::A_BYTES, &tb, &full[s], k0, nt * BN, tt);
-                    if (++s == C::STAGES) { s = 0; ph ^= 1; }
+                int nt, mt, t;
+                tile_coords(p, tile, nt, mt, t);
+                if (kps == 1) {
+                    for (int kb = 0; kb < kblocks; ++kb) {
+                        const int tt = p.kt > 1 ? kb / kpb : t;
+                        const int k0 = (p.kt > 1 ? kb % kpb : kb) * BK;
+                        uint8_t* sa = smem + s * stage_bytes;
+                        if (kb < npre) {                               // the stage is armed and its W copy on the way
+                            tma_load_3d(sa, &ta, &full[s], k0, mt * BM, tt);
+                        } else {
+                            if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_EMPTY_WAIT); *abort_flag = 1; break; }
+                            mbar_expect_tx(&full[s], stage_tx);
+                            tma_load_3d(sa, &ta, &full[s], k0, mt * BM, tt);
+                            tma_load_3d(sa + a_bytes, &tb, &full[s], k0, nt * BN, tt);
+                        }
+                        if (++s == stages) { s = 0; ph ^= 1; }
+                    }
+                } else {
+                    for (int it = 0; it < nsteps; ++it) {
+                        if (it >= npre) {
+                            if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_EMPTY_WAIT); *abort_flag = 1; break; }
+                            mbar_expect_tx(&full[s], stage_tx);
+                        }
+                        uint8_t* sa = smem + s * stage_bytes;
+                        for (int j = 0; j < kps; ++j)
+                            tma_load_3d(sa + j * a_bytes, &ta, &full[s], (it * kps + j) * BK, mt * BM, t);
+                        if (it >= npre) load_w(s, it, nt, t);
+                        if (++s == stages) { s = 0; ph ^= 1; }
+                    }
                 }
+                npre = 0;
             }
+        } else {
+            grid_dep_wait();
         }
         __syncwarp();
     } else if (warp == 1) {
         // whole warp walks the loop; the tcgen05 instructions run on one elected lane
+        grid_dep_wait();
         constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
         const uint64_t desc0 = smem_desc(smem_u32(smem));
         int s = 0; uint32_t ph = 0;
@@ -441,19 +515,41 @@ gemm_tc(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensor
             }
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + a * BN;
-            for (int kb = 0; kb < kblocks; ++kb) {
-                if (!__all_sync(0xffffffffu, mbar_wait(&full[s], ph, abort_flag))) {
-                    ok = false;
-                    if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_TMA_WAIT); *abort_flag = 1; }
-                    break;
-                }
-                tc_fence_after();
-                const uint64_t da = desc0 + (uint64_t)((s * C::STAGE_BYTES) >> 4), db = da + (uint64_t)(C::A_BYTES >> 4);
+            if (kps == 1) {
+                // one k-block per stage (every launch with many rows): the loop that bounds the tensor pipe
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!__all_sync(0xffffffffu, mbar_wait(&full[s], ph, abort_flag))) {
+                        ok = false;
+                        if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_TMA_WAIT); *abort_flag = 1; }
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint64_t da = desc0 + (uint64_t)((s * stage_bytes) >> 4), db = da + (uint64_t)(a_bytes >> 4);
 #pragma unroll
-                for (int k = 0; k < BK / 16; ++k)
-                    tc_mma(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
-                tc_commit(&empty[s]);                     // frees the stage when these MMAs retire
-                if (++s == C::STAGES) { s = 0; ph ^= 1; }
+                    for (int k = 0; k < BK / 16; ++k)
+                        tc_mma(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+                    tc_commit(&empty[s]);                     // frees the stage when these MMAs retire
+                    if (++s == stages) { s = 0; ph ^= 1; }
+                }
+            } else {
+                for (int it = 0; it < nsteps; ++it) {
+                    if (!__all_sync(0xffffffffu, mbar_wait(&full[s], ph, abort_flag))) {
+                        ok = false;
+                        if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_TMA_WAIT); *abort_flag = 1; }
+                        break;
+                    }
+                    tc_fence_after();
+                    uint64_t da = desc0 + (uint64_t)((s * stage_bytes) >> 4), db = da + (uint64_t)(w_off >> 4);
+                    for (int j = 0; j < kps; ++j) {
+#pragma unroll
+                        for (int k = 0; k < BK / 16; ++k)
+                            tc_mma(d_tmem, da + 2 * k, db + 2 * k, idesc, (it | j | k) != 0);
+                        da += a_bytes >> 4;
+                        db += p.w_kb_bytes >> 4;
+                    }
+                    tc_commit(&empty[s]);
+                    if (++s == stages) { s = 0; ph ^= 1; }
+                }
             }
             if (!ok) break;
             tc_commit(&acc_full[a]);                      // accumulator complete
@@ -463,9 +559,11 @@ gemm_tc(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensor
     } else {
         const int q = warp & 3;                            // TMEM lane quarter this warp may read
         const int half = (warp - 2) >> 2;                  // which half of the tile's 32-column units it takes
+        grid_dep_wait();
         int a = 0; uint32_t aph = 0;
         for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
-            int nt = tile % p.tiles_n, mt = (tile / p.tiles_n) % p.tiles_m, t = tile / (p.tiles_n * p.tiles_m);
+            int nt, mt, t;
+            tile_coords(p, tile, nt, mt, t);
             const int row = mt * BM + q * 32 + lane;       // the row this thread holds after tcgen05.ld
             const bool row_ok = row < p.M;
             const int n0 = nt * BN;
@@ -512,15 +610,20 @@ pt_status launch_t(const CUtensorMap& ta, const CUtensorMap& tb, GemmP p, cudaSt
     using C = Cfg<BN>;
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tc<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
+        cudaError_t e = cudaFuncSetAttribute(gemm_tc<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
         if (e != cudaSuccess) { set_error("cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
         attr_done = true;
     }
+    if (p.kps < 1) p.kps = 1;
+    p.a_bytes = (uint32_t)stage_a_bytes(p.M);
+    p.stages = ring_stages((int)p.a_bytes, C::B_BYTES, p.kps);
+    if (p.stages < 2 || ((p.K + BK - 1) / BK * p.kt) % p.kps) { set_error("GEMM ring: kps=%d does not fit M=%d K=%d bn=%d", p.kps, p.M, p.K, BN); return PT_ERR_UNSUPPORTED; }
     p.tiles_m = (p.M + BM - 1) / BM;
     p.tiles_n = (p.N + BN - 1) / BN;
     int tiles = p.tiles_m * p.tiles_n * p.T;
     int grid = std::min(tiles, sms);
-    gemm_tc<BN, EPI><<<grid, kGemmThreads, C::SMEM, st>>>(ta, tb, p);
+    cudaError_t e = launch_dependent(gemm_tc<BN, EPI>, dim3(grid), dim3(kGemmThreads), (size_t)kGemmSmem, st, ta, tb, p);
+    if (e != cudaSuccess) { set_error("GEMM launch: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return PT_OK;
 }
@@ -543,6 +646,29 @@ pt_status make_map_bf16_strided(CUtensorMap* out, const void* base, int64_t k, i
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled failed with code %d (k=%lld rows=%lld tracks=%lld)", (int)r, (long long)k, (long long)rows, (long long)tracks); return PT_ERR_CUDA; }
+    return PT_OK;
+}
+
+int gemm_kps(int bn, int M, int K, int kt) {
+    if (kt > 1 || K % BK || M > 256) return 1;
+    int kps = std::max(1, (M <= 64 ? 256 : 128) / bn);
+    while (kps > 1 && (K / BK) % kps) kps >>= 1;
+    return kps;
+}
+
+pt_status make_w_map(CUtensorMap* out, const void* base, int64_t k, int64_t rows, int64_t tracks, int bn, int kps) {
+    if (kps <= 1) return make_map_bf16(out, base, k, rows, tracks, bn);
+    EncodeFn enc = get_encode();
+    if (!enc) { set_error("cuTensorMapEncodeTiled is not available from this driver"); return PT_ERR_CUDA; }
+    if (k % BK) { set_error("a W map of several k-blocks needs k %% 64 == 0"); return PT_ERR_INVALID_ARG; }
+    cuuint64_t dims[4] = {(cuuint64_t)BK, (cuuint64_t)rows, (cuuint64_t)(k / BK), (cuuint64_t)tracks};
+    cuuint64_t strides[3] = {(cuuint64_t)k * 2, (cuuint64_t)BK * 2, (cuuint64_t)k * 2 * (cuuint64_t)rows};
+    cuuint32_t box[4] = {(cuuint32_t)BK, (cuuint32_t)std::min<int64_t>(bn, rows), (cuuint32_t)kps, 1};
+    cuuint32_t es[4] = {1, 1, 1, 1};
+    CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, es,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled (4-D W view) failed with code %d (k=%lld rows=%lld tracks=%lld kps=%d)", (int)r, (long long)k, (long long)rows, (long long)tracks, kps); return PT_ERR_CUDA; }
     return PT_OK;
 }
 
@@ -573,8 +699,10 @@ pt_status launch_gemm(int epi, int bn, const CUtensorMap& ta, const CUtensorMap&
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (sms <= 0) sms = 148;
     }
-    int box_a = std::min(BM, p.M), box_b = std::min(bn, p.kt > 1 ? p.N : p.N);
-    p.tx_bytes = (uint32_t)(box_a + box_b) * BK * 2;
+    const int box_a = std::min(BM, p.M), box_b = std::min(bn, p.N);
+    p.a_tx = (uint32_t)box_a * BK * 2;
+    p.w_kb_bytes = (uint32_t)box_b * BK * 2;
+    p.w_tx = (uint32_t)std::max(p.kps, 1) * p.w_kb_bytes;
 #define CASE(BN_, E_) if (bn == BN_ && epi == E_) return launch_t<BN_, E_>(ta, tb, p, st, sms)
     CASE(64, EPI_PLAIN); CASE(64, EPI_SWIGLU); CASE(64, EPI_RESID);
     CASE(128, EPI_PLAIN); CASE(128, EPI_QKV); CASE(128, EPI_SWIGLU); CASE(128, EPI_RESID);

@@ -25,6 +25,13 @@ def _operands(T, M, N, K, seed):
     (2, 1024, 1024, 1024, 0, False),      # enough tiles for several per CTA, library-chosen width
     (3, 64, 1024, 320, 64, False),        # narrow tiles (decode shapes), few rows
     (2, 200, 160, 192, 64, True),         # narrow tiles, N tail, tracks folded into K
+    (2, 1, 512, 1024, 64, False),         # one row: ring stages of 4 k-blocks, W copied 4 k-blocks at a time
+    (1, 8, 192, 2048, 64, False),         # 8 stages' worth of k-blocks per tile: the ring wraps inside a tile
+    (2, 64, 384, 768, 128, False),        # stages of 2 k-blocks
+    (2, 176, 256, 512, 64, False),        # two row tiles, stages of 2 k-blocks
+    (1, 40, 96, 256, 64, False),          # N tail inside a 4-k-block copy, one stage per tile
+    (1, 16, 48, 256, 64, False),          # N smaller than the tile: the W box is 48 rows
+    (2, 3, 640, 1024, 0, False),          # library-chosen width and stage shape at decode size
 ])
 def test_gemm_bf16_matches_definition(T, M, N, K, bn, fold):
     import torch
