@@ -173,8 +173,8 @@ pt_status pt_lm_head(pt_model* m, const float* h, int64_t row_stride, int64_t n,
     g_launches.fetch_add(1, std::memory_order_relaxed);
     const int bn = gemm_bn(V, (int)n, 1, EPI_PLAIN);
     CUtensorMap ta, tb;
-    if ((s = make_map_bf16(&ta, hn, H, n, 1, 128)) != PT_OK) return s;
     const int kps = gemm_kps(bn, (int)n, H, 1);
+    if ((s = make_a_map(&ta, hn, H, n, 1, kps)) != PT_OK) return s;
     if ((s = make_w_map(&tb, m->lm_buf + l.off_head, H, V, 1, bn, kps)) != PT_OK) return s;
     GemmP p{};
     p.kps = kps;

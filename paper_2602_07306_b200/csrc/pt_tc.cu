@@ -135,11 +135,20 @@ pt_status tc_forward(Call& k) {
     __nv_bfloat16* o = (__nv_bfloat16*)w.o;
     __nv_bfloat16* z = (__nv_bfloat16*)w.z;
 
-    CUtensorMap ta_h, ta_o, ta_z;
+    // A operands (normalised stream, attention output, SwiGLU output): one map per copy shape a GEMM of this call uses
+    struct AMaps { CUtensorMap m[3]; bool have[3] = {false, false, false}; } ta_h, ta_o, ta_z;
     pt_status s;
-    if ((s = make_map_bf16(&ta_h, hb, H, M, T, 128)) != PT_OK) return s;
-    if ((s = make_map_bf16(&ta_o, o, m->QD, M, T, 128)) != PT_OK) return s;
-    if ((s = make_map_bf16(&ta_z, z, F, M, T, 128)) != PT_OK) return s;
+    auto a_map = [&](AMaps& am, const void* base, int64_t kk, int kps, const CUtensorMap** out) -> pt_status {
+        const int i = kps_index(kps);
+        if (!am.have[i]) {
+            pt_status r = make_a_map(&am.m[i], base, kk, M, T, kps);
+            if (r != PT_OK) return r;
+            am.have[i] = true;
+        }
+        *out = &am.m[i];
+        return PT_OK;
+    };
+    const CUtensorMap* ta = nullptr;
 
     { ProfScope ps(m, st, 6);
     k_tc_prep<<<dim3((M * 32 + 255) / 256, T), 256, 0, st>>>((const __nv_bfloat16*)k.x, k.x_stride, m->gain(0, 0), w.hT, hb, w.ssq, M, H, tiles);
@@ -162,8 +171,9 @@ pt_status tc_forward(Call& k) {
             p.nq = g.heads; p.nkv = g.kv_heads; p.dh = m->dh; p.ps = c->ps;
             int bn = gemm_bn(p.N, M, T, EPI_QKV);
             p.kps = gemm_kps(bn, M, p.K, 1);
+            if ((s = a_map(ta_h, hb, H, p.kps, &ta)) != PT_OK) return s;
             ProfScope ps(m, st, 1);
-            if ((s = launch_gemm(EPI_QKV, bn, ta_h, wm[l].m[0][bn_index(bn)][kps_index(p.kps)], p, st)) != PT_OK) return s;
+            if ((s = launch_gemm(EPI_QKV, bn, *ta, wm[l].m[0][bn_index(bn)][kps_index(p.kps)], p, st)) != PT_OK) return s;
         }
         {
             ProfScope ps(m, st, 0);
@@ -179,8 +189,9 @@ pt_status tc_forward(Call& k) {
             p.ssq_out = w.ssq; p.ssq_out_tstride = (size_t)M * tiles; p.ssq_out_tiles = tiles;
             int bn = gemm_bn(p.N, M, T, EPI_RESID);
             p.kps = gemm_kps(bn, M, p.K, 1);
+            if ((s = a_map(ta_o, o, m->QD, p.kps, &ta)) != PT_OK) return s;
             ProfScope ps(m, st, 2);
-            if ((s = launch_gemm(EPI_RESID, bn, ta_o, wm[l].m[1][bn_index(bn)][kps_index(p.kps)], p, st)) != PT_OK) return s;
+            if ((s = launch_gemm(EPI_RESID, bn, *ta, wm[l].m[1][bn_index(bn)][kps_index(p.kps)], p, st)) != PT_OK) return s;
             ssq_tstride = (size_t)M * tiles;
         }
         tap_copy(k, l, 0, w.hT, MH);
@@ -191,8 +202,9 @@ pt_status tc_forward(Call& k) {
             p.z_out = z;
             int bn = gemm_bn(p.N, M, T, EPI_SWIGLU);
             p.kps = gemm_kps(bn, M, p.K, 1);
+            if ((s = a_map(ta_h, hb, H, p.kps, &ta)) != PT_OK) return s;
             ProfScope ps(m, st, 3);
-            if ((s = launch_gemm(EPI_SWIGLU, bn, ta_h, wm[l].m[2][bn_index(bn)][kps_index(p.kps)], p, st)) != PT_OK) return s;
+            if ((s = launch_gemm(EPI_SWIGLU, bn, *ta, wm[l].m[2][bn_index(bn)][kps_index(p.kps)], p, st)) != PT_OK) return s;
         }
         {   // down projection + residual (+ track-sync when the layer closes a track block)
             const bool sync = (l + 1) % g.D == 0, last = l + 1 == g.L;
@@ -218,8 +230,9 @@ pt_status tc_forward(Call& k) {
             }
             int bn = gemm_bn(p.N, M, p.T, EPI_RESID);
             p.kps = gemm_kps(bn, M, p.K, p.kt);
+            if ((s = a_map(ta_z, z, F, p.kps, &ta)) != PT_OK) return s;
             ProfScope ps(m, st, sync ? 5 : 4);
-            if ((s = launch_gemm(EPI_RESID, bn, ta_z, wm[l].m[3][bn_index(bn)][kps_index(p.kps)], p, st)) != PT_OK) return s;
+            if ((s = launch_gemm(EPI_RESID, bn, *ta, wm[l].m[3][bn_index(bn)][kps_index(p.kps)], p, st)) != PT_OK) return s;
             float* ho = last ? k.out : w.hS;
             __nv_bfloat16* hb_next = last ? nullptr : hb;
             const float* gain_next = last ? nullptr : m->gain(0, l + 1);
@@ -261,8 +274,8 @@ extern "C" pt_status pt_kernel_gemm_bf16(const void* a, const void* w, void* c, 
     if (bn != 64 && bn != 128 && bn != 256) { set_error("bn must be 0, 64, 128 or 256"); return PT_ERR_INVALID_ARG; }
     CUtensorMap ta, tb;
     pt_status s;
-    if ((s = make_map_bf16(&ta, a, K, M, T, 128)) != PT_OK) return s;
     const int kps = gemm_kps(bn, M, K, fold_tracks ? T : 1);
+    if ((s = make_a_map(&ta, a, K, M, T, kps)) != PT_OK) return s;
     if ((s = make_w_map(&tb, w, K, N, T, bn, kps)) != PT_OK) return s;
     GemmP p{};
     p.M = M; p.N = N; p.K = K; p.T = fold_tracks ? 1 : T; p.kt = fold_tracks ? T : 1; p.kps = kps;

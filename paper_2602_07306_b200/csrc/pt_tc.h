@@ -17,7 +17,7 @@ struct GemmP {
     int tiles_m, tiles_n;   // filled by the launcher
     int kps;                // k-blocks per ring stage (1, or 2 / 4 with a 4-D W map from make_w_map; see gemm_kps)
     // filled by the launcher:
-    uint32_t a_tx, w_tx;    // bytes one A copy and the stage's W copy deliver
+    uint32_t a_tx, w_tx;    // bytes a stage's A copy and its W copy deliver
     uint32_t a_bytes;       // shared-memory bytes reserved per k-block of A; the stage's W part follows its kps A pieces
     uint32_t w_kb_bytes;    // shared-memory bytes one k-block of W takes
     int stages;             // ring depth
@@ -100,6 +100,8 @@ int gemm_bn(int N, int M, int T, int epi);
 int gemm_kps(int bn, int M, int K, int kt);
 // tensor map of W [tracks][rows][k] for tiles of bn rows: 3-D (k, row, track) for kps = 1, else 4-D (64, row, k-block, track)
 pt_status make_w_map(CUtensorMap* out, const void* base, int64_t k, int64_t rows, int64_t tracks, int bn, int kps);
+// tensor map of A [tracks][rows][k] to go with it: 3-D with a box of min(rows, 128) rows for kps = 1, else 4-D with kps k-blocks per copy
+pt_status make_a_map(CUtensorMap* out, const void* base, int64_t k, int64_t rows, int64_t tracks, int kps);
 inline int bn_index(int bn) { return bn == 64 ? 0 : (bn == 128 ? 1 : 2); }
 pt_status launch_gemm(int epi, int bn, const CUtensorMap& ta, const CUtensorMap& tb, GemmP p, cudaStream_t st);
 

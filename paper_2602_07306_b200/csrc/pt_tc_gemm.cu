@@ -438,7 +438,7 @@ gemm_tc(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensor
     const int kpb = (p.K + BK - 1) / BK;            // k-blocks per track
     const int kblocks = kpb * p.kt;
     const int nsteps = kblocks / kps;                // ring stages one tile consumes (kps divides kblocks)
-    const uint32_t stage_tx = kps * p.a_tx + p.w_tx;
+    const uint32_t stage_tx = p.a_tx + p.w_tx;
 
     if (warp == 0) {
         if (lane == 0) {
@@ -487,9 +487,7 @@ gemm_tc(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensor
                             if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_EMPTY_WAIT); *abort_flag = 1; break; }
                             mbar_expect_tx(&full[s], stage_tx);
                         }
-                        uint8_t* sa = smem + s * stage_bytes;
-                        for (int j = 0; j < kps; ++j)
-                            tma_load_3d(sa + j * a_bytes, &ta, &full[s], (it * kps + j) * BK, mt * BM, t);
+                        tma_load_4d(smem + s * stage_bytes, &ta, &full[s], 0, mt * BM, it * kps, t);    // kps k-blocks of A, a_bytes apart
                         if (it >= npre) load_w(s, it, nt, t);
                         if (++s == stages) { s = 0; ph ^= 1; }
                     }
@@ -672,6 +670,25 @@ pt_status make_w_map(CUtensorMap* out, const void* base, int64_t k, int64_t rows
     return PT_OK;
 }
 
+pt_status make_a_map(CUtensorMap* out, const void* base, int64_t k, int64_t rows, int64_t tracks, int kps) {
+    if (kps <= 1) return make_map_bf16(out, base, k, rows, tracks, BM);
+    EncodeFn enc = get_encode();
+    if (!enc) { set_error("cuTensorMapEncodeTiled is not available from this driver"); return PT_ERR_CUDA; }
+    if (k % BK) { set_error("an A map of several k-blocks needs k %% 64 == 0"); return PT_ERR_INVALID_ARG; }
+    // the box is a whole number of 8-row swizzle atoms, so that every k-block of the copy starts one; rows past
+    // the tensor's end are filled with zeros by the copy
+    const int box_rows = stage_a_bytes((int)std::min<int64_t>(rows, BM)) / (BK * 2);
+    cuuint64_t dims[4] = {(cuuint64_t)BK, (cuuint64_t)rows, (cuuint64_t)(k / BK), (cuuint64_t)tracks};
+    cuuint64_t strides[3] = {(cuuint64_t)k * 2, (cuuint64_t)BK * 2, (cuuint64_t)k * 2 * (cuuint64_t)rows};
+    cuuint32_t box[4] = {(cuuint32_t)BK, (cuuint32_t)box_rows, (cuuint32_t)kps, 1};
+    cuuint32_t es[4] = {1, 1, 1, 1};
+    CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, es,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled (4-D A view) failed with code %d (k=%lld rows=%lld tracks=%lld kps=%d)", (int)r, (long long)k, (long long)rows, (long long)tracks, kps); return PT_ERR_CUDA; }
+    return PT_OK;
+}
+
 int gemm_bn(int N, int M, int T, int epi) {
     // Tile width by a round model: a launch runs ceil(tiles / SMs) rounds and a round costs about
     // bn + min(M, 128) (bytes of B and A streamed per k-block when M is small, and near enough the MMA
@@ -699,8 +716,8 @@ pt_status launch_gemm(int epi, int bn, const CUtensorMap& ta, const CUtensorMap&
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (sms <= 0) sms = 148;
     }
-    const int box_a = std::min(BM, p.M), box_b = std::min(bn, p.N);
-    p.a_tx = (uint32_t)box_a * BK * 2;
+    const int box_b = std::min(bn, p.N);
+    p.a_tx = p.kps > 1 ? (uint32_t)p.kps * (uint32_t)stage_a_bytes(p.M) : (uint32_t)std::min(BM, p.M) * BK * 2;
     p.w_kb_bytes = (uint32_t)box_b * BK * 2;
     p.w_tx = (uint32_t)std::max(p.kps, 1) * p.w_kb_bytes;
 #define CASE(BN_, E_) if (bn == BN_ && epi == E_) return launch_t<BN_, E_>(ta, tb, p, st, sms)
