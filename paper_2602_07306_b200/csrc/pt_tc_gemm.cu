@@ -118,9 +118,10 @@ __device__ __forceinline__ void report(int* status, int code, int loc) {
 // SM's TMA unit for about a memory latency whatever its size, so W streams from HBM at full rate only
 // with 16 KB or more per copy.
 constexpr int kMaxStages = 24;
-constexpr int kRingBytes = 216 * 1024;                       // stages + the slack behind the last one
+constexpr int kRingBytes = 192 * 1024;                       // stages + the slack behind the last one
+constexpr int kXposeBytes = kEpiWarps * 4096;                // per epilogue warp: 32 rows x 128 bytes to turn row-per-thread data
 constexpr int kBarBytes = 512;                               // 2 * kMaxStages + 4 mbarriers, TMEM slot, abort flag
-constexpr int kGemmSmem = kRingBytes + 1024 /*alignment*/ + kBarBytes;
+constexpr int kGemmSmem = kRingBytes + kXposeBytes + 1024 /*alignment*/ + kBarBytes;
 constexpr int kFullA = BM * BK * 2;
 
 template <int BN> struct Cfg {
@@ -302,82 +303,122 @@ __device__ __forceinline__ bool epi_qkv(const GemmP& p, uint32_t taddr, int t, i
 }
 
 // Residual add (+ track-sync sum), fp32 stream out, gain-scaled bf16 copy, partial sums of squares.
-// The 32 residual values of a unit (128 bytes of the thread's row) are fetched one unit ahead.
+// tcgen05.ld leaves one accumulator row per thread; global accesses in that shape touch 32 different
+// 128-byte lines per instruction, and this epilogue moves 10-14 bytes per element, so it was bound by
+// load/store-unit wavefronts.  Each 32 x 32 unit is therefore turned through the warp's 4 KB of shared
+// memory (16-byte chunks XOR-swizzled by row, conflict-free both ways) into "four lanes per row, eight
+// columns per lane": every global instruction then covers 8 rows x 128 contiguous bytes.  Residual rows
+// are fetched in the same shape, one unit ahead and before the wait for the accumulator.
 template <int BN, class Wait>
-__device__ __forceinline__ bool epi_resid(const GemmP& p, uint32_t taddr, int t, int row, bool row_ok, int n0, int half, Wait wait) {
+__device__ __forceinline__ bool epi_resid(const GemmP& p, uint32_t taddr, int t, int row, int n0, int half, uint8_t* xbuf, Wait wait) {
     constexpr int UNITS = BN / 32;                        // 32-column units of the tile; 64-column groups alternate between the two warps
-    const float* hrow = p.h_in + (size_t)(p.n_sum > 1 ? 0 : t) * p.h_in_tstride + (size_t)row * p.N;
-    auto fetch = [&](int u, float* h) {                   // h[0..31]: residual (summed over tracks at a sync)
-        const int col = n0 + u * 32;
+    const int lane = threadIdx.x & 31;
+    const int row0 = row - lane;                          // first row of the warp's 32
+    const int rsub = lane >> 2, cc = (lane & 3) * 8;      // this thread: rows row0 + 8r + rsub (r = 0..3), columns cc..cc+7 of the unit
+    const float* hbase = p.h_in + (size_t)(p.n_sum > 1 ? 0 : t) * p.h_in_tstride;
+    auto fetch = [&](int u, float* h) {                   // h[8r..8r+7]: residual of row r (summed over tracks at a sync)
+        const int col = n0 + u * 32 + cc;
 #pragma unroll
         for (int i = 0; i < 32; ++i) h[i] = 0.f;
-        if (!row_ok) return;
+        if (col >= p.N) return;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) if (col + 8 * i < p.N) ld256(hrow + col + 8 * i, h + 8 * i);
+        for (int r = 0; r < 4; ++r) {
+            const int rr = row0 + 8 * r + rsub;
+            if (rr < p.M) ld256(hbase + (size_t)rr * p.N + col, h + 8 * r);
+        }
         for (int tt = 1; tt < p.n_sum; ++tt) {
-            float x[32];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                if (col + 8 * i < p.N) {
-                    ld256(hrow + (size_t)tt * p.h_in_tstride + col + 8 * i, x + 8 * i);
+            for (int r = 0; r < 4; ++r) {
+                const int rr = row0 + 8 * r + rsub;
+                if (rr < p.M) {
+                    float x[8];
+                    ld256(hbase + (size_t)tt * p.h_in_tstride + (size_t)rr * p.N + col, x);
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) h[8 * i + k] += x[8 * i + k];
+                    for (int k = 0; k < 8; ++k) h[8 * r + k] += x[k];
                 }
             }
         }
     };
+    const uint32_t xs = smem_u32(xbuf);
+    const uint32_t st_base = xs + lane * 128;                         // row-per-thread side: my row
+    const uint32_t sw = (uint32_t)(lane & 7);
     float hres[32], hnxt[32];
     fetch(2 * half, hres);
     if (!wait()) return false;
-    float ssq = 0.f;
+    float ssq[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 1
     for (int u = 2 * half; u < UNITS; u += (u & 1) ? 3 : 1) {      // units 0,1, 4,5, ... or 2,3, 6,7, ...
         const int c = u * 32;
-        const int col = n0 + c;
-        if (col >= p.N) break;                             // uniform across the warp
+        if (n0 + c >= p.N) break;                          // uniform across the warp
+        const int col = n0 + c + cc;
+        const bool col_ok = col < p.N;
         float v[32];
         tc_ld16(taddr + c, v);
         tc_ld16(taddr + c + 16, v + 16);
         const int un = u + ((u & 1) ? 3 : 1);
         if (un < UNITS) fetch(un, hnxt);
         tc_wait_ld();
-        if (row_ok) {
+        __syncwarp();                                      // the previous unit's reads of the buffer are done
 #pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = (v[i] + hres[i]) * p.scale;
-            float* ho = p.h_out + (size_t)t * p.h_out_tstride + (size_t)row * p.N + col;
+        for (int j = 0; j < 8; ++j)
+            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(st_base + ((j ^ sw) << 4)),
+                         "f"(v[4 * j]), "f"(v[4 * j + 1]), "f"(v[4 * j + 2]), "f"(v[4 * j + 3]) : "memory");
+        __syncwarp();
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                if (col + 8 * i < p.N) {
-                    st256(ho + 8 * i, v + 8 * i);
+        for (int r = 0; r < 4; ++r) {
+            const uint32_t rb = xs + (8 * r + rsub) * 128;            // (8r + rsub) & 7 == rsub
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) ssq += v[8 * i + k] * v[8 * i + k];
-                }
+            for (int h2 = 0; h2 < 2; ++h2) {
+                const uint32_t chunk = (uint32_t)(2 * (lane & 3) + h2) ^ (uint32_t)rsub;
+                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                             : "=f"(v[8 * r + 4 * h2]), "=f"(v[8 * r + 4 * h2 + 1]), "=f"(v[8 * r + 4 * h2 + 2]), "=f"(v[8 * r + 4 * h2 + 3])
+                             : "r"(rb + (chunk << 4)) : "memory");
             }
-            if (p.hb_out) {
-                for (int to = 0; to < p.n_out; ++to) {
-                    const int tg = p.n_out > 1 ? to : t;
-                    const float4* gp = (const float4*)(p.gain + (size_t)tg * p.N + col);
-                    __nv_bfloat16* hb = p.hb_out + ((size_t)tg * p.M + row) * p.N + col;
+        }
+        float part[4];
 #pragma unroll
-                    for (int g2 = 0; g2 < 2; ++g2) {
-                        if (col + 16 * g2 < p.N) {
-                            float w[16];
+        for (int r = 0; r < 4; ++r) {
+            const int rr = row0 + 8 * r + rsub;
+            const bool ok = col_ok && rr < p.M;
+            float sq = 0.f;
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                const float4 g = gp[4 * g2 + i];
-                                w[4 * i] = v[16 * g2 + 4 * i] * g.x; w[4 * i + 1] = v[16 * g2 + 4 * i + 1] * g.y;
-                                w[4 * i + 2] = v[16 * g2 + 4 * i + 2] * g.z; w[4 * i + 3] = v[16 * g2 + 4 * i + 3] * g.w;
-                            }
-                            store16_bf16(hb + 16 * g2, w);
-                        }
+            for (int k = 0; k < 8; ++k) { v[8 * r + k] = (v[8 * r + k] + hres[8 * r + k]) * p.scale; sq += v[8 * r + k] * v[8 * r + k]; }
+            part[r] = ok ? sq : 0.f;
+            if (ok) st256(p.h_out + (size_t)t * p.h_out_tstride + (size_t)rr * p.N + col, v + 8 * r);
+        }
+        if (p.hb_out && col_ok) {
+            for (int to = 0; to < p.n_out; ++to) {
+                const int tg = p.n_out > 1 ? to : t;
+                const float4 g0 = *(const float4*)(p.gain + (size_t)tg * p.N + col), g1 = *(const float4*)(p.gain + (size_t)tg * p.N + col + 4);
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const int rr = row0 + 8 * r + rsub;
+                    if (rr < p.M) {
+                        const float* w = v + 8 * r;
+                        uint4 o;
+                        o.x = pack_bf16(w[0] * g0.x, w[1] * g0.y); o.y = pack_bf16(w[2] * g0.z, w[3] * g0.w);
+                        o.z = pack_bf16(w[4] * g1.x, w[5] * g1.y); o.w = pack_bf16(w[6] * g1.z, w[7] * g1.w);
+                        *reinterpret_cast<uint4*>(p.hb_out + ((size_t)tg * p.M + rr) * p.N + col) = o;
                     }
                 }
             }
         }
-        if ((u & 1) == 1 || col + 32 >= p.N) {             // a kSsqTile-column group is complete
-            if (row_ok && p.ssq_out)
-                p.ssq_out[(size_t)t * p.ssq_out_tstride + (size_t)row * p.ssq_out_tiles + col / kSsqTile] = ssq;
-            ssq = 0.f;
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {                      // row sums over the four lanes of a row
+            part[r] += __shfl_xor_sync(0xffffffffu, part[r], 1);
+            part[r] += __shfl_xor_sync(0xffffffffu, part[r], 2);
+            ssq[r] += part[r];
+        }
+        if ((u & 1) == 1 || n0 + c + 32 >= p.N) {          // a kSsqTile-column group is complete
+            if (p.ssq_out && (lane & 3) == 0) {
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const int rr = row0 + 8 * r + rsub;
+                    if (rr < p.M) p.ssq_out[(size_t)t * p.ssq_out_tstride + (size_t)rr * p.ssq_out_tiles + (n0 + c) / kSsqTile] = ssq[r];
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < 4; ++r) ssq[r] = 0.f;
         }
 #pragma unroll
         for (int i = 0; i < 32; ++i) hres[i] = hnxt[i];     // last: the fetch stays in flight until here
@@ -386,11 +427,11 @@ __device__ __forceinline__ bool epi_resid(const GemmP& p, uint32_t taddr, int t,
 }
 
 template <int BN, int EPI, class Wait>
-__device__ __forceinline__ bool epilogue(const GemmP& p, uint32_t taddr, int t, int row, bool row_ok, int n0, int half, Wait wait) {
+__device__ __forceinline__ bool epilogue(const GemmP& p, uint32_t taddr, int t, int row, bool row_ok, int n0, int half, uint8_t* xbuf, Wait wait) {
     if (EPI == EPI_PLAIN) return epi_plain<BN>(p, taddr, t, row, row_ok, n0, half, wait);
     else if (EPI == EPI_QKV) return epi_qkv<BN>(p, taddr, t, row, row_ok, n0, half, wait);
     else if (EPI == EPI_SWIGLU) return epi_swiglu<BN>(p, taddr, t, row, row_ok, n0, half, wait);
-    else return epi_resid<BN>(p, taddr, t, row, row_ok, n0, half, wait);
+    else return epi_resid<BN>(p, taddr, t, row, n0, half, xbuf, wait);
 }
 
 // Tile index -> (column tile, row tile, track).  With one or two row tiles (a decode step) the row
@@ -408,7 +449,8 @@ gemm_tc(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensor
     using C = Cfg<BN>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint64_t* full = (uint64_t*)(smem + kRingBytes);
+    uint8_t* xpose = smem + kRingBytes;
+    uint64_t* full = (uint64_t*)(xpose + kXposeBytes);
     uint64_t* empty = full + kMaxStages;
     uint64_t* acc_full = empty + kMaxStages;
     uint64_t* acc_empty = acc_full + 2;
@@ -573,7 +615,7 @@ gemm_tc(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensor
                 tc_fence_after();
                 return true;
             };
-            if (!epilogue<BN, EPI>(p, taddr, t, row, row_ok, n0, half, wait_acc)) break;
+            if (!epilogue<BN, EPI>(p, taddr, t, row, row_ok, n0, half, xpose + (warp - 2) * 4096, wait_acc)) break;
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[a]);
@@ -650,7 +692,7 @@ pt_status make_map_bf16_strided(CUtensorMap* out, const void* base, int64_t k, i
 int gemm_kps(int bn, int M, int K, int kt) {
     if (kt > 1 || K % BK || M > 256) return 1;
     int kps = std::max(1, (M <= 64 ? 256 : 128) / bn);
-    while (kps > 1 && (K / BK) % kps) kps >>= 1;
+    while (kps > 1 && ((K / BK) % kps || ring_stages(stage_a_bytes(M), bn * BK * 2, kps) < 3)) kps >>= 1;
     return kps;
 }
 
