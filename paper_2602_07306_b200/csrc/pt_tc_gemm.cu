@@ -691,7 +691,7 @@ pt_status make_map_bf16_strided(CUtensorMap* out, const void* base, int64_t k, i
 
 int gemm_kps(int bn, int M, int K, int kt) {
     if (kt > 1 || K % BK || M > 256) return 1;
-    int kps = std::max(1, (M <= 64 ? 256 : 128) / bn);
+    int kps = std::max(1, 256 / bn);
     while (kps > 1 && ((K / BK) % kps || ring_stages(stage_a_bytes(M), bn * BK * 2, kps) < 3)) kps >>= 1;
     return kps;
 }
