@@ -432,6 +432,14 @@ def aggregate_over_ranks(ms, tokens, e2e_tokens_per_s, world, device):
     return float(tmax[0].item()), total, total / float(tmax[1].item())
 
 
+def aggregate_track_ranks(ms, tokens, e2e_tokens_per_s, world, device):
+    """Whole-job numbers of a track-parallel run: every rank holds T / world tracks of ONE model and
+    all ranks process the same batch, so the job's tokens are one rank's (not the sum) and its step
+    time is the slowest rank's; the same for the end-to-end leg.  Returns (ms, tokens, e2e_tokens_per_s)."""
+    ms_max, total, e2e_sum_over_max = aggregate_over_ranks(ms, tokens, e2e_tokens_per_s, world, device)
+    return ms_max, total / world, e2e_sum_over_max / world
+
+
 # ------------------------------------------------------------------------------ main
 
 def main():
@@ -502,8 +510,7 @@ def main():
         assert wl.T % world == 0, "the number of ranks must divide the number of tracks"
         TRACK_PARALLEL.update(on=True, world=world, rank=rank, tracks=wl.T)
         r = run(dataclasses.replace(wl, T=wl.T // world), dev, a.steps, a.warmup, barrier, 0)
-        ms, _, e2e_value = aggregate_over_ranks(r["ms"], r["tokens"], r["e2e"]["value"], world, dev)
-        total_tokens, e2e_value = float(r["tokens"]), e2e_value / world
+        ms, total_tokens, e2e_value = aggregate_track_ranks(r["ms"], r["tokens"], r["e2e"]["value"], world, dev)
         r["config"]["parallelism"] = f"tracks: {wl.T} tracks over {world} rank(s), one all-reduce per track block"
     else:
         r = run(wl, dev, a.steps, a.warmup, barrier, rank)
