@@ -1,5 +1,5 @@
 """Track parallelism across ranks (the paper's deployment: some tracks per GPU, one all-reduce per track
-block).  Every gpurun-style single-GPU machine can still check it end to end: a rank is a model that holds
+block).  One GPU is enough to check it end to end: a rank is a model that holds
 part of the tracks plus an all-reduce hook, and two such ranks can share one GPU as long as their kernels
 never wait for each other on the device - here the exchange is a host-side barrier between two threads."""
 import threading
