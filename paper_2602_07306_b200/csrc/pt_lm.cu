@@ -174,10 +174,11 @@ pt_status pt_lm_head(pt_model* m, const float* h, int64_t row_stride, int64_t n,
     const int bn = gemm_bn(V, (int)n, 1, EPI_PLAIN);
     CUtensorMap ta, tb;
     const int kps = gemm_kps(bn, (int)n, H, 1);
+    const bool pair = gemm_pair_ok(bn, (int)n, V);
     if ((s = make_a_map(&ta, hn, H, n, 1, kps)) != PT_OK) return s;
-    if ((s = make_w_map(&tb, m->lm_buf + l.off_head, H, V, 1, bn, kps)) != PT_OK) return s;
+    if ((s = make_w_map(&tb, m->lm_buf + l.off_head, H, V, 1, pair ? 128 : bn, kps)) != PT_OK) return s;
     GemmP p{};
-    p.kps = kps;
+    p.kps = kps; p.pair = pair;
     p.M = (int)n; p.N = V; p.K = H; p.T = 1; p.kt = 1; p.status = m->status(); p.c_out = logits; p.scale = 1.f; p.n_sum = 1; p.n_out = 1;
     if ((s = launch_gemm(EPI_PLAIN, bn, ta, tb, p, st)) != PT_OK) return s;
     if (next_token) {

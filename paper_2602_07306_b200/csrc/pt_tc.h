@@ -15,6 +15,7 @@ struct GemmP {
     int T;                  // tracks folded into the grid
     int kt;                 // tracks folded into the K loop (1, or all tracks for the sync GEMM with T = 1)
     int tiles_m, tiles_n;   // filled by the launcher
+    int pair;               // 1: CTA-pair kernel (256 x 256 tiles, tb with 128-row boxes); see gemm_pair_ok
     int kps;                // k-blocks per ring stage (1, or 2 / 4 with a 4-D W map from make_w_map; see gemm_kps)
     // filled by the launcher:
     uint32_t a_tx, w_tx;    // bytes a stage's A copy and its W copy deliver
@@ -98,6 +99,8 @@ pt_status make_map_bf16_strided(CUtensorMap* out, const void* base, int64_t k, i
 int gemm_bn(int N, int M, int T, int epi);
 // k-blocks per ring stage for a launch of M rows: more than one when the rows are few, so that a copy of W is 16-32 KB
 int gemm_kps(int bn, int M, int K, int kt);
+// whether a launch should use the CTA-pair kernel (then W's map is the one with 128-row boxes and kps = 1)
+bool gemm_pair_ok(int bn, int M, int N);
 // tensor map of W [tracks][rows][k] for tiles of bn rows: 3-D (k, row, track) for kps = 1, else 4-D (64, row, k-block, track)
 pt_status make_w_map(CUtensorMap* out, const void* base, int64_t k, int64_t rows, int64_t tracks, int bn, int kps);
 // tensor map of A [tracks][rows][k] to go with it: 3-D with a box of min(rows, 128) rows for kps = 1, else 4-D with kps k-blocks per copy

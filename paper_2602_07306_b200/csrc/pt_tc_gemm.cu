@@ -630,6 +630,182 @@ gemm_tc(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensor
     }
 }
 
+// ---- CTA-pair variant ------------------------------------------------------------------------
+// With one CTA per tile the main loop of a 128 x 256 tile pulls 48 KB per k-block into the SM, and that
+// copy (about 70 bytes per cycle per SM) takes longer than the 512 cycles of its four MMAs.  Two CTAs of a
+// cluster therefore share a 256 x 256 tile: each loads its own 128 rows of A and HALF of the W tile (128
+// rows), and one tcgen05.mma.cta_group::2 per 16 columns of K, issued by the even CTA, multiplies both A
+// halves with both W halves, leaving each CTA the accumulator of its own 128 rows in its own tensor
+// memory.  Per CTA and k-block: 32 KB copied for the same 512 MMA cycles, and six ring stages.
+// Barriers live at the same shared-memory offsets in both CTAs.  The even CTA's full[s] collects both
+// CTAs' copies (two arrivals with expected bytes); after the MMAs of a stage it commits to both CTAs'
+// empty[s], after a tile to both CTAs' acc_full[a]; the epilogue warps of both CTAs arrive at the even
+// CTA's acc_empty[a].  No copy is multicast.  Every wait is bounded as in gemm_tc.
+constexpr int kPairStages = 6;
+constexpr int kPairStageBytes = 2 * BM * BK * 2;             // 128 rows of A + 128 rows of W per k-block
+
+__device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t bar_cluster_addr, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(bar_cluster_addr), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+// copy whose completion bytes go to a barrier of the even CTA of the pair
+__device__ __forceinline__ void tma_load_3d_pair(void* dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int c0, int c1, int c2) {
+    asm volatile("cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                 ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(c0), "r"(c1), "r"(c2), "r"(bar_cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n .reg .pred p, e;\n elect.sync _|e, 0xffffffff;\n setp.ne.b32 p, %4, 0;\n"
+                 " @e tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar_cluster_addr) {
+    asm volatile("{\n .reg .pred e;\n elect.sync _|e, 0xffffffff;\n"
+                 " @e tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}" ::"r"(bar_cluster_addr) : "memory");
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_tc_pair(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensorMap tb, const GemmP p) {
+    constexpr int BN = 256;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t* xpose = smem + kRingBytes;
+    uint64_t* full = (uint64_t*)(xpose + kXposeBytes);
+    uint64_t* empty = full + kMaxStages;
+    uint64_t* acc_full = empty + kMaxStages;
+    uint64_t* acc_empty = acc_full + 2;
+    uint32_t* tmem_slot = (uint32_t*)(acc_empty + 2);
+    volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+    const uint32_t rank = cluster_rank();                   // 0: issues the MMAs; 1: its partner
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kPairStages; ++s) { mbar_init(&full[s], 2); mbar_init(&empty[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 2 * kEpiWarps); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {                                        // the same warp of both CTAs, the same slot address
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(2 * BN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                     // both CTAs' barriers exist before anything arrives at them
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int tiles_m2 = (p.M + 2 * BM - 1) / (2 * BM);     // row tiles of 256
+    const int num_tiles = tiles_m2 * p.tiles_n * p.T;
+    const int kpb = (p.K + BK - 1) / BK;
+    const int kblocks = kpb * p.kt;
+    const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+    auto coords = [&](int tile, int& nt, int& mt2, int& t) { nt = tile % p.tiles_n; mt2 = (tile / p.tiles_n) % tiles_m2; t = tile / (p.tiles_n * tiles_m2); };
+    grid_dep_wait();
+    if (threadIdx.x == 0) grid_dep_launch();
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int s = 0; uint32_t ph = 0;
+            bool ok = true;
+            for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
+                int nt, mt2, t;
+                coords(tile, nt, mt2, t);
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_EMPTY_WAIT); *abort_flag = 1; break; }
+                    const int tt = p.kt > 1 ? kb / kpb : t;
+                    const int k0 = (p.kt > 1 ? kb % kpb : kb) * BK;
+                    uint8_t* sa = smem + s * kPairStageBytes;
+                    const uint32_t fb = map_to_cta(smem_u32(&full[s]), 0);
+                    mbar_expect_tx_cluster(fb, p.a_tx + p.w_tx);
+                    tma_load_3d_pair(sa, &ta, fb, k0, (mt2 * 2 + (int)rank) * BM, tt);
+                    tma_load_3d_pair(sa + BM * BK * 2, &tb, fb, k0, nt * BN + (int)rank * (BN / 2), tt);
+                    if (++s == kPairStages) { s = 0; ph ^= 1; }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (rank == 0) {
+            constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+            const uint64_t desc0 = smem_desc(smem_u32(smem));
+            int s = 0; uint32_t ph = 0;
+            int a = 0; uint32_t aph = 0;
+            bool ok = true;
+            for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
+                if (!__all_sync(0xffffffffu, mbar_wait(&acc_empty[a], aph ^ 1, abort_flag))) {
+                    if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_ACC_WAIT); *abort_flag = 1; }
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + a * BN;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!__all_sync(0xffffffffu, mbar_wait(&full[s], ph, abort_flag))) {
+                        ok = false;
+                        if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_TMA_WAIT); *abort_flag = 1; }
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint64_t da = desc0 + (uint64_t)((s * kPairStageBytes) >> 4), db = da + (uint64_t)((BM * BK * 2) >> 4);
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)
+                        tc_mma_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+                    tc_commit_pair(smem_u32(&empty[s]));                        // both CTAs may refill the stage
+                    tc_commit_pair(map_to_cta(smem_u32(&empty[s]), 1));
+                    if (++s == kPairStages) { s = 0; ph ^= 1; }
+                }
+                if (!ok) break;
+                tc_commit_pair(smem_u32(&acc_full[a]));                         // both CTAs' epilogues may drain
+                tc_commit_pair(map_to_cta(smem_u32(&acc_full[a]), 1));
+                if (++a == 2) { a = 0; aph ^= 1; }
+            }
+        }
+        __syncwarp();
+    } else {
+        const int q = warp & 3;
+        const int half = (warp - 2) >> 2;
+        int a = 0; uint32_t aph = 0;
+        for (int tile = pair; tile < num_tiles; tile += npairs) {
+            int nt, mt2, t;
+            coords(tile, nt, mt2, t);
+            const int row = (mt2 * 2 + (int)rank) * BM + q * 32 + lane;
+            const bool row_ok = row < p.M;
+            const int n0 = nt * BN;
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN;
+            auto wait_acc = [&]() -> bool {
+                bool ok = mbar_wait(&acc_full[a], aph, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) { if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_EPI_WAIT); *abort_flag = 1; } return false; }
+                tc_fence_after();
+                return true;
+            };
+            if (!epilogue<BN, EPI>(p, taddr, t, row, row_ok, n0, half, xpose + (warp - 2) * 4096, wait_acc)) break;
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&acc_empty[a]), 0));
+            if (++a == 2) { a = 0; aph ^= 1; }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                     // the partner's shared and tensor memory are in use until both are here
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * BN) : "memory");
+    }
+}
+
 typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -668,6 +844,39 @@ pt_status launch_t(const CUtensorMap& ta, const CUtensorMap& tb, GemmP p, cudaSt
     return PT_OK;
 }
 
+template <int EPI>
+pt_status launch_pair_t(const CUtensorMap& ta, const CUtensorMap& tb, GemmP p, cudaStream_t st, int sms) {
+    static int max_pairs = -1;
+    if (max_pairs < 0) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_tc_pair<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
+        if (e != cudaSuccess) { set_error("cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
+        cudaLaunchConfig_t q = {};
+        q.gridDim = dim3(sms & ~1); q.blockDim = dim3(kGemmThreads); q.dynamicSmemBytes = kGemmSmem;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension; at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        q.attrs = at; q.numAttrs = 1;
+        int n = 0;
+        e = cudaOccupancyMaxActiveClusters(&n, gemm_tc_pair<EPI>, &q);
+        if (e != cudaSuccess || n < 1) { set_error("cudaOccupancyMaxActiveClusters: %s (%d clusters)", cudaGetErrorString(e), n); cudaGetLastError(); return PT_ERR_CUDA; }
+        max_pairs = n;
+    }
+    p.a_tx = (uint32_t)std::min(BM, p.M) * BK * 2;
+    p.w_tx = (uint32_t)std::min(BM, p.N) * BK * 2;
+    p.tiles_n = (p.N + 255) / 256;
+    const int tiles = ((p.M + 2 * BM - 1) / (2 * BM)) * p.tiles_n * p.T;
+    const int pairs = std::min(tiles, max_pairs);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(kGemmThreads); cfg.dynamicSmemBytes = kGemmSmem; cfg.stream = st;
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeClusterDimension; at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization; at[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = 2;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_tc_pair<EPI>, ta, tb, p);
+    if (e != cudaSuccess) { set_error("GEMM (CTA pairs) launch: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return PT_OK;
+}
+
 }  // namespace
 
 pt_status make_map_bf16(CUtensorMap* out, const void* base, int64_t k, int64_t rows, int64_t tracks, int box_rows) {
@@ -687,6 +896,11 @@ pt_status make_map_bf16_strided(CUtensorMap* out, const void* base, int64_t k, i
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled failed with code %d (k=%lld rows=%lld tracks=%lld)", (int)r, (long long)k, (long long)rows, (long long)tracks); return PT_ERR_CUDA; }
     return PT_OK;
+}
+
+bool gemm_pair_ok(int bn, int M, int N) {
+    // two CTAs per 256 x 256 tile: worth it when there are many full row tiles (a prefill)
+    return bn == 256 && M >= 1024 && N >= 256;
 }
 
 int gemm_kps(int bn, int M, int K, int kt) {
@@ -762,6 +976,15 @@ pt_status launch_gemm(int epi, int bn, const CUtensorMap& ta, const CUtensorMap&
     p.a_tx = p.kps > 1 ? (uint32_t)p.kps * (uint32_t)stage_a_bytes(p.M) : (uint32_t)std::min(BM, p.M) * BK * 2;
     p.w_kb_bytes = (uint32_t)box_b * BK * 2;
     p.w_tx = (uint32_t)std::max(p.kps, 1) * p.w_kb_bytes;
+    if (p.pair) {          // tb holds 128-row boxes of W; see gemm_pair_ok
+        if (bn != 256) { set_error("the CTA-pair GEMM has 256-column tiles"); return PT_ERR_INVALID_ARG; }
+        switch (epi) {
+        case EPI_PLAIN: return launch_pair_t<EPI_PLAIN>(ta, tb, p, st, sms);
+        case EPI_QKV: return launch_pair_t<EPI_QKV>(ta, tb, p, st, sms);
+        case EPI_SWIGLU: return launch_pair_t<EPI_SWIGLU>(ta, tb, p, st, sms);
+        default: return launch_pair_t<EPI_RESID>(ta, tb, p, st, sms);
+        }
+    }
 #define CASE(BN_, E_) if (bn == BN_ && epi == E_) return launch_t<BN_, E_>(ta, tb, p, st, sms)
     CASE(64, EPI_PLAIN); CASE(64, EPI_SWIGLU); CASE(64, EPI_RESID);
     CASE(128, EPI_PLAIN); CASE(128, EPI_QKV); CASE(128, EPI_SWIGLU); CASE(128, EPI_RESID);

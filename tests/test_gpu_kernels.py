@@ -32,6 +32,11 @@ def _operands(T, M, N, K, seed):
     (1, 40, 96, 256, 64, False),          # N tail inside a 4-k-block copy, one stage per tile
     (1, 16, 48, 256, 64, False),          # N smaller than the tile: the W box is 48 rows
     (2, 3, 640, 1024, 0, False),          # library-chosen width and stage shape at decode size
+    (2, 1024, 512, 256, 256, False),      # CTA pairs on 256 x 256 tiles: full tiles, tracks in the grid
+    (1, 1100, 640, 320, 256, False),      # CTA pairs: ragged M (the odd CTA's last rows are past M), N tail of half a tile
+    (1, 1300, 256, 1376, 256, False),     # CTA pairs: last row tile has no rows for the odd CTA; K tail
+    (3, 1024, 256, 192, 256, True),       # CTA pairs with tracks folded into K
+    (1, 4096, 1024, 1024, 256, False),    # CTA pairs: more tiles than pairs, both accumulators in use
 ])
 def test_gemm_bf16_matches_definition(T, M, N, K, bn, fold):
     import torch
