@@ -898,9 +898,31 @@ pt_status make_map_bf16_strided(CUtensorMap* out, const void* base, int64_t k, i
     return PT_OK;
 }
 
+// Clusters of two CTAs with this kernel's shared memory must be launchable on the current device; asked once.
+static bool pair_launchable() {
+    static int state = -1;
+    if (state < 0) {
+        state = 0;
+        int dev = 0, sms = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (cudaFuncSetAttribute(gemm_tc_pair<EPI_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem) == cudaSuccess && sms >= 2) {
+            cudaLaunchConfig_t q = {};
+            q.gridDim = dim3(sms & ~1); q.blockDim = dim3(kGemmThreads); q.dynamicSmemBytes = kGemmSmem;
+            cudaLaunchAttribute at[1];
+            at[0].id = cudaLaunchAttributeClusterDimension; at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+            q.attrs = at; q.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, gemm_tc_pair<EPI_PLAIN>, &q) == cudaSuccess && n >= 1) state = 1;
+        }
+        cudaGetLastError();
+    }
+    return state == 1;
+}
+
 bool gemm_pair_ok(int bn, int M, int N) {
     // two CTAs per 256 x 256 tile: worth it when there are many full row tiles (a prefill)
-    return bn == 256 && M >= 1024 && N >= 256;
+    return bn == 256 && M >= 1024 && N >= 256 && pair_launchable();
 }
 
 int gemm_kps(int bn, int M, int K, int kt) {
