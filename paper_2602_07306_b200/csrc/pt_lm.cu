@@ -174,7 +174,7 @@ pt_status pt_lm_head(pt_model* m, const float* h, int64_t row_stride, int64_t n,
     const int bn = gemm_bn(V, (int)n, 1, EPI_PLAIN);
     CUtensorMap ta, tb;
     const int kps = gemm_kps(bn, (int)n, H, 1);
-    const bool pair = gemm_pair_ok(bn, (int)n, V);
+    const bool pair = gemm_pair_ok(bn, (int)n, V, 1);
     if ((s = make_a_map(&ta, hn, H, n, 1, kps)) != PT_OK) return s;
     if ((s = make_w_map(&tb, m->lm_buf + l.off_head, H, V, 1, pair ? 128 : bn, kps)) != PT_OK) return s;
     GemmP p{};

@@ -171,7 +171,7 @@ pt_status tc_forward(Call& k) {
             p.nq = g.heads; p.nkv = g.kv_heads; p.dh = m->dh; p.ps = c->ps;
             int bn = gemm_bn(p.N, M, T, EPI_QKV);
             p.kps = gemm_kps(bn, M, p.K, 1);
-            p.pair = gemm_pair_ok(bn, M, p.N);
+            p.pair = gemm_pair_ok(bn, M, p.N, p.T);
             if ((s = a_map(ta_h, hb, H, p.kps, &ta)) != PT_OK) return s;
             ProfScope ps(m, st, 1);
             if ((s = launch_gemm(EPI_QKV, bn, *ta, wm[l].m[0][bn_index(p.pair ? 128 : bn)][kps_index(p.kps)], p, st)) != PT_OK) return s;
@@ -190,7 +190,7 @@ pt_status tc_forward(Call& k) {
             p.ssq_out = w.ssq; p.ssq_out_tstride = (size_t)M * tiles; p.ssq_out_tiles = tiles;
             int bn = gemm_bn(p.N, M, T, EPI_RESID);
             p.kps = gemm_kps(bn, M, p.K, 1);
-            p.pair = gemm_pair_ok(bn, M, p.N);
+            p.pair = gemm_pair_ok(bn, M, p.N, p.T);
             if ((s = a_map(ta_o, o, m->QD, p.kps, &ta)) != PT_OK) return s;
             ProfScope ps(m, st, 2);
             if ((s = launch_gemm(EPI_RESID, bn, *ta, wm[l].m[1][bn_index(p.pair ? 128 : bn)][kps_index(p.kps)], p, st)) != PT_OK) return s;
@@ -204,7 +204,7 @@ pt_status tc_forward(Call& k) {
             p.z_out = z;
             int bn = gemm_bn(p.N, M, T, EPI_SWIGLU);
             p.kps = gemm_kps(bn, M, p.K, 1);
-            p.pair = gemm_pair_ok(bn, M, p.N);
+            p.pair = gemm_pair_ok(bn, M, p.N, p.T);
             if ((s = a_map(ta_h, hb, H, p.kps, &ta)) != PT_OK) return s;
             ProfScope ps(m, st, 3);
             if ((s = launch_gemm(EPI_SWIGLU, bn, *ta, wm[l].m[2][bn_index(p.pair ? 128 : bn)][kps_index(p.kps)], p, st)) != PT_OK) return s;
@@ -233,7 +233,7 @@ pt_status tc_forward(Call& k) {
             }
             int bn = gemm_bn(p.N, M, p.T, EPI_RESID);
             p.kps = gemm_kps(bn, M, p.K, p.kt);
-            p.pair = gemm_pair_ok(bn, M, p.N);
+            p.pair = gemm_pair_ok(bn, M, p.N, p.T);
             if ((s = a_map(ta_z, z, F, p.kps, &ta)) != PT_OK) return s;
             ProfScope ps(m, st, sync ? 5 : 4);
             if ((s = launch_gemm(EPI_RESID, bn, *ta, wm[l].m[3][bn_index(p.pair ? 128 : bn)][kps_index(p.kps)], p, st)) != PT_OK) return s;
@@ -279,7 +279,7 @@ extern "C" pt_status pt_kernel_gemm_bf16(const void* a, const void* w, void* c, 
     CUtensorMap ta, tb;
     pt_status s;
     const int kps = gemm_kps(bn, M, K, fold_tracks ? T : 1);
-    const bool pair = gemm_pair_ok(bn, M, N);
+    const bool pair = gemm_pair_ok(bn, M, N, fold_tracks ? 1 : T);
     if ((s = make_a_map(&ta, a, K, M, T, kps)) != PT_OK) return s;
     if ((s = make_w_map(&tb, w, K, N, T, pair ? 128 : bn, kps)) != PT_OK) return s;
     GemmP p{};

@@ -100,7 +100,7 @@ int gemm_bn(int N, int M, int T, int epi);
 // k-blocks per ring stage for a launch of M rows: more than one when the rows are few, so that a copy of W is 16-32 KB
 int gemm_kps(int bn, int M, int K, int kt);
 // whether a launch should use the CTA-pair kernel (then W's map is the one with 128-row boxes and kps = 1)
-bool gemm_pair_ok(int bn, int M, int N);
+bool gemm_pair_ok(int bn, int M, int N, int T);
 // tensor map of W [tracks][rows][k] for tiles of bn rows: 3-D (k, row, track) for kps = 1, else 4-D (64, row, k-block, track)
 pt_status make_w_map(CUtensorMap* out, const void* base, int64_t k, int64_t rows, int64_t tracks, int bn, int kps);
 // tensor map of A [tracks][rows][k] to go with it: 3-D with a box of min(rows, 128) rows for kps = 1, else 4-D with kps k-blocks per copy

@@ -37,6 +37,8 @@ def _operands(T, M, N, K, seed):
     (1, 1300, 256, 1376, 256, False),     # CTA pairs: last row tile has no rows for the odd CTA; K tail
     (3, 1024, 256, 192, 256, True),       # CTA pairs with tracks folded into K
     (1, 4096, 1024, 1024, 256, False),    # CTA pairs: more tiles than pairs, both accumulators in use
+    (2, 176, 768, 512, 0, False),         # a large decode batch: one 256-row pair tile whose odd CTA holds 48 rows
+    (3, 130, 256, 320, 0, False),         # the odd CTA holds two rows
 ])
 def test_gemm_bf16_matches_definition(T, M, N, K, bn, fold):
     import torch
