@@ -34,7 +34,7 @@ from paper_2602_07306_b200 import inputs as I  # noqa: E402
 # 8 sequences instead of 64, same kernel): dram read + write bytes per launch over the algorithmic K/V
 # bytes of that launch.  Traffic is proportional to the keys read, so a bench launch is scaled by its own
 # algorithmic bytes.  Set to None when the kernel changes until the counters are taken again.
-DECODE_ATTN_TRAFFIC_RATIO = (541.2e6 + 4.0e6) / 537.1e6
+DECODE_ATTN_TRAFFIC_RATIO = (541.24e6 + 4.18e6) / 537.13e6
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
