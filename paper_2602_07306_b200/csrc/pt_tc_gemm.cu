@@ -13,9 +13,16 @@
 //   EPI_PLAIN   fp32 C (kernel-level tests)
 // Epilogue data path: a warp owns 32 accumulator rows (its tensor-memory lane quarter); the two
 // warps of a quarter split the tile's columns.  tcgen05.ld hands every thread one row, and the
-// thread reads and writes whole 32-byte sectors of that row.  Global loads that do not depend on
-// the accumulator (row statistics, rotary table, residual rows) are issued before the wait for
-// the accumulator and one 32-column unit ahead, so their latency hides behind the tensor pipe.
+// thread reads and writes whole 32-byte sectors of that row (the residual epilogue, which moves
+// the most bytes, first turns each 32 x 32 unit through shared memory so that its global accesses
+// are 128 contiguous bytes per row).  Global loads that do not depend on the accumulator (row
+// statistics, rotary table, residual rows) are issued before the wait for the accumulator and one
+// 32-column unit ahead, so their latency hides behind the tensor pipe.
+// Three shapes of the same pipeline, chosen by the launch's row count (gemm_bn, gemm_kps,
+// gemm_pair_ok): gemm_tc with one k-block per ring stage; gemm_tc with stages of 2 or 4 k-blocks
+// and one 4-D copy of W and of A per stage (few rows: a decode step streams W from HBM);
+// gemm_tc_pair, two CTAs of a cluster on a 256 x 256 tile with tcgen05.mma.cta_group::2 (many
+// rows: halves the W bytes copied into each SM).  All are programmatic dependent launches.
 // Every mbarrier wait is bounded; on a timeout the CTA records PT_ERR_DEVICE_TIMEOUT, stops
 // issuing work, frees its tensor memory and exits.
 #include "pt_tc.h"
