@@ -90,6 +90,18 @@ pt_status pt_kernel_decode_attn_static(const void* q, const void* pool_l, int64_
                                        int32_t T, int32_t B, int32_t nq, int32_t nkv, int32_t dh, int32_t ps,
                                        int32_t num_pages, void* out, void* status, void* stream);
 
+/* ---- the bounded wait, exercised ------------------------------------------------------------
+ * Every device-side wait of the library (an mbarrier of a TMA -> MMA -> epilogue pipeline) gives up
+ * after a time limit (2 s of device time, whatever the iteration counts), records PT_ERR_DEVICE_TIMEOUT with
+ * a location code in the status block and lets its kernel wind down, so that the context stays usable.
+ * This entry point runs that same wait loop on a barrier at which nothing ever arrives, with the limit
+ * given here, in a one-CTA kernel on `stream`:
+ *   status    device, int32[16], zeroed by the caller; afterwards status[0] = PT_ERR_DEVICE_TIMEOUT and
+ *             status[1] = 20 (the self-test's location code)
+ *   limit_ns  how long the wait may last, 1 000 .. 1 000 000 000 (else PT_ERR_INVALID_ARG)
+ * Returns PT_OK once the kernel is enqueued (PT_ERR_CUDA if the launch failed). */
+pt_status pt_kernel_wait_selftest(void* status, uint64_t limit_ns, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

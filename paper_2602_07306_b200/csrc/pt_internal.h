@@ -26,7 +26,7 @@ enum : int {
     LOC_GEMM_EPI_WAIT = 5, LOC_GEMM_EMPTY_WAIT = 6, LOC_DECODE_PAGE = 7, LOC_FLASH_PAGE = 8,
     LOC_GEMM_ACC_WAIT = 9,
     LOC_FLASH_KEMPTY = 10, LOC_FLASH_VEMPTY = 11, LOC_FLASH_VRAW = 12, LOC_FLASH_KFULL = 13, LOC_FLASH_QFULL = 14,
-    LOC_EMBED_TOKEN = 19,
+    LOC_EMBED_TOKEN = 19, LOC_SELFTEST_WAIT = 20,
     LOC_FLASH_PFULL = 15, LOC_FLASH_VFULL = 16, LOC_FLASH_SFULL = 17, LOC_FLASH_OREADY = 18,
 };
 

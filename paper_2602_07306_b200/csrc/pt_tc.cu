@@ -434,3 +434,10 @@ extern "C" pt_status pt_kernel_decode_attn_static(const void* q, const void* poo
     return decode_attn_with_scratch(q, pool_l, pool_track_stride, block_table, maxp, kv_len, T, B, nq, nkv, dh, ps,
                                     num_pages, out, (char*)g_static_scratch_addr[dev], status, (cudaStream_t)stream);
 }
+
+extern "C" pt_status pt_kernel_wait_selftest(void* status, uint64_t limit_ns, void* stream) {
+    using namespace pt;
+    if (!status) { set_error("null status"); return PT_ERR_INVALID_ARG; }
+    if (limit_ns < 1000 || limit_ns > 1000000000ull) { set_error("limit_ns must be in [1e3, 1e9]"); return PT_ERR_INVALID_ARG; }
+    return launch_wait_selftest((int*)status, (unsigned long long)limit_ns, (cudaStream_t)stream);
+}

@@ -71,6 +71,21 @@ struct AttnP {
 // its wait sees the results of every launch before it.  In a kernel launched the ordinary way both
 // calls do nothing.
 #ifdef __CUDACC__
+// Every wait in these kernels is a loop of mbarrier.try_wait (which itself suspends the thread for a hardware-chosen
+// while) with an iteration limit; the iteration limit alone does not bound the time, so each loop also gives up once
+// WaitClock::expired() says that more than kWaitLimitNs have passed since its first slow poll.  A wait that gives up
+// records PT_ERR_DEVICE_TIMEOUT and the kernel winds down.
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;        // 2 s: far beyond any wait of a healthy launch
+struct WaitClock {
+    unsigned long long t0 = 0;
+    __device__ __forceinline__ static unsigned long long now() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+    // call every few hundred polls
+    __device__ __forceinline__ bool expired(unsigned long long limit_ns = kWaitLimitNs) {
+        const unsigned long long t = now();
+        if (t0 == 0) { t0 = t; return false; }
+        return t - t0 > limit_ns;
+    }
+};
 __device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
@@ -111,6 +126,9 @@ pt_status launch_gemm(int epi, int bn, const CUtensorMap& ta, const CUtensorMap&
 // pt_simt.cu
 void tap_copy(Call& k, int layer, int point, const float* src, size_t src_tstride);
 void launch_simt_attn_bf16(Call& k, const __nv_bfloat16* q, int q_row_stride, const __nv_bfloat16* pool_l, __nv_bfloat16* o);
+
+// pt_tc_gemm.cu: a one-CTA kernel that waits on an mbarrier nothing arrives at, with the kernels' own wait loop and a short limit
+pt_status launch_wait_selftest(int* status, unsigned long long limit_ns, cudaStream_t st);
 
 // pt_tc_flash.cu
 bool flash_tc_supported(int dh, int ps);

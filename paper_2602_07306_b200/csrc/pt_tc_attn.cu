@@ -380,7 +380,13 @@ k_decode_attn_tma(const __grid_constant__ CUtensorMap kvmap, const AttnP p) {
         const int slot = it % kDecStages;
         const uint32_t parity = (it / kDecStages) & 1;
         bool ok = false;
-        for (uint32_t spin = 0; spin < kDecSpin; ++spin) if (mbar_try(&wbar[slot], parity)) { ok = true; break; }
+        {
+            WaitClock clock;
+            for (uint32_t spin = 0; spin < kDecSpin; ++spin) {
+                if (mbar_try(&wbar[slot], parity)) { ok = true; break; }
+                if ((spin & 255) == 255 && clock.expired()) break;
+            }
+        }
         if (!__all_sync(0xffffffffu, ok)) { timed_out = true; break; }
         const uint32_t k_base = smem_u32(ring + slot * SLOT_BYTES), v_base = k_base + PAGE_BYTES;
         const int key0 = kstart + gi * 16;
@@ -449,8 +455,12 @@ k_decode_attn_tma(const __grid_constant__ CUtensorMap kvmap, const AttnP p) {
     }
     if (timed_out) {
         // give the copies this warp still has in flight a bounded chance to land, then give up
+        WaitClock clock;
         for (int s2 = 0; s2 < kDecStages; ++s2)
-            for (uint32_t spin = 0; spin < (1u << 16); ++spin) if (mbar_try(&wbar[s2], 0) || mbar_try(&wbar[s2], 1)) break;
+            for (uint32_t spin = 0; spin < (1u << 16); ++spin) {
+                if (mbar_try(&wbar[s2], 0) || mbar_try(&wbar[s2], 1)) break;
+                if ((spin & 63) == 63 && clock.expired(100000000ull)) break;
+            }
         if (lane == 0) report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_DECODE_PAGE);
     }
     if (bad_page) report(p.status, PT_ERR_DEVICE_BOUNDS, LOC_DECODE_PAGE);

@@ -47,10 +47,11 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
 // `relaxed` waits (the copy warp's, which run stages ahead of their consumers) back off between polls:
 // a spinning warp costs issue slots and power; the softmax and MMA hand-offs poll at full rate.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, bool relaxed = false) {
+    WaitClock clock;
     for (uint32_t i = 0; i < kSpin; ++i) {
         if (mbar_try(bar, parity)) return true;
         if (relaxed && i >= 2) __nanosleep(128);
-        if ((i & 1023) == 1023 && *abort_flag) return false;
+        if ((i & 255) == 255 && (*abort_flag || clock.expired())) return false;
     }
     return false;
 }

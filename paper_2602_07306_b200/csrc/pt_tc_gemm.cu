@@ -54,11 +54,12 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait: false when the limit ran out or another warp already gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, unsigned long long limit_ns = kWaitLimitNs) {
+    WaitClock clock;
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         if (mbar_try(bar, parity)) return true;
         if (i >= 4) __nanosleep(64);                       // back off: a spinning warp costs issue slots and power
-        if ((i & 1023) == 1023 && *abort_flag) return false;
+        if ((i & 255) == 255 && (*abort_flag || clock.expired(limit_ns))) return false;
     }
     return false;
 }
@@ -813,6 +814,19 @@ gemm_tc_pair(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUt
     }
 }
 
+// One CTA, one mbarrier that nothing arrives at: the wait must give up after limit_ns, record the timeout and return.
+__global__ void k_wait_selftest(int* status, unsigned long long limit_ns) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_word;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_word = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && !mbar_wait(&bar, 0, &abort_word, limit_ns)) report(status, PT_ERR_DEVICE_TIMEOUT, LOC_SELFTEST_WAIT);
+}
+
 typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -931,6 +945,14 @@ static bool pair_launchable() {
 // 176 tiles 11 % faster, QKV with 48 tiles 3 %, the projections back to the hidden size with 32 tiles 20 % slower).
 static bool enough_pair_tiles(int N, int M, int T) {
     return M > 128 && N >= 256 && (int64_t)((M + 255) / 256) * ((N + 255) / 256) * T >= 40;
+}
+
+pt_status launch_wait_selftest(int* status, unsigned long long limit_ns, cudaStream_t st) {
+    k_wait_selftest<<<1, 32, 0, st>>>(status, limit_ns);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_error("kernel launch failed: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return PT_OK;
 }
 
 bool gemm_pair_ok(int bn, int M, int N, int T) {

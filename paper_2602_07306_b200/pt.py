@@ -78,6 +78,7 @@ _PROTOS = {
                                      _P, _P, _SZ, _P, _P]),
     "pt_kernel_decode_attn_static": (_I32, [_P, _P, _I64, _P, _I32, C.POINTER(_I32), _I32, _I32, _I32, _I32, _I32, _I32, _I32,
                                             _P, _P, _P]),
+    "pt_kernel_wait_selftest": (_I32, [_P, C.c_uint64, _P]),
     "pt_last_error": (C.c_char_p, []),
 }
 EXPORTS = tuple(_PROTOS)
@@ -417,6 +418,15 @@ def kernel_gemm_bf16(a, w, bn: int = 0, fold_tracks: bool = False):
         check(lib().pt_kernel_gemm_bf16(a.data_ptr(), w.data_ptr(), c.data_ptr(), T, M, N, K, bn, int(fold_tracks),
                                         status.data_ptr(), torch.cuda.current_stream().cuda_stream))
     return c, status
+
+
+def kernel_wait_selftest(limit_ns: int, device="cuda:0"):
+    """Run the library's bounded wait on a barrier nothing arrives at; returns the status block (int32[16], CUDA)."""
+    import torch
+    status = torch.zeros(16, dtype=torch.int32, device=device)
+    with torch.cuda.device(status.device):
+        check(lib().pt_kernel_wait_selftest(status.data_ptr(), int(limit_ns), torch.cuda.current_stream().cuda_stream))
+    return status
 
 
 def kernel_decode_attn(q, pool_l, block_table, kv_len, *, nq, nkv, dh, ps, scratch=None):

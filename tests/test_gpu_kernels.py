@@ -176,3 +176,27 @@ def test_prefill_attention_kernel_matches_oracle(T, B, S, nq, nkv, dh, ps, start
     assert np.all(np.isfinite(got))
     d = np.abs(got - ref)
     assert d.max() <= 2e-2 * np.abs(ref).max() and d.mean() <= 4e-3 * np.abs(ref).mean(), (d.max() / np.abs(ref).max(), d.mean() / np.abs(ref).mean())
+
+
+def test_a_wait_that_nothing_ends_gives_up_in_time_and_leaves_the_context_usable():
+    """The library's device-side waits are bounded in time: the self-test waits on a barrier at which nothing
+    arrives, must come back after its limit with PT_ERR_DEVICE_TIMEOUT in the status block, and the next launch
+    on the same context must still work (no trap, no fault, no endless spin)."""
+    import time
+    import torch
+    from paper_2602_07306_b200 import pt
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    status = pt.kernel_wait_selftest(20_000_000)             # 20 ms
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    assert status[:2].tolist() == [9, 20], status[:4].tolist()      # PT_ERR_DEVICE_TIMEOUT, the self-test's location code
+    assert 0.015 <= dt < 1.0, dt
+    with pytest.raises(pt.PtError):
+        pt.kernel_wait_selftest(10)                          # below the accepted range: refused on the host
+    a, w = _operands(1, 64, 64, 64, seed=1)
+    c, st = pt.kernel_gemm_bf16(torch.from_numpy(a).cuda().to(torch.bfloat16), torch.from_numpy(w).cuda().to(torch.bfloat16))
+    torch.cuda.synchronize()
+    assert st[:2].tolist() == [0, 0]
+    ref = np.einsum("tmk,tnk->tmn", a.astype(np.float64), w.astype(np.float64))
+    assert np.abs(c.cpu().numpy() - ref).max() <= 1e-4 * np.abs(ref).max() + 1e-6
