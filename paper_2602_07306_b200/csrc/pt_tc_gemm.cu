@@ -240,8 +240,8 @@ __device__ __forceinline__ bool epi_swiglu(const GemmP& p, uint32_t taddr, int t
 }
 
 // A unit is 32 accumulator columns of one head: for q and k heads the 16 columns j0..j0+15 and
-// their rotary partners j0+dh/2.., for v heads 32 consecutive columns.  The 16 (cos, sin) pairs
-// of the row's position (fp16, 64 bytes) are fetched one unit ahead.
+// their rotary partners j0+dh/2.., for v heads 32 consecutive columns.  The (cos, sin) pairs of the
+// row's position (fp16, 64 bytes per slice) are fetched before the wait for the accumulator.
 template <int BN, class Wait>
 __device__ __forceinline__ bool epi_qkv(const GemmP& p, uint32_t taddr, int t, int row, bool row_ok, int n0, int half, Wait wait) {
     constexpr int UNITS = BN / 32;                        // units of the tile, alternating between the two warps
@@ -253,27 +253,32 @@ __device__ __forceinline__ bool epi_qkv(const GemmP& p, uint32_t taddr, int t, i
     const bool slot_ok = row_ok && kvoff >= 0 && kvoff + (int64_t)(2 * p.nkv - 1) * p.ps * dh + dh <= p.slab_elems;
     if (row_ok && !slot_ok) report(p.status, PT_ERR_DEVICE_BOUNDS, LOC_ROPE_PAGE);
     const float* csr = reinterpret_cast<const float*>(p.cs16 + (size_t)pos * halfdh);   // (cos, sin) fp16 pairs, moved as 32-bit words
-    auto fetch = [&](int u, float* tab) {                 // tab[i] = packed (cos, sin) of column j0 + i
-        const int hs = n0 / dh + u / upd;
-        if (hs >= p.nq + p.nkv || !row_ok) return;         // v heads, columns past N, rows past M: no rotation
-        const int j0 = (u % upd) * 16;
+    // tab[i] = packed (cos, sin) of column j0 + i for the row's position.  The slice depends on the unit's place inside
+    // its head (sub = u % upd), not on the head, and a warp's units u = half, half + 2, ... only ever have the places
+    // sub0 = half % upd and sub1 = (half + 2) % upd: both slices are fetched once per tile, before the wait for the
+    // accumulator, instead of once per unit.
+    auto fetch = [&](int sub, float* tab) {
+        if (!row_ok) return;
+        const int j0 = sub * 16;
         ld256(csr + j0, tab); ld256(csr + j0 + 8, tab + 8);
     };
-    float tab[16], nxt[16];
-    fetch(half, tab);
+    const bool rotates = n0 / dh < p.nq + p.nkv;          // the tile starts in a q or k head (v heads are not rotated)
+    const int sub0 = half % upd, sub1 = (half + 2) % upd;
+    float tab0[16], tab1[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) { tab0[i] = 0.f; tab1[i] = 0.f; }
+    if (rotates) { fetch(sub0, tab0); if (sub1 != sub0) fetch(sub1, tab1); }
     if (!wait()) return false;
-#pragma unroll 1
-    for (int u = half; u < UNITS; u += 2) {
+    auto unit = [&](int u, const float* tab) -> bool {     // false: past the last head (uniform across the warp)
         const int hc = u / upd, sub = u % upd;
         const int hs = n0 / dh + hc;                       // head slot: q heads, then k heads, then v heads
-        if (hs >= heads_total) break;                      // uniform across the warp
+        if (hs >= heads_total) return false;
         const bool is_v = hs >= p.nq + p.nkv;
         float lo[16], hi[16];
         const int c_lo = hc * dh + (is_v ? sub * 32 : sub * 16);
         const int c_hi = is_v ? c_lo + 16 : c_lo + halfdh;
         tc_ld16(taddr + c_lo, lo);
         tc_ld16(taddr + c_hi, hi);
-        if (u + 2 < UNITS) fetch(u + 2, nxt);
         __nv_bfloat16* dst;
         bool st_ok;
         if (hs < p.nq) {
@@ -304,8 +309,12 @@ __device__ __forceinline__ bool epi_qkv(const GemmP& p, uint32_t taddr, int t, i
                 store16_bf16(dst + sub * 32 + 16, hi);
             }
         }
-#pragma unroll
-        for (int i = 0; i < 16; ++i) tab[i] = nxt[i];      // last: the fetch stays in flight until here
+        return true;
+    };
+#pragma unroll 1
+    for (int u = half; u < UNITS; u += 4) {                // two units per turn: places sub0 and sub1
+        if (!unit(u, tab0)) break;
+        if (u + 2 < UNITS && !unit(u + 2, sub1 != sub0 ? tab1 : tab0)) break;
     }
     return true;
 }
