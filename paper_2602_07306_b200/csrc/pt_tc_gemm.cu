@@ -823,6 +823,225 @@ gemm_tc_pair(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUt
     }
 }
 
+// The same pair kernel for the plain residual epilogue (one residual stream in, one track's operand out), with the
+// epilogue's global traffic on the TMA unit instead of the load/store unit: per 32 x 32 unit a warp receives the residual
+// rows as one 4 KB box in shared memory, adds them row-per-thread (128-byte swizzled, conflict-free), puts the fp32 result
+// and the gain-scaled bf16 copy back into shared memory and stores both as boxes.  The shared memory for it (10 KB per
+// epilogue warp) comes from the ring: four stages.
+constexpr int kRtStages = 4;
+constexpr int kRtStageBytes = 10 * 1024;                     // per epilogue warp: residual in 4 KB, fp32 out 4 KB, bf16 out 2 KB
+
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3}], [%4];"
+                 ::"l"((uint64_t)map), "r"(c0), "r"(c1), "r"(c2), "r"(src) : "memory");
+}
+
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_tc_pair_resid(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensorMap tb,
+                   const __grid_constant__ CUtensorMap th_in, const __grid_constant__ CUtensorMap th_out,
+                   const __grid_constant__ CUtensorMap thb, const GemmP p) {
+    constexpr int BN = 256;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t* staging = smem + kRtStages * kPairStageBytes;
+    uint64_t* full = (uint64_t*)(smem + kRingBytes + kXposeBytes);
+    uint64_t* empty = full + kMaxStages;
+    uint64_t* acc_full = empty + kMaxStages;
+    uint64_t* acc_empty = acc_full + 2;
+    uint32_t* tmem_slot = (uint32_t*)(acc_empty + 2);
+    volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+    uint64_t* inbar = (uint64_t*)(tmem_slot + 2);           // one per epilogue warp: its residual box has landed
+    const uint32_t rank = cluster_rank();                   // 0: issues the MMAs; 1: its partner
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kRtStages; ++s) { mbar_init(&full[s], 2); mbar_init(&empty[s], 1); }
+        for (int w = 0; w < kEpiWarps; ++w) mbar_init(&inbar[w], 1);
+        for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 2 * kEpiWarps); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {                                        // the same warp of both CTAs, the same slot address
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(2 * BN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                     // both CTAs' barriers exist before anything arrives at them
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int tiles_m2 = (p.M + 2 * BM - 1) / (2 * BM);     // row tiles of 256
+    const int num_tiles = tiles_m2 * p.tiles_n * p.T;
+    const int kpb = (p.K + BK - 1) / BK;
+    const int kblocks = kpb * p.kt;
+    const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+    auto coords = [&](int tile, int& nt, int& mt2, int& t) { nt = tile % p.tiles_n; mt2 = (tile / p.tiles_n) % tiles_m2; t = tile / (p.tiles_n * tiles_m2); };
+    grid_dep_wait();
+    if (threadIdx.x == 0) grid_dep_launch();
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int s = 0; uint32_t ph = 0;
+            bool ok = true;
+            for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
+                int nt, mt2, t;
+                coords(tile, nt, mt2, t);
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_EMPTY_WAIT); *abort_flag = 1; break; }
+                    const int tt = p.kt > 1 ? kb / kpb : t;
+                    const int k0 = (p.kt > 1 ? kb % kpb : kb) * BK;
+                    uint8_t* sa = smem + s * kPairStageBytes;
+                    const uint32_t fb = map_to_cta(smem_u32(&full[s]), 0);
+                    mbar_expect_tx_cluster(fb, p.a_tx + p.w_tx);
+                    tma_load_3d_pair(sa, &ta, fb, k0, (mt2 * 2 + (int)rank) * BM, tt);
+                    tma_load_3d_pair(sa + BM * BK * 2, &tb, fb, k0, nt * BN + (int)rank * (BN / 2), tt);
+                    if (++s == kRtStages) { s = 0; ph ^= 1; }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (rank == 0) {
+            constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+            const uint64_t desc0 = smem_desc(smem_u32(smem));
+            int s = 0; uint32_t ph = 0;
+            int a = 0; uint32_t aph = 0;
+            bool ok = true;
+            for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
+                if (!__all_sync(0xffffffffu, mbar_wait(&acc_empty[a], aph ^ 1, abort_flag))) {
+                    if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_ACC_WAIT); *abort_flag = 1; }
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + a * BN;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!__all_sync(0xffffffffu, mbar_wait(&full[s], ph, abort_flag))) {
+                        ok = false;
+                        if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_TMA_WAIT); *abort_flag = 1; }
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint64_t da = desc0 + (uint64_t)((s * kPairStageBytes) >> 4), db = da + (uint64_t)((BM * BK * 2) >> 4);
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)
+                        tc_mma_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+                    tc_commit_pair(smem_u32(&empty[s]));                        // both CTAs may refill the stage
+                    tc_commit_pair(map_to_cta(smem_u32(&empty[s]), 1));
+                    if (++s == kRtStages) { s = 0; ph ^= 1; }
+                }
+                if (!ok) break;
+                tc_commit_pair(smem_u32(&acc_full[a]));                         // both CTAs' epilogues may drain
+                tc_commit_pair(map_to_cta(smem_u32(&acc_full[a]), 1));
+                if (++a == 2) { a = 0; aph ^= 1; }
+            }
+        }
+        __syncwarp();
+    } else {
+        const int q = warp & 3;
+        const int half = (warp - 2) >> 2;
+        const int ew = warp - 2;
+        uint8_t* stg = staging + ew * kRtStageBytes;
+        const uint32_t s_in = smem_u32(stg), s_out = s_in + 4096, s_outb = s_in + 8192;
+        uint64_t* ib = &inbar[ew];
+        uint32_t inph = 0;
+        bool in_flight = false;                                            // a residual box has been requested and not yet consumed
+        constexpr int UNITS = BN / 32;
+        int a = 0; uint32_t aph = 0;
+        bool ok = true;
+        for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
+            int nt, mt2, t;
+            coords(tile, nt, mt2, t);
+            const int r0 = (mt2 * 2 + (int)rank) * BM + q * 32;          // first of this warp's 32 rows
+            const int row = r0 + lane;
+            const bool row_ok = row < p.M;
+            const int n0 = nt * BN;
+            const int t_in = p.h_in_tstride ? t : 0, t_out = p.h_out_tstride ? t : 0;
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN;
+            auto issue_in = [&](int u) {                                   // residual rows of unit u: one box
+                if (lane == 0) { mbar_expect_tx(ib, 4096); tma_load_3d(stg, &th_in, ib, n0 + u * 32, r0, t_in); }
+                in_flight = true;
+            };
+            const int u_first = 2 * half;
+            if (n0 + u_first * 32 < p.N) issue_in(u_first);
+            {
+                bool w = mbar_wait(&acc_full[a], aph, abort_flag);
+                w = __all_sync(0xffffffffu, w);
+                if (!w) { if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_EPI_WAIT); *abort_flag = 1; } break; }
+                tc_fence_after();
+            }
+            float ssq = 0.f;
+#pragma unroll 1
+            for (int u = u_first; u < UNITS; u += (u & 1) ? 3 : 1) {       // units 0,1, 4,5, ... or 2,3, 6,7, ...
+                const int c = u * 32, col = n0 + c;
+                if (col >= p.N) break;                                      // uniform across the warp
+                float v[32], h[32];
+                tc_ld16(taddr + c, v);
+                tc_ld16(taddr + c + 16, v + 16);
+                if (!__all_sync(0xffffffffu, mbar_wait(ib, inph, abort_flag))) {
+                    if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_EPI_WAIT); *abort_flag = 1; }
+                    ok = false; break;
+                }
+                inph ^= 1;
+                in_flight = false;
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(h[4 * j]), "=f"(h[4 * j + 1]), "=f"(h[4 * j + 2]), "=f"(h[4 * j + 3])
+                                 : "r"(s_in + lane * 128 + ((j ^ (lane & 7)) << 4)) : "memory");
+                __syncwarp();                                               // every lane has its residual row: the box is free
+                const int un = u + ((u & 1) ? 3 : 1);
+                if (un < UNITS && n0 + un * 32 < p.N) issue_in(un);
+                tc_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) { v[i] = (v[i] + h[i]) * p.scale; if (row_ok) ssq += v[i] * v[i]; }
+                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the previous unit's stores have read their boxes
+                __syncwarp();
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(s_out + lane * 128 + ((j ^ (lane & 7)) << 4)),
+                                 "f"(v[4 * j]), "f"(v[4 * j + 1]), "f"(v[4 * j + 2]), "f"(v[4 * j + 3]) : "memory");
+                if (p.hb_out) {
+                    const float4* gp = (const float4*)(p.gain + (size_t)t * p.N + col);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {                          // 16-byte chunks of 8 bf16, 64-byte swizzle
+                        const float4 g0 = col + 8 * j < p.N ? gp[2 * j] : make_float4(0.f, 0.f, 0.f, 0.f);
+                        const float4 g1 = col + 8 * j < p.N ? gp[2 * j + 1] : make_float4(0.f, 0.f, 0.f, 0.f);
+                        const float* w = v + 8 * j;
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(s_outb + lane * 64 + ((j ^ ((lane >> 1) & 3)) << 4)),
+                                     "r"(pack_bf16(w[0] * g0.x, w[1] * g0.y)), "r"(pack_bf16(w[2] * g0.z, w[3] * g0.w)),
+                                     "r"(pack_bf16(w[4] * g1.x, w[5] * g1.y)), "r"(pack_bf16(w[6] * g1.z, w[7] * g1.w)) : "memory");
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0 && r0 < p.M) {                               // rows and columns past the ends are clipped by the copy
+                    tma_store_3d(&th_out, s_out, col, r0, t_out);
+                    if (p.hb_out) tma_store_3d(&thb, s_outb, col, r0, t);
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                }
+                if ((u & 1) == 1 || col + 32 >= p.N) {                     // a kSsqTile-column group is complete
+                    if (row_ok && p.ssq_out) p.ssq_out[(size_t)t * p.ssq_out_tstride + (size_t)row * p.ssq_out_tiles + col / kSsqTile] = ssq;
+                    ssq = 0.f;
+                }
+            }
+            if (!ok) break;
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&acc_empty[a]), 0));
+            if (++a == 2) { a = 0; aph ^= 1; }
+        }
+        if (in_flight) mbar_wait(ib, inph, abort_flag);                     // only after a time-out elsewhere: let the copy land before the CTA ends
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // every store of this warp has completed
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                     // the partner's shared and tensor memory are in use until both are here
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * BN) : "memory");
+    }
+}
+
 // One CTA, one mbarrier that nothing arrives at: the wait must give up after limit_ns, record the timeout and return.
 __global__ void k_wait_selftest(int* status, unsigned long long limit_ns) {
     __shared__ uint64_t bar;
@@ -905,6 +1124,69 @@ pt_status launch_pair_t(const CUtensorMap& ta, const CUtensorMap& tb, GemmP p, c
     if (e != cudaSuccess) { set_error("GEMM (CTA pairs) launch: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return PT_OK;
+}
+
+// 3-D map (column, row, track) of a row-major [tracks][rows][cols] array with 32 x 32 boxes for the epilogue's copies
+pt_status make_box_map(CUtensorMap* out, bool bf16, const void* base, int64_t cols, int64_t rows, int64_t tracks, int64_t tstride_elems) {
+    EncodeFn enc = get_encode();
+    if (!enc) { set_error("cuTensorMapEncodeTiled is not available from this driver"); return PT_ERR_CUDA; }
+    const int es = bf16 ? 2 : 4;
+    cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)tracks};
+    cuuint64_t strides[2] = {(cuuint64_t)cols * es, (cuuint64_t)(tracks > 1 ? tstride_elems : cols * rows) * es};
+    cuuint32_t box[3] = {32, 32, 1};
+    cuuint32_t ones[3] = {1, 1, 1};
+    CUresult r = enc(out, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, ones,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled (epilogue boxes) failed with code %d (cols=%lld rows=%lld tracks=%lld)", (int)r, (long long)cols, (long long)rows, (long long)tracks); return PT_ERR_CUDA; }
+    return PT_OK;
+}
+
+// The plain residual epilogue on CTA pairs with its global traffic on the TMA unit; the caller has checked resid_by_tma().
+pt_status launch_pair_resid(const CUtensorMap& ta, const CUtensorMap& tb, GemmP p, cudaStream_t st, int sms) {
+    static int max_pairs = -1;
+    if (max_pairs < 0) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_tc_pair_resid, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
+        if (e != cudaSuccess) { set_error("cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
+        cudaLaunchConfig_t q = {};
+        q.gridDim = dim3(sms & ~1); q.blockDim = dim3(kGemmThreads); q.dynamicSmemBytes = kGemmSmem;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension; at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        q.attrs = at; q.numAttrs = 1;
+        int n = 0;
+        e = cudaOccupancyMaxActiveClusters(&n, gemm_tc_pair_resid, &q);
+        if (e != cudaSuccess || n < 1) { set_error("cudaOccupancyMaxActiveClusters: %s (%d clusters)", cudaGetErrorString(e), n); cudaGetLastError(); return PT_ERR_CUDA; }
+        max_pairs = n;
+    }
+    CUtensorMap th_in, th_out, thb;
+    pt_status s;
+    if ((s = make_box_map(&th_in, false, p.h_in, p.N, p.M, p.h_in_tstride ? p.T : 1, (int64_t)p.h_in_tstride)) != PT_OK) return s;
+    if ((s = make_box_map(&th_out, false, p.h_out, p.N, p.M, p.h_out_tstride ? p.T : 1, (int64_t)p.h_out_tstride)) != PT_OK) return s;
+    if (p.hb_out) { if ((s = make_box_map(&thb, true, p.hb_out, p.N, p.M, p.T, (int64_t)p.M * p.N)) != PT_OK) return s; }
+    else thb = th_out;
+    p.a_tx = (uint32_t)std::min(BM, p.M) * BK * 2;
+    p.w_tx = (uint32_t)std::min(BM, p.N) * BK * 2;
+    p.tiles_n = (p.N + 255) / 256;
+    const int tiles = ((p.M + 2 * BM - 1) / (2 * BM)) * p.tiles_n * p.T;
+    const int pairs = std::min(tiles, max_pairs);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(kGemmThreads); cfg.dynamicSmemBytes = kGemmSmem; cfg.stream = st;
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeClusterDimension; at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization; at[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = 2;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_tc_pair_resid, ta, tb, th_in, th_out, thb, p);
+    if (e != cudaSuccess) { set_error("GEMM (CTA pairs, residual by TMA) launch: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return PT_OK;
+}
+
+static bool resid_by_tma(const GemmP& p) {
+    // One residual stream, this track's operand only, whole 16-byte pieces per row, many rows - and a short K: the four-stage
+    // ring costs a main-loop-bound GEMM more than the epilogue gains (measured at the cfg3 width: out-projection, K = 1024,
+    // 730 -> 888 TFLOP/s; down, K = 2816, 9 % slower)
+    return p.n_sum == 1 && p.n_out == 1 && p.kt == 1 && p.K <= 2048 && p.N % 4 == 0 && p.M >= 1024 && p.h_in && p.h_out
+        && ((uintptr_t)p.h_in % 16) == 0 && ((uintptr_t)p.h_out % 16) == 0 && (p.h_in_tstride % 4) == 0 && (p.h_out_tstride % 4) == 0;
 }
 
 }  // namespace
@@ -1051,7 +1333,7 @@ pt_status launch_gemm(int epi, int bn, const CUtensorMap& ta, const CUtensorMap&
         case EPI_PLAIN: return launch_pair_t<EPI_PLAIN>(ta, tb, p, st, sms);
         case EPI_QKV: return launch_pair_t<EPI_QKV>(ta, tb, p, st, sms);
         case EPI_SWIGLU: return launch_pair_t<EPI_SWIGLU>(ta, tb, p, st, sms);
-        default: return launch_pair_t<EPI_RESID>(ta, tb, p, st, sms);
+        default: return resid_by_tma(p) ? launch_pair_resid(ta, tb, p, st, sms) : launch_pair_t<EPI_RESID>(ta, tb, p, st, sms);
         }
     }
 #define CASE(BN_, E_) if (bn == BN_ && epi == E_) return launch_t<BN_, E_>(ta, tb, p, st, sms)
