@@ -657,7 +657,7 @@ gemm_tc(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensor
 // Barriers live at the same shared-memory offsets in both CTAs.  The even CTA's full[s] collects both
 // CTAs' copies (two arrivals with expected bytes); after the MMAs of a stage it commits to both CTAs'
 // empty[s], after a tile to both CTAs' acc_full[a]; the epilogue warps of both CTAs arrive at the even
-// CTA's acc_empty[a].  No copy is multicast.  Every wait is bounded as in gemm_tc.
+// CTA's acc_empty[a].  Every copy has exactly one destination CTA.  Every wait is bounded as in gemm_tc.
 constexpr int kPairStages = 6;
 constexpr int kPairStageBytes = 2 * BM * BK * 2;             // 128 rows of A + 128 rows of W per k-block
 
