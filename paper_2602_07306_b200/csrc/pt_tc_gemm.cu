@@ -1182,10 +1182,10 @@ pt_status launch_pair_resid(const CUtensorMap& ta, const CUtensorMap& tb, GemmP 
 }
 
 static bool resid_by_tma(const GemmP& p) {
-    // One residual stream, this track's operand only, whole 16-byte pieces per row, many rows - and a short K: the four-stage
+    // One residual stream, this track's operand only, whole 32-column units, many rows - and a short K: the four-stage
     // ring costs a main-loop-bound GEMM more than the epilogue gains (measured at the cfg3 width: out-projection, K = 1024,
     // 730 -> 888 TFLOP/s; down, K = 2816, 9 % slower)
-    return p.n_sum == 1 && p.n_out == 1 && p.kt == 1 && p.K <= 2048 && p.N % 4 == 0 && p.M >= 1024 && p.h_in && p.h_out
+    return p.n_sum == 1 && p.n_out == 1 && p.kt == 1 && p.K <= 2048 && p.N % 32 == 0 && p.M >= 1024 && p.h_in && p.h_out
         && ((uintptr_t)p.h_in % 16) == 0 && ((uintptr_t)p.h_out % 16) == 0 && (p.h_in_tstride % 4) == 0 && (p.h_out_tstride % 4) == 0;
 }
 
