@@ -33,8 +33,25 @@ from paper_2602_07306_b200 import inputs as I  # noqa: E402
 # DRAM traffic of k_decode_attn_tma<128> from its ncu capture (profiles/decode_attn_tma_T8_B8_kv2049.md:
 # 8 sequences instead of 64, same kernel): dram read + write bytes per launch over the algorithmic K/V
 # bytes of that launch.  Traffic is proportional to the keys read, so a bench launch is scaled by its own
-# algorithmic bytes.  Set to None when the kernel changes until the counters are taken again.
+# algorithmic bytes.  The counters belong to one version of the kernel's source file: its SHA-256 is kept
+# beside them, and when the file on disk differs the bench reports "traffic": null with the reason.
 DECODE_ATTN_TRAFFIC_RATIO = (541.24e6 + 4.18e6) / 537.13e6
+DECODE_ATTN_TRAFFIC_SOURCE = ("paper_2602_07306_b200/csrc/pt_tc_attn.cu",
+                              "03c6e8b160838ab3fdff043f52a2a4395f8d007ab509076042188809fe89cc64")
+
+
+def decode_attn_traffic_ratio():
+    """(ratio, None) while the kernel source is the one the counters were taken on, else (None, reason)."""
+    import hashlib
+    path, want = DECODE_ATTN_TRAFFIC_SOURCE
+    try:
+        with open(os.path.join(ROOT, path), "rb") as f:
+            have = hashlib.sha256(f.read()).hexdigest()
+    except OSError as e:
+        return None, f"kernel source not readable: {e}"
+    if have != want:
+        return None, f"{path} changed since the ncu counters were taken"
+    return DECODE_ATTN_TRAFFIC_RATIO, None
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -204,9 +221,9 @@ def run_decode(wl, dev, steps, warmup, barrier, rank):
         step()
     torch.cuda.synchronize()
     barrier()
-    # timed region: only the dominant kernel's launches are bracketed with events (bracketing all 161
-    # launches of a step costs about 0.7 ms per step)
-    model.profile(True, only=("attention",))
+    # timed region: `value` comes from K steps with no event brackets inside; the dominant kernel's launch
+    # time from K more steps, under the same clock sampler, with only that kernel's launches bracketed
+    # (a bracket costs about 2 us, so bracketing every launch of a step would cost about 0.7 ms per step)
     l0 = pt.lib().pt_launch_count()
     with ClockSampler(dev) as clk:
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -215,8 +232,12 @@ def run_decode(wl, dev, steps, warmup, barrier, rank):
             step()
         ev1.record()
         torch.cuda.synchronize()
+        launches = pt.lib().pt_launch_count() - l0
+        model.profile(True, only=("attention",))
+        for _ in range(steps):
+            step()
+        torch.cuda.synchronize()
     ms = ev0.elapsed_time(ev1) / steps
-    launches = pt.lib().pt_launch_count() - l0
     prof = model.profile_read()
     # per-kernel breakdown from a second pass with every launch bracketed (not part of `value`)
     n_break = max(2, steps // 4)
@@ -230,10 +251,12 @@ def run_decode(wl, dev, steps, warmup, barrier, rank):
     attn_ms, attn_n = prof["attention"]
     attn_avg_ms = attn_ms / max(attn_n, 1) if attn_n else float("nan")
     achieved = alg["attn_bytes_per_layer"] / (attn_avg_ms * 1e-3) / 1e9
+    ratio, why_not = decode_attn_traffic_ratio()
+    if ratio is not None and not (wl.head_dim == 128 and wl.page_size == 16 and wl.dtype == "bf16"):
+        ratio, why_not = None, "counters were taken on head_dim 128, 16-token pages, bf16 cache"
     roof = {"bound": "hbm", "kernel": "k_decode_attn", "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s",
             "frac": achieved / pk["hbm_gbs"],
-            "traffic": (alg["attn_bytes_per_layer"] * DECODE_ATTN_TRAFFIC_RATIO
-                        if DECODE_ATTN_TRAFFIC_RATIO and wl.head_dim == 128 and wl.page_size == 16 else None),
+            "traffic": alg["attn_bytes_per_layer"] * ratio if ratio else None, "traffic_note": why_not,
             "peak_kind": f"of {pk_kind}", "avg_launch_ms": attn_avg_ms, "launches": attn_n,
             "step_hbm_gbs": alg["bytes"] / (ms * 1e-3) / 1e9, "step_frac": alg["bytes"] / (ms * 1e-3) / 1e9 / pk["hbm_gbs"],
             "step_frac_of_nominal_8tbs": alg["bytes"] / (ms * 1e-3) / 8e12}
@@ -295,7 +318,8 @@ def run_prefill(wl, dev, steps, warmup, barrier, rank):
         step()
     torch.cuda.synchronize()
     barrier()
-    model.profile(True)
+    # `value` from K steps with no event brackets inside; the per-kernel times from K more steps, under the
+    # same clock sampler, with every launch bracketed
     l0 = pt.lib().pt_launch_count()
     with ClockSampler(dev) as clk:
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -304,8 +328,12 @@ def run_prefill(wl, dev, steps, warmup, barrier, rank):
             step()
         ev1.record()
         torch.cuda.synchronize()
+        launches = pt.lib().pt_launch_count() - l0
+        model.profile(True)
+        for _ in range(steps):
+            step()
+        torch.cuda.synchronize()
     ms = ev0.elapsed_time(ev1) / steps
-    launches = pt.lib().pt_launch_count() - l0
     prof = model.profile_read()
     model.profile(False)
     assert model.device_status() == (0, 0)
@@ -449,7 +477,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2")
-    ap.add_argument("--extra", default="cfg3", help="comma-separated workloads reported under 'extra' (N=1 only); '' for none")
+    ap.add_argument("--extra", default="cfg3,cfg4,cfg1,cfg0", help="comma-separated workloads reported under 'extra' (N=1 only); '' for none")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--parallel", default="replicas", choices=["replicas", "tracks"],
                     help="N > 1: 'replicas' = every rank runs the whole model on its own batch (weak scaling, no collective); "
@@ -481,7 +509,7 @@ def main():
             vals.append(v)
         ms = (time.perf_counter() - t0) / a.steps * 1e3
         v = float(np.mean(vals))
-        print(json.dumps({"impl": "reference", "metric": f"PT {metric} (CPU oracle, bounded sample)", "value": v, "unit": "tokens/s",
+        print(json.dumps({"impl": "reference", "metric": f"PT {metric}", "value": v, "unit": "tokens/s",
                           "n_gpus": a.gpus, "steps": a.steps, "warmup": a.warmup, "ms_per_step": ms, "higher_is_better": True,
                           "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
                           "config": {"workload": f"{wl.name} ({wl.mode})"},
@@ -521,7 +549,7 @@ def main():
         for name in [n for n in a.extra.split(",") if n and n != a.workload]:
             w2 = I.WORKLOADS[name]
             try:
-                r2 = (run_decode if w2.mode == "decode" else run_prefill)(w2, dev, max(3, a.steps // 4), 3, barrier, rank)
+                r2 = (run_decode if w2.mode == "decode" else run_prefill)(w2, dev, max(10, a.steps // 2), 3, barrier, rank)
                 extra[name] = {"metric": "decode tokens/s" if w2.mode == "decode" else "prefill tokens/s",
                                "value": r2["tokens"] / (r2["ms"] * 1e-3), "ms_per_step": r2["ms"], "roofline": r2["roofline"],
                                "kernels_ms_per_step": r2["kernels_ms_per_step"], "config": r2["config"], "clocks": r2["clocks"],
@@ -533,7 +561,7 @@ def main():
         v, sample, dt, cores = oracle_sample(wl)
         cpu = {"value": v, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample, "seconds": round(dt, 2)}
     if rank == 0:
-        line = {"metric": f"PT {metric} on B200", "value": total_tokens / (ms * 1e-3), "unit": "tokens/s", "n_gpus": world,
+        line = {"metric": f"PT {metric}", "value": total_tokens / (ms * 1e-3), "unit": "tokens/s", "n_gpus": world,
                 "steps": a.steps, "warmup": a.warmup, "ms_per_step": ms, "higher_is_better": True,
                 "scaling": "strong" if tracks_mode else "weak",
                 "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",

@@ -65,13 +65,12 @@ pt_status pt_kernel_prefill_attn(const void* q, const void* pool_l, int64_t pool
 /* The same decode attention for callers that cannot allocate device memory.  (The paper has no
  * counterpart: this is a packaging variant of pt_kernel_decode_attn.)
  *
- * Who needs it: code that runs where cudaMalloc is off limits - inside a region that is being
- * captured into a CUDA graph, in a real-time or serving loop that must not touch the allocator
- * after start-up, or in a host program that handed all device memory to another component and
- * has no pool of its own to carve a scratch buffer from.  Such a caller passes only inputs and
- * outputs; the split plan and the per-range partial results live in a fixed array inside the
- * library image (PT_STATIC_SCRATCH_BYTES, 8 MiB, resident on every GPU that loads the library
- * until the process exits).
+ * Who needs it: code that runs where cudaMalloc is off limits - a real-time or serving loop that
+ * must not touch the allocator after start-up, or a host program that handed all device memory to
+ * another component and has no pool of its own to carve a scratch buffer from.  Such a caller
+ * passes only inputs and outputs; the split plan and the per-range partial results live in a fixed
+ * array inside the library image (PT_STATIC_SCRATCH_BYTES, 8 MiB, resident on every GPU that loads
+ * the library until the process exits).
  *
  *  - Arguments are those of pt_kernel_decode_attn without scratch / scratch_bytes; results are
  *    identical to it.
@@ -79,6 +78,8 @@ pt_status pt_kernel_prefill_attn(const void* q, const void* pool_l, int64_t pool
  *    PT_STATIC_SCRATCH_BYTES are refused with PT_ERR_BUFFER_TOO_SMALL and nothing is launched.
  *  - The first call on each device looks up the array's device address (no allocation, but a
  *    driver query): make that first call before any stream capture begins.
+ *  - Like pt_kernel_decode_attn, every call builds the split plan on the host from kv_len and
+ *    uploads it with an asynchronous copy on `stream`.
  *  - The entry point calls no cudaMalloc, cudaFree or any allocating library routine.
  *  - All calls on a device share the one array, which keeps whatever the previous call left.
  *    Nothing in it has to start at zero - every word a call reads it has written first - but

@@ -20,9 +20,8 @@ OBJ = os.path.join(ROOT, "_build")
 LIB = os.path.join(HERE, "libpt.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-         "--use_fast_math=false", "-Xcompiler", "-fPIC,-O2,-Wall,-Wno-unused-function",
+         "-Xcompiler", "-fPIC,-O2,-Wall,-Wno-unused-function",
          "-I", os.path.join(ROOT, "include"), "-I", CSRC]
-FLAGS = [f for f in FLAGS if f != "--use_fast_math=false"]
 
 
 def _newer(target: str, deps: list[str]) -> bool:

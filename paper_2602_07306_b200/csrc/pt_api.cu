@@ -147,7 +147,6 @@ pt_status pt_model_create(const pt_config* cfg, pt_model** out) {
 
 void pt_model_destroy(pt_model* m) {
     if (!m) return;
-    tc_forget_model(m);
     for (auto& e : m->prof_ev) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
     delete m;
 }

@@ -40,6 +40,18 @@ struct Seq {
     int32_t len = 0;
 };
 
+// Tensor maps of one layer's packed weights: [qkv, o, gu, d][bn 64, 128, 256][k-blocks per copy 1, 2, 4];
+// combinations the GEMM launcher never picks stay unset.
+struct WMaps { CUtensorMap m[4][3][3]; };
+
+// Per-device caches (function attributes, SM counts, symbol addresses) are indexed by the current device.
+constexpr int kMaxDevices = 64;
+inline int current_device() {
+    int d = 0;
+    if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= kMaxDevices) d = 0;
+    return d;
+}
+
 }  // namespace pt
 
 struct pt_model {
@@ -58,6 +70,7 @@ struct pt_model {
     int tap_layer = -2;
     float* tap_buf = nullptr;
     std::vector<char> meta_host;          // staging for the per-call metadata upload
+    std::vector<pt::WMaps> wmaps;         // [L] tensor maps of the bound weights (tensor-core path)
     // optional per-kernel timing (pt_profile_enable)
     struct ProfEv { cudaEvent_t a, b; int cat; };
     uint32_t prof_mask = 0;               // bit c set: launches of category c are bracketed with events
@@ -160,6 +173,5 @@ void launch_pack(const pt_model* m, int kind, const void* src, void* dst_matrix_
 // pt_tc.cu (bf16 tensor-core path)
 pt_status tc_build_weight_maps(pt_model* m);
 pt_status tc_forward(Call& k);
-void tc_forget_model(const pt_model* m);
 
 }  // namespace pt

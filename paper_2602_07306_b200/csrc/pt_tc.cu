@@ -80,13 +80,9 @@ __global__ void k_track_sync(const float* __restrict__ hT, size_t tstride, int T
     if (ssq && (lane & 15) == 0 && tile < tiles) ssq[(size_t)row * tiles + tile] = s;
 }
 
-// [qkv, o, gu, d][bn 64, 128, 256][k-blocks per copy 1, 2, 4]; combinations gemm_kps never picks stay unset
-struct WMaps { CUtensorMap m[4][3][3]; };
 inline int kps_index(int kps) { return kps == 4 ? 2 : (kps == 2 ? 1 : 0); }
 
 }  // namespace
-
-static std::unordered_map<const pt_model*, std::vector<WMaps>> g_wmaps;
 
 pt_status tc_build_weight_maps(pt_model* m) {
     const pt_config& c = m->cfg;
@@ -110,11 +106,9 @@ pt_status tc_build_weight_maps(pt_model* m) {
                     if (s != PT_OK) return s;
                 }
             }
-    g_wmaps[m] = std::move(v);
+    m->wmaps = std::move(v);
     return PT_OK;
 }
-
-void tc_forget_model(const pt_model* m) { g_wmaps.erase(m); }
 
 pt_status tc_forward(Call& k) {
     pt_model* m = k.m;
@@ -124,9 +118,8 @@ pt_status tc_forward(Call& k) {
     const size_t MH = (size_t)M * H;
     cudaStream_t st = k.st;
     Work& w = k.w;
-    auto it = g_wmaps.find(m);
-    if (it == g_wmaps.end()) { set_error("weights not bound"); return PT_ERR_STATE; }
-    const std::vector<WMaps>& wm = it->second;
+    if ((int)m->wmaps.size() != g.L) { set_error("weights not bound"); return PT_ERR_STATE; }
+    const std::vector<WMaps>& wm = m->wmaps;
     __nv_bfloat16* pool = (__nv_bfloat16*)c->pool;
     const int64_t pool_tstride = (int64_t)g.L * c->slab_elems;
     const int tiles = (H + kSsqTile - 1) / kSsqTile;
@@ -405,7 +398,6 @@ extern "C" pt_status pt_kernel_decode_attn(const void* q, const void* pool_l, in
 static __device__ __align__(256) unsigned char g_static_scratch[PT_STATIC_SCRATCH_BYTES];
 
 namespace pt {
-constexpr int kMaxDevices = 64;
 static void* g_static_scratch_addr[kMaxDevices] = {};
 }
 

@@ -606,7 +606,7 @@ pt_status launch_flash_prefill_p(const AttnP& p, int T, int dh, bool legacy, cud
     dim3 grid((p.S + 63) / 64, p.nq, T * p.B);
     const int smem = 2 * 2 * kTileKeys * dh * 2;
     pt_status s = PT_OK;
-#define GO(DH_) { static bool done = false; if (!done) { if ((s = set_smem(k_flash_prefill<DH_>, smem)) != PT_OK) return s; done = true; } \
+#define GO(DH_) { static bool done_[kMaxDevices] = {}; bool& done = done_[current_device()]; if (!done) { if ((s = set_smem(k_flash_prefill<DH_>, smem)) != PT_OK) return s; done = true; } \
                   k_flash_prefill<DH_><<<grid, kThreads, smem, st>>>(p); }
     if (dh == 32) GO(32) else if (dh == 64) GO(64) else GO(128)
 #undef GO
@@ -628,7 +628,7 @@ pt_status launch_decode_attn_p(const AttnP& p, int T, int dh, int n_items, int m
                                             p.pool_tstride * 2, 16);
         if (s != PT_OK) return s;
         const int smem = 1024 + 4 * kDecStages * 2 * 16 * dh * 2 + 4 * kDecStages * 8;
-#define GOT(DH_) { static bool done = false; if (!done) { if ((s = set_smem(k_decode_attn_tma<DH_>, smem)) != PT_OK) return s; done = true; } \
+#define GOT(DH_) { static bool done_[kMaxDevices] = {}; bool& done = done_[current_device()]; if (!done) { if ((s = set_smem(k_decode_attn_tma<DH_>, smem)) != PT_OK) return s; done = true; } \
                    launch_dependent(k_decode_attn_tma<DH_>, grid, dim3(kThreads), (size_t)smem, st, kvmap, p); \
                    if (max_splits > 1) { launch_dependent(k_decode_combine<DH_>, dim3((p.B * p.nq * 32 + 127) / 128, T), dim3(128), (size_t)0, st, p); \
                                          g_launches.fetch_add(1, std::memory_order_relaxed); } }
@@ -639,7 +639,7 @@ pt_status launch_decode_attn_p(const AttnP& p, int T, int dh, int n_items, int m
     }
     const int smem = std::max(3 * 2 * kTileKeys * dh * 2, 4 * 8 * (dh + 2) * 4);
     pt_status s = PT_OK;
-#define GO(DH_) { static bool done = false; if (!done) { if ((s = set_smem(k_decode_attn<DH_>, smem)) != PT_OK) return s; done = true; } \
+#define GO(DH_) { static bool done_[kMaxDevices] = {}; bool& done = done_[current_device()]; if (!done) { if ((s = set_smem(k_decode_attn<DH_>, smem)) != PT_OK) return s; done = true; } \
                   k_decode_attn<DH_><<<grid, kThreads, smem, st>>>(p); \
                   if (max_splits > 1) { k_decode_combine<DH_><<<dim3((p.B * p.nq * 32 + 127) / 128, T), 128, 0, st>>>(p); g_launches.fetch_add(1, std::memory_order_relaxed); } }
     if (dh == 32) GO(32) else if (dh == 64) GO(64) else GO(128)

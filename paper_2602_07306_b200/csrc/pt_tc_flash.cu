@@ -470,7 +470,7 @@ pt_status launch_flash_prefill_tc(const AttnP& p, int T, int dh, cudaStream_t st
     if ((s = make_map_bf16_strided(&kvmap, p.pool_l, dh, (int64_t)p.num_pages * 2 * p.nkv * p.ps, T, p.pool_tstride * 2, 16)) != PT_OK) return s;
     const int q_box_rows = std::min(128, p.M);
     dim3 grid((p.S + 255) / 256, p.nq, T * p.B);
-#define GO(DH_) { static bool done = false; \
+#define GO(DH_) { static bool done_[kMaxDevices] = {}; bool& done = done_[current_device()]; \
         if (!done) { cudaError_t e = cudaFuncSetAttribute(k_flash_prefill_tc<DH_>, cudaFuncAttributeMaxDynamicSharedMemorySize, FlashCfg<DH_>::SMEM); \
                      if (e != cudaSuccess) { set_error("cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; } done = true; } \
         k_flash_prefill_tc<DH_><<<grid, kFlashThreads, FlashCfg<DH_>::SMEM, st>>>(qmap, kvmap, p, q_box_rows); }

@@ -1073,7 +1073,8 @@ EncodeFn get_encode() {
 template <int BN, int EPI>
 pt_status launch_t(const CUtensorMap& ta, const CUtensorMap& tb, GemmP p, cudaStream_t st, int sms) {
     using C = Cfg<BN>;
-    static bool attr_done = false;
+    static bool attr_done_[kMaxDevices] = {};
+    bool& attr_done = attr_done_[current_device()];
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(gemm_tc<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
         if (e != cudaSuccess) { set_error("cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
@@ -1095,8 +1096,9 @@ pt_status launch_t(const CUtensorMap& ta, const CUtensorMap& tb, GemmP p, cudaSt
 
 template <int EPI>
 pt_status launch_pair_t(const CUtensorMap& ta, const CUtensorMap& tb, GemmP p, cudaStream_t st, int sms) {
-    static int max_pairs = -1;
-    if (max_pairs < 0) {
+    static int max_pairs_[kMaxDevices] = {};           // 0 = not asked yet on that device
+    int& max_pairs = max_pairs_[current_device()];
+    if (max_pairs <= 0) {
         cudaError_t e = cudaFuncSetAttribute(gemm_tc_pair<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
         if (e != cudaSuccess) { set_error("cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
         cudaLaunchConfig_t q = {};
@@ -1144,8 +1146,9 @@ pt_status make_box_map(CUtensorMap* out, bool bf16, const void* base, int64_t co
 
 // The plain residual epilogue on CTA pairs with its global traffic on the TMA unit; the caller has checked resid_by_tma().
 pt_status launch_pair_resid(const CUtensorMap& ta, const CUtensorMap& tb, GemmP p, cudaStream_t st, int sms) {
-    static int max_pairs = -1;
-    if (max_pairs < 0) {
+    static int max_pairs_[kMaxDevices] = {};           // 0 = not asked yet on that device
+    int& max_pairs = max_pairs_[current_device()];
+    if (max_pairs <= 0) {
         cudaError_t e = cudaFuncSetAttribute(gemm_tc_pair_resid, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
         if (e != cudaSuccess) { set_error("cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
         cudaLaunchConfig_t q = {};
@@ -1212,11 +1215,12 @@ pt_status make_map_bf16_strided(CUtensorMap* out, const void* base, int64_t k, i
 
 // Clusters of two CTAs with this kernel's shared memory must be launchable on the current device; asked once.
 static bool pair_launchable() {
-    static int state = -1;
-    if (state < 0) {
-        state = 0;
-        int dev = 0, sms = 0;
-        cudaGetDevice(&dev);
+    static int state_[kMaxDevices] = {};               // 0 = not asked yet on that device, 1 = yes, 2 = no
+    const int dev = current_device();
+    int& state = state_[dev];
+    if (state == 0) {
+        state = 2;
+        int sms = 0;
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (cudaFuncSetAttribute(gemm_tc_pair<EPI_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem) == cudaSuccess && sms >= 2) {
             cudaLaunchConfig_t q = {};
@@ -1316,10 +1320,10 @@ int gemm_bn(int N, int M, int T, int epi) {
 }
 
 pt_status launch_gemm(int epi, int bn, const CUtensorMap& ta, const CUtensorMap& tb, GemmP p, cudaStream_t st) {
-    static int sms = 0;
+    static int sms_[kMaxDevices] = {};
+    const int dev = current_device();
+    int& sms = sms_[dev];
     if (!sms) {
-        int dev = 0;
-        cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (sms <= 0) sms = 148;
     }

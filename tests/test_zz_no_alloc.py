@@ -1,8 +1,8 @@
 """The allocation-free decode-attention entry point (collected last on purpose).
 
-pt_kernel_decode_attn_static serves callers that cannot obtain device memory at call time - code
-inside a CUDA-graph capture, a serving loop that must stay away from the allocator once it is
-running, a host that owns no device pool to carve scratch from.  It keeps its split plan and
+pt_kernel_decode_attn_static serves callers that cannot obtain device memory at call time - a
+serving loop that must stay away from the allocator once it is running, a host that owns no device
+pool to carve scratch from.  It keeps its split plan and
 partial results in an 8 MiB array built into the library, so all calls on a device share that
 array and it still holds the previous call's data when the next one starts.  The test therefore
 makes two different calls in a row and checks each against the ordinary entry point (which takes
