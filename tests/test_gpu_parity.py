@@ -163,3 +163,12 @@ def test_bf16_table1_head_layout_eight_query_heads_one_kv_head(D):
     prefill in chunks, then decode steps over split key ranges."""
     wl = small("bf16", T=2, L=4, D=D, H=512, nq=8, nkv=1, F=256)
     run_case(wl, B=2, S=300, chunks=[290, 10], decode_steps=2, shuffle=True, gain_jitter=0.1)
+
+
+@pytest.mark.parametrize("B", [256, 257])
+def test_bf16_decode_track_sync_on_both_sides_of_256_rows(B):
+    """A decode step of up to 256 rows reduces the tracks with per-track down GEMMs plus the reduction kernel,
+    a larger one inside the K-concatenated down GEMM: both schedules against the oracle, with a sync after
+    every layer."""
+    wl = small("bf16", T=3, L=2, D=1, H=128, nq=2, nkv=1, F=176)
+    run_case(wl, B=B, S=2, decode_steps=2, check_pool=False)
