@@ -21,12 +21,44 @@ namespace pt {
 namespace {
 
 constexpr int kFlashThreads = 384;
-constexpr int kStages = 2;                 // K ring and V ring depth
+#ifndef FLASH_KSTAGES
+#define FLASH_KSTAGES 3
+#endif
+constexpr int kStagesK = FLASH_KSTAGES;    // K ring depth (head_dim 128: 2 Q tiles + 3 K + 2 V tiles of 32 KB fill the 227 KB of a CTA)
+constexpr int kStagesV = 2;                // V ring depth
+// Alternatives that were built and measured on the 8 x 4096-token causal shape of 8 tracks (one launch alone,
+// 924 TFLOP/s with all of them off and a two-stage K ring), kept as compile-time switches:
+//   FLASH_SPLIT_P   P handed to the MMA warp in two parts of 64 keys, so that the first half of P V runs under
+//                   the second half of the exponentials: 854 (the extra tcgen05.wait::st and arrive cost more)
+//   FLASH_PREFETCH  cp.async.bulk.prefetch.tensor of the K/V pages one ring depth ahead: 780 (the prefetches
+//                   take turns with the copies on the SM's one TMA unit)
+//   FLASH_POLY      exp2 of 4 / 8 of every 16 scores as a cubic on the FMA pipe instead of the MUFU: 905 / 829
+//                   (one softmax warp per scheduler and tile is bound by its own issue rate, not by the MUFU)
+//   FLASH_KSTAGES   three K stages instead of two: 938, kept
+//   FLASH_SWAIT_NS  softmax warps sleeping between polls of their score barrier: no change
+// Two softmax threads per query row (sixteen softmax warps, each thread 64 score columns, half-row maxima
+// exchanged through shared memory at a two-warp named barrier) was also built: 814 with the scores kept in
+// registers, 697 with a second read of the scores from tensor memory; its per-step overheads (barrier,
+// exchange, twice the polls, 104 registers) outweigh the shorter chain.
+#ifndef FLASH_SPLIT_P
+#define FLASH_SPLIT_P 0
+#endif
+#ifndef FLASH_PREFETCH
+#define FLASH_PREFETCH 0
+#endif
+#ifndef FLASH_POLY
+#define FLASH_POLY 0                       // of every 16 scores, this many (a multiple of 4) take the polynomial exp2
+#endif
+#ifndef FLASH_SWAIT_NS
+#define FLASH_SWAIT_NS 0                   // > 0: the softmax warps sleep this long between polls of their score barrier
+#endif
+constexpr int kPParts = FLASH_SPLIT_P ? 2 : 1;
 constexpr uint32_t kSpin = 1u << 26;
 constexpr int kHalfBytes = 128 * 128;      // 128 rows x 64 bf16: one swizzled column block of a tile
 
-enum { B_QFULL = 0, B_KFULL = 2, B_KEMPTY = 4, B_VFULL = 6, B_VEMPTY = 8, B_SFULL = 10, B_PFULL = 12,
-       B_OREADY = 14, B_VRAW = 16, B_COUNT = 17 };
+enum { B_QFULL = 0, B_KFULL = 2, B_KEMPTY = 5, B_VFULL = 8, B_VEMPTY = 10, B_SFULL = 12, B_PFULL = 14 /* [tile][part] */,
+       B_OREADY = 18, B_VRAW = 20, B_COUNT = 21 };
+static_assert(kStagesK <= 3 && kStagesV <= 2, "barrier slots");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
@@ -46,14 +78,18 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
 }
 // `relaxed` waits (the copy warp's, which run stages ahead of their consumers) back off between polls:
 // a spinning warp costs issue slots and power; the softmax and MMA hand-offs poll at full rate.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, bool relaxed = false) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, bool relaxed = false, unsigned sleep_ns = 128) {
     WaitClock clock;
     for (uint32_t i = 0; i < kSpin; ++i) {
         if (mbar_try(bar, parity)) return true;
-        if (relaxed && i >= 2) __nanosleep(128);
+        if (relaxed && i >= 2) __nanosleep(sleep_ns);
         if ((i & 255) == 255 && (*abort_flag || clock.expired())) return false;
     }
     return false;
+}
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* map, int c0, int c1, int c2) {
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
+                 ::"l"((uint64_t)map), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2) {
     asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
@@ -129,6 +165,31 @@ __device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1) {
     asm("{\n .reg .b64 ra, rd;\n mov.b64 ra, {%2, %3};\n mov.b64 rd, {%0, %1};\n add.rn.f32x2 rd, rd, ra;\n mov.b64 {%0, %1}, rd;\n}"
         : "+f"(d0), "+f"(d1) : "f"(a0), "f"(a1));
 }
+// 2^x for a pair of arguments on the FMA pipe instead of the MUFU: x = n + f with n = round(x) (adding 1.5 * 2^23
+// leaves n in the low mantissa bits), 2^f by a cubic on [-0.5, 0.5] (relative error 7.5e-5, a twenty-fifth of the
+// bf16 rounding the result receives), 2^n by adding n to the exponent field.  Arguments below -125 give 2^-125
+// (1e-38: a masked score's probability is not exactly zero on this path, but it is far below anything fp32 sums keep).
+__device__ __forceinline__ void ex2_poly2(float& x0, float& x1) {
+    const float magic = 12582912.0f;
+    x0 = fmaxf(x0, -125.0f); x1 = fmaxf(x1, -125.0f);
+    float r0, r1, p0, p1;
+    asm("{\n .reg .b64 x, m, r, n, f, p, c;\n"
+        " mov.b64 x, {%4, %5};\n mov.b64 m, {%6, %6};\n"
+        " add.rn.f32x2 r, x, m;\n"                      // r = x + magic: the integer part lands in the mantissa
+        " sub.rn.f32x2 n, r, m;\n"                      // n = round(x)
+        " sub.rn.f32x2 f, x, n;\n"                      // f in [-0.5, 0.5]
+        " mov.b64 p, {%7, %7};\n mov.b64 c, {%8, %8};\n"
+        " fma.rn.f32x2 p, p, f, c;\n"
+        " mov.b64 c, {%9, %9};\n"
+        " fma.rn.f32x2 p, p, f, c;\n"
+        " mov.b64 c, {%10, %10};\n"
+        " fma.rn.f32x2 p, p, f, c;\n"
+        " mov.b64 {%0, %1}, r;\n mov.b64 {%2, %3}, p;\n}"
+        : "=f"(r0), "=f"(r1), "=f"(p0), "=f"(p1)
+        : "f"(x0), "f"(x1), "f"(magic), "f"(0.05517137795686722f), "f"(0.24261121451854706f), "f"(0.6932610273361206f), "f"(0.9999280571937561f));
+    x0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(r0) << 23));
+    x1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(r1) << 23));
+}
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float d;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -168,7 +229,8 @@ __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t saddr) {
 template <int DH> struct FlashCfg {
     static constexpr int HALVES = DH / 64;
     static constexpr int TILE_BYTES = HALVES * kHalfBytes;          // one Q, K or V tile of 128 rows
-    static constexpr int SMEM = (2 + 2 * kStages) * TILE_BYTES + 1024 + 256;
+    static constexpr int SMEM = (2 + kStagesK + kStagesV) * TILE_BYTES + 1024 + 256;
+    static_assert(SMEM <= 232448, "shared memory of one CTA");
 };
 
 template <int DH>
@@ -181,8 +243,8 @@ k_flash_prefill_tc(const __grid_constant__ CUtensorMap qmap, const __grid_consta
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* sq = smem;
     uint8_t* sk = sq + 2 * TILE;
-    uint8_t* sv = sk + kStages * TILE;
-    uint64_t* bars = (uint64_t*)(sv + kStages * TILE);
+    uint8_t* sv = sk + kStagesK * TILE;
+    uint64_t* bars = (uint64_t*)(sv + kStagesV * TILE);
     uint32_t* tmem_slot = (uint32_t*)(bars + B_COUNT);
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
@@ -203,7 +265,7 @@ k_flash_prefill_tc(const __grid_constant__ CUtensorMap qmap, const __grid_consta
     const int n_max = max(n_t[0], n_t[1]);
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < B_COUNT; ++i) mbar_init(&bars[i], (i == B_PFULL || i == B_PFULL + 1) ? 4 : 1);
+        for (int i = 0; i < B_COUNT; ++i) mbar_init(&bars[i], (i >= B_PFULL && i < B_PFULL + 4) ? 4 : 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -238,8 +300,8 @@ k_flash_prefill_tc(const __grid_constant__ CUtensorMap qmap, const __grid_consta
         __syncwarp();
         bool bad_page = false;
         for (int j = 0; j < n_max; ++j) {
-            const int s = j % kStages;
-            const uint32_t ph = (uint32_t)(j / kStages) & 1u;
+            const int sK = j % kStagesK, s = j % kStagesV;
+            const uint32_t phK = (uint32_t)(j / kStagesK) & 1u, ph = (uint32_t)(j / kStagesV) & 1u;
             const int key0 = j * 128;
             const int ng = min(8, (key_end - key0 + 15) >> 4);    // 16-key groups of this tile that hold keys
             int row_k = 0;
@@ -250,13 +312,13 @@ k_flash_prefill_tc(const __grid_constant__ CUtensorMap qmap, const __grid_consta
                 row_k = (page * 2 * p.nkv + kvh) * p.ps + key % p.ps;
             }
             const uint32_t bytes = (uint32_t)ng * 16u * DH * 2u;
-            if (!mbar_wait(&bars[B_KEMPTY + s], ph ^ 1u, abort_flag, true)) { if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_FLASH_KEMPTY); *abort_flag = 1; } break; }
-            if (lane == 0) mbar_expect_tx(&bars[B_KFULL + s], bytes);
+            if (!mbar_wait(&bars[B_KEMPTY + sK], phK ^ 1u, abort_flag, true)) { if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_FLASH_KEMPTY); *abort_flag = 1; } break; }
+            if (lane == 0) mbar_expect_tx(&bars[B_KFULL + sK], bytes);
             __syncwarp();
             if (lane < ng) {
 #pragma unroll
                 for (int h = 0; h < HALVES; ++h)
-                    tma_load_3d(smem_u32(sk + s * TILE + h * kHalfBytes + lane * 2048), &kvmap, &bars[B_KFULL + s], h * 64, row_k, t);
+                    tma_load_3d(smem_u32(sk + sK * TILE + h * kHalfBytes + lane * 2048), &kvmap, &bars[B_KFULL + sK], h * 64, row_k, t);
             }
             if (!mbar_wait(&bars[B_VEMPTY + s], ph ^ 1u, abort_flag, true)) { if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_FLASH_VEMPTY); *abort_flag = 1; } break; }
             const bool partial = key0 + 128 > key_end;             // rows past the last key must read as zero
@@ -267,6 +329,20 @@ k_flash_prefill_tc(const __grid_constant__ CUtensorMap qmap, const __grid_consta
 #pragma unroll
                 for (int h = 0; h < HALVES; ++h)
                     tma_load_3d(smem_u32(sv + s * TILE + h * kHalfBytes + lane * 2048), &kvmap, vbar, h * 64, row_k + p.nkv * p.ps, t);
+            }
+            if (FLASH_PREFETCH && j + kStagesK < n_max) {          // the tile one ring depth ahead: bring its pages into L2 now
+                const int keyp = (j + kStagesK) * 128 + lane * 16;
+                if (lane < 8 && keyp < key_end) {
+                    const int page = p.bt[(size_t)b * p.maxp + keyp / p.ps];
+                    if (page >= 0 && page < p.num_pages) {
+                        const int row_p = (page * 2 * p.nkv + kvh) * p.ps + keyp % p.ps;
+#pragma unroll
+                        for (int h = 0; h < HALVES; ++h) {
+                            tma_prefetch_3d(&kvmap, h * 64, row_p, t);
+                            tma_prefetch_3d(&kvmap, h * 64, row_p + p.nkv * p.ps, t);
+                        }
+                    }
+                }
             }
             if (partial) {                                         // at most once per CTA: its last tile
                 if (!mbar_wait(&bars[B_VRAW], 0u, abort_flag)) { if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_FLASH_VRAW); *abort_flag = 1; } break; }
@@ -302,12 +378,20 @@ k_flash_prefill_tc(const __grid_constant__ CUtensorMap qmap, const __grid_consta
                 }
                 tc_commit(&bars[B_SFULL + i]);
             };
-            auto pv = [&](int i, int s, bool acc) {                // O_i (+)= P_i V_s
-                if (!ok) return;
+            auto pv = [&](int i, int s, int j) {                   // O_i (+)= P_i V_s, in the parts P arrives in
                 const uint32_t va = smem_u32(sv + s * TILE);
+                wait(B_PFULL + 2 * i, (uint32_t)j & 1u, LOC_FLASH_PFULL);
+                wait(B_VFULL + s, (uint32_t)(j / kStagesV) & 1u, LOC_FLASH_VFULL);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    mma_ts(tmem_base + 256 + i * DH, tmem_base + i * 128 + ks * 8, desc_mnmajor(va + ks * 2048), idesc_pv, acc || ks != 0);
+                for (int part = 0; part < kPParts; ++part) {
+                    if (part) wait(B_PFULL + 2 * i + 1, (uint32_t)j & 1u, LOC_FLASH_PFULL);
+                    if (!ok) return;
+#pragma unroll
+                    for (int u = 0; u < 8 / kPParts; ++u) {
+                        const int ks = part * (8 / kPParts) + u;
+                        mma_ts(tmem_base + 256 + i * DH, tmem_base + i * 128 + ks * 8, desc_mnmajor(va + ks * 2048), idesc_pv, j > 0 || ks != 0);
+                    }
+                }
                 tc_commit(&bars[B_OREADY + i]);
             };
             wait(B_KFULL + 0, 0, LOC_FLASH_KFULL);
@@ -316,14 +400,12 @@ k_flash_prefill_tc(const __grid_constant__ CUtensorMap qmap, const __grid_consta
                 if (n_t[i] > 0) { wait(B_QFULL + i, 0, LOC_FLASH_QFULL); qk(i, 0); }
             if (ok) tc_commit(&bars[B_KEMPTY + 0]);
             for (int j = 0; j < n_max && ok; ++j) {
-                const int s = j % kStages, sn = (j + 1) % kStages;
-                const uint32_t ph = (uint32_t)(j / kStages) & 1u, phn = (uint32_t)((j + 1) / kStages) & 1u;
+                const int s = j % kStagesV, sn = (j + 1) % kStagesK;
+                const uint32_t phn = (uint32_t)((j + 1) / kStagesK) & 1u;
 #pragma unroll
                 for (int i = 0; i < 2; ++i) {
                     if (j < n_t[i]) {
-                        wait(B_PFULL + i, (uint32_t)j & 1u, LOC_FLASH_PFULL);
-                        wait(B_VFULL + s, ph, LOC_FLASH_VFULL);
-                        pv(i, s, j > 0);
+                        pv(i, s, j);
                         if (j + 1 < n_t[i]) { wait(B_KFULL + sn, phn, LOC_FLASH_KFULL); qk(i, sn); }
                     }
                 }
@@ -351,7 +433,7 @@ k_flash_prefill_tc(const __grid_constant__ CUtensorMap qmap, const __grid_consta
         float m_ref = -INFINITY, l_run = 0.f;
         bool ok = true;
         for (int j = 0; j < n_i; ++j) {
-            ok = mbar_wait(&bars[B_SFULL + i], (uint32_t)j & 1u, abort_flag);
+            ok = mbar_wait(&bars[B_SFULL + i], (uint32_t)j & 1u, abort_flag, FLASH_SWAIT_NS > 0, FLASH_SWAIT_NS);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) { if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_FLASH_SFULL); *abort_flag = 1; } break; }
             tc_fence_after();
@@ -409,19 +491,26 @@ k_flash_prefill_tc(const __grid_constant__ CUtensorMap qmap, const __grid_consta
                     float x0, x1, x2, x3;
                     fma2(x0, x1, v[cc * 32 + e], v[cc * 32 + e + 1], c, nmc);
                     fma2(x2, x3, v[cc * 32 + e + 2], v[cc * 32 + e + 3], c, nmc);
-                    x0 = ex2(x0); x1 = ex2(x1); x2 = ex2(x2); x3 = ex2(x3);
+                    if ((e & 15) < FLASH_POLY) { ex2_poly2(x0, x1); ex2_poly2(x2, x3); }
+                    else { x0 = ex2(x0); x1 = ex2(x1); x2 = ex2(x2); x3 = ex2(x3); }
                     add2(l0, l1, x0, x1);
                     add2(l2, l3, x2, x3);
                     pk[e >> 1] = pack_bf16(x0, x1);
                     pk[(e >> 1) + 1] = pack_bf16(x2, x3);
                 }
                 tm_st16(t_s + cc * 16, pk);
+                if (FLASH_SPLIT_P && cc == 1) {                    // keys 0-63 are in place: the first half of P V may start
+                    tm_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars[B_PFULL + 2 * i]);
+                }
             }
             l_run += (l0 + l1) + (l2 + l3);
             tm_wait_st();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&bars[B_PFULL + i]);
+            if (lane == 0) mbar_arrive(&bars[B_PFULL + 2 * i + kPParts - 1]);
         }
         if (ok && n_i > 0) {
             ok = mbar_wait(&bars[B_OREADY + i], (uint32_t)(n_i - 1) & 1u, abort_flag);
