@@ -15,7 +15,8 @@ invariants of Algorithm 1, brute-force page enumeration); no function here is
 consistent choice is valid): rotary pairs are (j, j + dh/2); query head i reads
 KV head i // G; the all-reduce of Algorithm 1 is a SUM (MEAN is available as an
 option); "Set h_i = h" of Algorithm 1 is read as inside the if-block (its own
-comment says it follows the all-reduce).
+comment says it follows the all-reduce); the optional FP8 storage format of the KV
+cache (E4M3 codes with one power-of-two scale per cached vector).
 
 Shapes: T tracks, L layers, D track-block depth, H per-track hidden, nq / nkv
 query / KV heads per track, dh = H / nq, G = nq / nkv, F feed-forward width.
@@ -128,6 +129,45 @@ def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, qpos: np.ndarray) -> 
     return out
 
 
+# ----------------------------------------------------------------------------- FP8 KV-cache format
+# Not in the paper (it has no cache at all): a declared storage format for K and V that halves the
+# bytes of the cache, so that the ragged decode workload fits one device whole.  Every cached vector
+# (one token, one KV head, head_dim values, K or V) is stored as E4M3 codes times one scale:
+#   scale = the smallest power of two s with max|v| / s <= 448   (1 for an all-zero vector)
+#   code  = v / s rounded to the nearest E4M3 value, ties to the even mantissa, saturating at +-448
+# E4M3 (the "FN" variant of the OCP 8-bit floating point formats): 1 sign, 4 exponent (bias 7) and 3
+# mantissa bits; normal values (1 + m/8) * 2^(e-7) for e = 1..15 (the code e = 15, m = 7 is NaN, so the
+# largest value is 1.75 * 2^8 = 448), subnormals (m/8) * 2^-6, no infinities.  Attention reads code * s.
+
+E4M3_MAX = 448.0
+
+
+def e4m3_round(x: np.ndarray) -> np.ndarray:
+    """x (float64) -> the nearest E4M3 value, ties to even, saturating at +-448."""
+    x = np.asarray(x, np.float64)
+    a = np.minimum(np.abs(x), E4M3_MAX)
+    with np.errstate(divide="ignore"):
+        e = np.floor(np.log2(np.where(a > 0, a, 1.0)))
+    e = np.maximum(e, -6.0)                        # below 2^-6 the spacing stays that of the subnormals
+    step = np.exp2(e - 3.0)                        # 8 steps per binade
+    q = np.rint(a / step) * step                   # numpy rounds halves to even; a carry into the next binade is exact
+    return np.copysign(np.minimum(q, E4M3_MAX), x)
+
+
+def kv_scale(v: np.ndarray) -> np.ndarray:
+    """Power-of-two scale of each vector along the last axis (shape [..., 1])."""
+    amax = np.max(np.abs(np.asarray(v, np.float64)), axis=-1, keepdims=True)
+    with np.errstate(divide="ignore"):
+        e = np.ceil(np.log2(np.where(amax > 0, amax, 1.0) / E4M3_MAX))
+    return np.where(amax > 0, np.exp2(e), 1.0)
+
+
+def kv_quantize(v: np.ndarray):
+    """(codes, scale): codes are E4M3 values (as float64), scale [..., 1]; the cached value is codes * scale."""
+    s = kv_scale(v)
+    return e4m3_round(np.asarray(v, np.float64) / s), s
+
+
 # ----------------------------------------------------------------------------- paged KV cache
 
 def kv_slot_offset(cfg: PTConfig, num_pages: int, page_size: int,
@@ -148,9 +188,14 @@ class PagedKVCache:
     i*page_size .. (i+1)*page_size-1 of sequence ``seq``.
     """
 
-    def __init__(self, cfg: PTConfig, num_pages: int, page_size: int = 16, free_order=None):
-        self.cfg, self.num_pages, self.page_size = cfg, num_pages, page_size
+    def __init__(self, cfg: PTConfig, num_pages: int, page_size: int = 16, free_order=None, kv_format: str = "model"):
+        if kv_format not in ("model", "e4m3"):
+            raise ValueError("kv_format")
+        self.cfg, self.num_pages, self.page_size, self.kv_format = cfg, num_pages, page_size, kv_format
+        # what attention reads: the values themselves, or (kv_format "e4m3") code * scale of the FP8 format above
         self.pool = np.zeros((cfg.T, cfg.L, num_pages, 2, cfg.kv_heads, page_size, cfg.head_dim))
+        # one scale per cached vector, indexed like the pool without its last axis (all ones for "model")
+        self.scale = np.ones((cfg.T, cfg.L, num_pages, 2, cfg.kv_heads, page_size))
         order = list(range(num_pages)) if free_order is None else [int(p) for p in free_order]
         if sorted(order) != list(range(num_pages)):
             raise ValueError("free_order must be a permutation of the page ids")
@@ -184,6 +229,11 @@ class PagedKVCache:
     def write(self, t: int, l: int, seq: int, pos: np.ndarray, k: np.ndarray, v: np.ndarray) -> None:
         """Store k, v [n, nkv, dh] at positions pos[n] of ``seq``."""
         pages, slots = self._pages_slots(seq, pos)
+        if self.kv_format == "e4m3":
+            (kc, ks), (vc, vs) = kv_quantize(k), kv_quantize(v)
+            k, v = kc * ks, vc * vs
+            self.scale[t, l, pages, 0, :, slots] = ks[..., 0]
+            self.scale[t, l, pages, 1, :, slots] = vs[..., 0]
         self.pool[t, l, pages, 0, :, slots, :] = k
         self.pool[t, l, pages, 1, :, slots, :] = v
 

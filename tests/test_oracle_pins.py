@@ -423,3 +423,97 @@ def test_generation_equals_teacher_forced_prefill():
     assert np.allclose(logits, want, rtol=1e-9, atol=1e-9)
     assert np.array_equal(toks, O.greedy(want))
     assert cache.length[0] == cache.length[1] == 8
+
+
+# ---------------------------------------------------------------- FP8 KV-cache format
+
+def _e4m3_table():
+    """Every finite non-negative E4M3 value, decoded from the bit fields (independent of e4m3_round)."""
+    vals = []
+    for code in range(0x7F):                          # 0x7F is NaN
+        e, m = code >> 3, code & 7
+        vals.append((m / 8.0) * 2.0 ** -6 if e == 0 else (1 + m / 8.0) * 2.0 ** (e - 7))
+    return np.array(vals)
+
+
+def test_e4m3_rounding_against_the_enumerated_format_and_torch():
+    fmt = {k: float(v) for k, v in _rows("e4m3_format.txt")}
+    table = _e4m3_table()
+    assert len(table) == fmt["finite_codes_per_sign"] and table.max() == fmt["max_normal"] == O.E4M3_MAX
+    assert table[1] == fmt["min_subnormal"] and table[8] == fmt["min_normal"]
+    rng = np.random.default_rng(0)
+    x = np.concatenate([rng.standard_normal(20000) * s for s in (1e-3, 0.05, 1.0, 30.0, 300.0)])
+    mids = (table[:-1] + table[1:]) / 2                # exact ties between neighbouring values
+    x = np.concatenate([x, mids, -mids, table, -table, [0.0, 448.0, 449.0, 1e6, -1e6, 463.9, 464.1]])
+    got = O.e4m3_round(x)
+    # brute force: nearest table value, ties to the even code (= even mantissa bit), saturating
+    a = np.minimum(np.abs(x), 448.0)
+    d = np.abs(a[:, None] - table[None, :])
+    best = d.min(axis=1)
+    want = np.empty_like(a)
+    for i in range(len(a)):
+        cand = np.flatnonzero(d[i] == best[i])
+        want[i] = table[[c for c in cand if c % 2 == 0][0]] if len(cand) > 1 else table[cand[0]]
+    np.testing.assert_array_equal(got, np.copysign(want, x))
+    assert np.all(np.isin(np.abs(got), table))
+    # the library's conversion (round to nearest even; it does not saturate, so in-range values only)
+    xin = x[np.abs(x) <= 448.0].astype(np.float32)
+    lib = torch.from_numpy(xin).to(torch.float8_e4m3fn).to(torch.float32).numpy()
+    np.testing.assert_array_equal(O.e4m3_round(xin.astype(np.float64)).astype(np.float32), lib)
+
+
+def test_kv_scale_is_the_smallest_power_of_two_without_saturation():
+    rng = np.random.default_rng(1)
+    v = rng.standard_normal((200, 16)) * np.exp2(rng.integers(-20, 12, (200, 1)))
+    v[0] = 0.0
+    v[1] = 0.0; v[1, 3] = 448.0                        # exactly the largest code at scale 1
+    v[2] = 0.0; v[2, 5] = -448.0000001
+    s = O.kv_scale(v)
+    assert s.shape == (200, 1) and s[0, 0] == 1.0 and s[1, 0] == 1.0 and s[2, 0] == 2.0
+    for i in range(3, 200):
+        amax = np.abs(v[i]).max()
+        cands = [2.0 ** e for e in range(-60, 40) if amax / 2.0 ** e <= 448.0]
+        assert s[i, 0] == min(cands)
+        assert 224.0 < amax / s[i, 0] <= 448.0         # the largest element uses the top binade
+    codes, s2 = O.kv_quantize(v)
+    np.testing.assert_array_equal(s, s2)
+    assert np.all(np.isin(np.abs(codes), _e4m3_table()))
+    # round-trip bound: half a unit in the last place, relative 2^-4 for normal codes, absolute for subnormal ones
+    back = codes * s
+    err = np.abs(back - v)
+    normal = np.abs(v) >= s * 2.0 ** -6
+    assert np.all(err[normal] <= np.abs(v)[normal] * 2.0 ** -4 * (1 + 1e-12))
+    assert np.all(err[~normal] <= (s * 2.0 ** -10 * np.ones_like(v))[~normal] * (1 + 1e-12))
+
+
+def test_fp8_cache_quantises_what_it_stores_and_nothing_else():
+    wl, cfg = tiny(T=2, L=2, D=1, H=32, nq=4, nkv=2)
+    ws = I.WeightSource(wl, std=0.2)
+    S = 21
+    x = I.prefill_inputs(wl, batch=2, seq=S)
+    exact, c0 = run_prefill(wl, cfg, ws, x, pages=8)
+    c8 = O.PagedKVCache(cfg, 8, 16, kv_format="e4m3")
+    got = O.pt_prefill(cfg, ws, x, c8, [0, 1])
+    # layer 0 caches the same K/V in both runs (its inputs do not depend on any cache): the FP8 pool is the
+    # quantisation of the exact pool, vector by vector, and its scales are the ones kv_scale gives
+    for t in range(cfg.T):
+        for seq in (0, 1):
+            k, v = c0.gather(t, 0, seq, S)
+            k8, v8 = c8.gather(t, 0, seq, S)
+            for a, b in ((k, k8), (v, v8)):
+                codes, s = O.kv_quantize(a)
+                np.testing.assert_array_equal(b, codes * s)
+    assert np.all(np.log2(c8.scale) == np.round(np.log2(c8.scale)))
+    assert np.all(c0.scale == 1.0)
+    # the output moves by the quantisation error of attention's inputs and by no more: a few percent of its scale
+    rel = np.abs(got - exact).max() / np.abs(exact).max()
+    assert 1e-4 < rel < 0.1
+    # Algorithm 1's invariants survive: a decode step equals a prefill row, chunked prefill equals one prefill
+    # (each vector is quantised on its own, so it does not matter in which call it was written)
+    c8b = O.PagedKVCache(cfg, 8, 16, kv_format="e4m3")
+    first = O.pt_prefill(cfg, ws, x[:, :, :10], c8b, [0, 1])
+    np.testing.assert_allclose(first, got[:, :10], rtol=1e-12, atol=1e-13)
+    rest = O.pt_prefill(cfg, ws, x[:, :, 10:S - 1], c8b, [0, 1])
+    np.testing.assert_allclose(rest, got[:, 10:S - 1], rtol=1e-12, atol=1e-13)
+    last = O.pt_decode_step(cfg, ws, x[:, :, S - 1], c8b, [0, 1])
+    np.testing.assert_allclose(last, got[:, S - 1], rtol=1e-12, atol=1e-13)
