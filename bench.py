@@ -121,14 +121,20 @@ class ClockSampler:
 
 # ------------------------------------------------------------------------------ workloads
 
+def kv8(wl):
+    """Workloads whose name ends in _kv8 keep their cache in the E4M3 format (8-bit codes + one fp32 scale per vector)."""
+    return wl.name.endswith("_kv8")
+
+
 def algorithmic(wl, B, lens=None, S=None):
     """Algorithmic work of one step (no padding, no re-reads, causal triangle only)."""
     P = wl.params_per_track_layer()
     dh = wl.head_dim
     if wl.mode == "decode":
         keys = int(np.sum(np.asarray(lens, np.int64) + 1))
-        kv_read = wl.T * wl.L * 2 * wl.kv_heads * dh * 2 * keys
-        kv_write = wl.T * wl.L * 2 * wl.kv_heads * dh * 2 * B
+        vec_bytes = dh + 4 if kv8(wl) else dh * 2          # one cached vector: codes + scale, or bf16 values
+        kv_read = wl.T * wl.L * 2 * wl.kv_heads * vec_bytes * keys
+        kv_write = wl.T * wl.L * 2 * wl.kv_heads * vec_bytes * B
         weights = wl.T * wl.L * P * 2
         return {"bytes": kv_read + kv_write + weights, "kv_read_bytes": kv_read, "weight_bytes": weights,
                 "attn_bytes_per_layer": kv_read // wl.L}
@@ -180,7 +186,7 @@ def run_decode(wl, dev, steps, warmup, barrier, rank):
     model = make_model(wl, dev, max_pos=int(lens_all.max()) + 16)
     # choose the batch: everything, or the largest prefix (multiple of 16) whose pages fit
     free, _ = torch.cuda.mem_get_info(dev)
-    page_bytes = wl.T * wl.L * 2 * wl.kv_heads * ps * wl.head_dim * 2
+    page_bytes = wl.T * wl.L * 2 * wl.kv_heads * ps * ((wl.head_dim + 4) if kv8(wl) else wl.head_dim * 2)
     pages_of = (lens_all.astype(np.int64) + 1 + ps - 1) // ps
     budget = free - (6 << 30)
     B = wl.batch
@@ -188,7 +194,7 @@ def run_decode(wl, dev, steps, warmup, barrier, rank):
         B -= 16
     lens = lens_all[:B]
     num_pages = int(pages_of[:B].sum())
-    cache = model.new_cache(num_pages, ps)
+    cache = model.new_cache(num_pages, ps, kv_dtype="e4m3" if kv8(wl) else "model")
     seq_ids = list(range(B))
     # fill the cache by real prefills of N(0,1) inputs, grouped by length, in bounded sub-batches
     g = torch.Generator(device=dev).manual_seed(rank_batch_seed(wl.seed, rank))
@@ -252,9 +258,9 @@ def run_decode(wl, dev, steps, warmup, barrier, rank):
     attn_avg_ms = attn_ms / max(attn_n, 1) if attn_n else float("nan")
     achieved = alg["attn_bytes_per_layer"] / (attn_avg_ms * 1e-3) / 1e9
     ratio, why_not = decode_attn_traffic_ratio()
-    if ratio is not None and not (wl.head_dim == 128 and wl.page_size == 16 and wl.dtype == "bf16"):
+    if ratio is not None and not (wl.head_dim == 128 and wl.page_size == 16 and wl.dtype == "bf16" and not kv8(wl)):
         ratio, why_not = None, "counters were taken on head_dim 128, 16-token pages, bf16 cache"
-    roof = {"bound": "hbm", "kernel": "k_decode_attn", "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s",
+    roof = {"bound": "hbm", "kernel": "k_decode_attn_e4m3" if kv8(wl) else "k_decode_attn_tma", "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s",
             "frac": achieved / pk["hbm_gbs"],
             "traffic": alg["attn_bytes_per_layer"] * ratio if ratio else None, "traffic_note": why_not,
             "peak_kind": f"of {pk_kind}", "avg_launch_ms": attn_avg_ms, "launches": attn_n,
@@ -285,7 +291,8 @@ def run_decode(wl, dev, steps, warmup, barrier, rank):
            "e2e": {"value": B / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": xh.numel() * 2,
                    "d2h_bytes_per_step": oh.numel() * 4},
            "config": {"workload": f"{wl.name}: decode T={wl.T} L={wl.L} D={wl.D} H={wl.hidden} heads={wl.heads}/{wl.kv_heads} "
-                                  f"F={wl.ffn} batch={B} kv_len={'U[%d,%d]' % wl.ragged if wl.ragged else wl.seq} page={ps}",
+                                  f"F={wl.ffn} batch={B} kv_len={'U[%d,%d]' % wl.ragged if wl.ragged else wl.seq} page={ps}"
+                                  f" cache={'e4m3 codes + fp32 scale per vector' if kv8(wl) else 'bf16'}",
                       "batch": B, "batch_requested": wl.batch, "kv_tokens": int(lens.sum()), "cache_fill_s": round(t_fill, 2),
                       "l2": "working set (KV cache + weights) far larger than L2; no flush needed"}}
     cache.close()
@@ -477,7 +484,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2")
-    ap.add_argument("--extra", default="cfg3,cfg4,cfg1,cfg0", help="comma-separated workloads reported under 'extra' (N=1 only); '' for none")
+    ap.add_argument("--extra", default="cfg3,cfg4,cfg4_kv8,cfg1,cfg0", help="comma-separated workloads reported under 'extra' (N=1 only); '' for none")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--parallel", default="replicas", choices=["replicas", "tracks"],
                     help="N > 1: 'replicas' = every rank runs the whole model on its own batch (weak scaling, no collective); "

@@ -53,6 +53,15 @@ typedef enum {
 
 typedef enum { PT_F32 = 0, PT_BF16 = 1 } pt_dtype;
 
+/* Storage format of the KV cache.  PT_KV_MODEL keeps K and V in the model dtype.  PT_KV_E4M3 (bf16 models
+ * on the tensor-core path, head_dim 128, pages of a multiple of 16 tokens) halves the cache: every cached
+ * vector (one token, one KV head, K or V) is stored as head_dim E4M3 codes (1 sign, 4 exponent bits with
+ * bias 7, 3 mantissa bits; largest value 448) and one fp32 scale, the smallest power of two s (not below
+ * 2^-100) with max|v| / s <= 448 (1 for an all-zero vector); a code is v / s rounded to nearest even,
+ * saturating.  Attention reads code * s.  The paper has no cache and no such format: it is this library's
+ * own, there so that the ragged decode workload fits one device whole. */
+typedef enum { PT_KV_MODEL = 0, PT_KV_E4M3 = 1 } pt_kv_dtype;
+
 typedef enum {
     PT_WQ = 0, PT_WK = 1, PT_WV = 2, PT_WO = 3, PT_WG = 4, PT_WU = 5, PT_WD = 6,
     PT_G1 = 7, /* RMSNorm gain before attention */
@@ -119,12 +128,17 @@ int32_t pt_sync_count(const pt_model* m);
  * starts as 0, 1, 2, ...; released pages go to the back in block-table order. */
 
 pt_status pt_kv_cache_bytes(const pt_model* m, int32_t num_pages, int32_t page_size, size_t* bytes);
+/* The same for a cache of the given pt_kv_dtype.  An E4M3 pool is the codes, laid out as above with one byte
+ * per element, followed (256-byte aligned) by the fp32 scales [T][L][page][K|V][kv_head][slot]. */
+pt_status pt_kv_cache_bytes_ex(const pt_model* m, int32_t num_pages, int32_t page_size, int32_t kv_dtype, size_t* bytes);
 
 /* Wrap the caller-owned device buffer `dev_pool` (256-byte aligned) as a cache of `num_pages`
  * pages of `page_size` tokens (16 is the tuned size; any multiple of 8 up to 64 is accepted).
  * Host only: the pool's contents are left as they are. */
 pt_status pt_kv_cache_alloc(const pt_model* m, int32_t num_pages, int32_t page_size,
                             void* dev_pool, size_t bytes, pt_kv_cache** out);
+pt_status pt_kv_cache_alloc_ex(const pt_model* m, int32_t num_pages, int32_t page_size, int32_t kv_dtype,
+                               void* dev_pool, size_t bytes, pt_kv_cache** out);
 void pt_kv_cache_free(pt_kv_cache* c);
 
 /* Replace the free list by `order` (host, a permutation of 0..num_pages-1).  Only while no
@@ -147,12 +161,24 @@ pt_status pt_kv_block_table(const pt_kv_cache* c, int32_t seq, int32_t* pages, i
 pt_status pt_kv_slot(const pt_kv_cache* c, int32_t track, int32_t layer, int32_t seq, int32_t pos,
                      int32_t kv, int32_t kv_head, int64_t* elem_offset);
 
+/* E4M3 caches: byte offset, from the start of the pool, of the fp32 scale of the vector that pt_kv_slot
+ * addresses (there the offset counts one-byte codes).  PT_ERR_STATE for a cache in the model dtype. */
+pt_status pt_kv_scale_slot(const pt_kv_cache* c, int32_t track, int32_t layer, int32_t seq, int32_t pos,
+                           int32_t kv, int32_t kv_head, int64_t* byte_offset);
+
 /* ---- forward pass --------------------------------------------------------------------------- */
 
 /* Bytes of workspace (device) that pt_prefill / pt_decode_step need for up to `max_tokens`
  * = B*S tokens and `max_batch` sequences per call. */
 pt_status pt_workspace_bytes(const pt_model* m, int64_t max_tokens, int32_t max_batch,
                              int32_t page_size, size_t* bytes);
+/* The same for calls on a cache of the given pt_kv_dtype.  With an E4M3 cache the projections' K and V pass
+ * through a bf16 staging area on their way into the cache, and a prefill call attends to a bf16 copy of
+ * code * scale of every key its sequences hold: `max_context` bounds, over one prefill call, the sum over its
+ * sequences of the cached length after the call, each rounded up to 16 (0 = prefill calls only ever start
+ * from empty sequences: max_tokens + 16 * max_batch is used).  Decode calls need no such copy. */
+pt_status pt_workspace_bytes_ex(const pt_model* m, int64_t max_tokens, int32_t max_batch, int32_t page_size,
+                                int32_t kv_dtype, int64_t max_context, size_t* bytes);
 
 /* Algorithm 1 over B sequences of S new tokens each.
  *   x         device, 16-byte aligned, model dtype, [T][B][S][hidden]; track t starts at
@@ -163,6 +189,7 @@ pt_status pt_workspace_bytes(const pt_model* m, int64_t max_tokens, int32_t max_
  *             to everything cached for it, themselves included causally
  *   out_h     device, 32-byte aligned, fp32 [B][S][hidden]: the activation h after the last sync
  *   workspace device, 256-byte aligned, >= pt_workspace_bytes(B*S, B, page_size)
+ *             (pt_workspace_bytes_ex for an E4M3 cache)
  * On success the sequences' lengths grow by S.  Errors: PT_ERR_CACHE_FULL,
  * PT_ERR_BUFFER_TOO_SMALL, PT_ERR_INVALID_ARG (position >= max_pos, duplicate ids),
  * PT_ERR_STATE (weights not bound), PT_ERR_CUDA.  Kernel-side faults are reported through

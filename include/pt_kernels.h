@@ -91,6 +91,15 @@ pt_status pt_kernel_decode_attn_static(const void* q, const void* pool_l, int64_
                                        int32_t T, int32_t B, int32_t nq, int32_t nkv, int32_t dh, int32_t ps,
                                        int32_t num_pages, void* out, void* status, void* stream);
 
+/* The quantiser of the E4M3 KV-cache format alone (pt_kv_dtype PT_KV_E4M3 in pt.h; the paper has no cache, the
+ * format is this library's): for each of n vectors of 128 bf16 values
+ *   scales[i] = the smallest power of two s >= 2^-100 with max|v| / s <= 448 (1 for an all-zero vector)
+ *   codes[i][j] = v[j] / s rounded to the nearest E4M3 value, ties to even, saturating at +-448.
+ *   src     device bf16 [n][128], 8-byte aligned        codes  device uint8 [n][128]
+ *   scales  device fp32 [n]                             status device int32[16], zeroed by the caller
+ * Asynchronous on `stream`; nothing is allocated. */
+pt_status pt_kernel_kv_quant_e4m3(const void* src, void* codes, float* scales, int64_t n, void* status, void* stream);
+
 /* ---- the bounded wait, exercised ------------------------------------------------------------
  * Every device-side wait of the library (an mbarrier of a TMA -> MMA -> epilogue pipeline) gives up
  * after a time limit (2 s of device time, whatever the iteration counts), records PT_ERR_DEVICE_TIMEOUT with

@@ -133,7 +133,8 @@ def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, qpos: np.ndarray) -> 
 # Not in the paper (it has no cache at all): a declared storage format for K and V that halves the
 # bytes of the cache, so that the ragged decode workload fits one device whole.  Every cached vector
 # (one token, one KV head, head_dim values, K or V) is stored as E4M3 codes times one scale:
-#   scale = the smallest power of two s with max|v| / s <= 448   (1 for an all-zero vector)
+#   scale = the smallest power of two s >= 2^-100 with max|v| / s <= 448   (1 for an all-zero vector;
+#           the floor keeps the scale a normal fp32 number whatever the vector holds)
 #   code  = v / s rounded to the nearest E4M3 value, ties to the even mantissa, saturating at +-448
 # E4M3 (the "FN" variant of the OCP 8-bit floating point formats): 1 sign, 4 exponent (bias 7) and 3
 # mantissa bits; normal values (1 + m/8) * 2^(e-7) for e = 1..15 (the code e = 15, m = 7 is NaN, so the
@@ -158,7 +159,7 @@ def kv_scale(v: np.ndarray) -> np.ndarray:
     """Power-of-two scale of each vector along the last axis (shape [..., 1])."""
     amax = np.max(np.abs(np.asarray(v, np.float64)), axis=-1, keepdims=True)
     with np.errstate(divide="ignore"):
-        e = np.ceil(np.log2(np.where(amax > 0, amax, 1.0) / E4M3_MAX))
+        e = np.maximum(np.ceil(np.log2(np.where(amax > 0, amax, 1.0) / E4M3_MAX)), -100.0)
     return np.where(amax > 0, np.exp2(e), 1.0)
 
 

@@ -26,22 +26,28 @@ void set_error(const char* fmt, ...) {
     pt::set_error("%s failed: %s", #call, cudaGetErrorString(e_)); return PT_ERR_CUDA; } } while (0)
 
 
-static size_t meta_bytes(int64_t M, int B, int maxp) {
+static size_t meta_bytes(int64_t M, int B, int maxp, bool fp8) {
     size_t b = 0;
     b += align_up((size_t)M * 8, 256);                 // row_kvoff
     b += align_up((size_t)M * 4, 256) * 2;             // row_pos, row_b
     b += align_up((size_t)B * 4, 256) * 2;             // kvlen, nsplit
     b += align_up((size_t)B * maxp * 4, 256);          // block table rows
     b += align_up((size_t)B * kMaxSplits * 16, 256);   // decode work items
+    if (fp8) {
+        b += align_up((size_t)M * 8, 256) * 2;         // row_stageoff, row_attnoff
+        b += align_up((size_t)B * 4, 256);             // ctx_start
+        b += align_up((size_t)B * ((size_t)maxp * 4 + 1) * 4, 256);   // pages of the attention copy (16 tokens each; cache pages hold up to 64)
+    }
     return b;
 }
 
-// Carve the workspace; with base == nullptr only the size is computed.
-static size_t carve(const pt_model* m, int64_t M, int B, int maxp, char* base, Work* w) {
+// Carve the workspace; with base == nullptr only the size is computed.  fp8: the cache holds E4M3 codes;
+// ctx_keys: keys of the attention copy a prefill call needs (0 for a decode call).
+static size_t carve(const pt_model* m, int64_t M, int B, int maxp, bool fp8, int64_t ctx_keys, char* base, Work* w) {
     const pt_config& c = m->cfg;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes, 256); return base ? base + o : nullptr; };
-    char* meta = (char*)take(meta_bytes(M, B, maxp));
+    char* meta = (char*)take(meta_bytes(M, B, maxp, fp8));
     size_t TMH = (size_t)c.T * M * c.hidden;
     float* hT = (float*)take(TMH * 4);
     float* hS = (float*)take((size_t)M * c.hidden * 4);
@@ -52,7 +58,10 @@ static size_t carve(const pt_model* m, int64_t M, int B, int maxp, char* base, W
     void* z = take((size_t)c.T * M * c.ffn * m->esz);
     float* ssq = m->tc ? (float*)take((size_t)c.T * M * ((c.hidden + kSsqTile - 1) / kSsqTile) * 4) : nullptr;
     float* part = m->tc ? (float*)take((size_t)c.T * B * kMaxSplits * c.heads * (m->dh + 2) * 4) : nullptr;
+    void* kv_stage = fp8 ? take((size_t)c.T * 2 * m->KVD * M * 2) : nullptr;
+    void* attn_kv = fp8 && ctx_keys > 0 ? take((size_t)c.T * 2 * m->KVD * (size_t)ctx_keys * 2) : nullptr;
     if (w) {
+        w->kv_stage = kv_stage; w->attn_kv = attn_kv;
         w->hT = hT; w->hS = hS; w->a = a; w->qkv = qkv; w->o = o; w->gu = gu; w->z = z;
         w->ssq = ssq; w->part = part; w->total = off;
         (void)meta;
@@ -254,25 +263,55 @@ pt_status pt_model_set_weight(pt_model* m, int32_t track, int32_t layer, int32_t
 
 /* ------------------------------------------------------------------ KV cache (host logic) */
 
-pt_status pt_kv_cache_bytes(const pt_model* m, int32_t num_pages, int32_t page_size, size_t* bytes) {
-    if (!m || !bytes) PT_FAIL(PT_ERR_INVALID_ARG, "null argument");
+// Bytes of the codes (or model-dtype values) of a pool; an E4M3 pool's scales follow, 256-byte aligned.
+static pt_status kv_pool_layout(const pt_model* m, int32_t num_pages, int32_t page_size, int32_t kv_dtype,
+                                size_t* codes_bytes, size_t* total) {
+    if (!m) PT_FAIL(PT_ERR_INVALID_ARG, "null argument");
     if (num_pages < 1) PT_FAIL(PT_ERR_INVALID_ARG, "num_pages must be >= 1");
     if (page_size < 8 || page_size > 64 || page_size % 8) PT_FAIL(PT_ERR_INVALID_ARG, "page_size must be a multiple of 8 in [8, 64]");
-    *bytes = (size_t)m->cfg.T * m->cfg.L * num_pages * 2 * m->cfg.kv_heads * page_size * m->dh * m->esz;
+    if (kv_dtype != PT_KV_MODEL && kv_dtype != PT_KV_E4M3) PT_FAIL(PT_ERR_INVALID_ARG, "kv_dtype must be PT_KV_MODEL or PT_KV_E4M3");
+    const size_t vecs = (size_t)m->cfg.T * m->cfg.L * num_pages * 2 * m->cfg.kv_heads * page_size;
+    if (kv_dtype == PT_KV_E4M3) {
+        if (!m->tc) PT_FAIL(PT_ERR_UNSUPPORTED, "an E4M3 cache needs a bf16 model on the tensor-core path");
+        if (m->dh != 128 || page_size % 16) PT_FAIL(PT_ERR_UNSUPPORTED, "an E4M3 cache needs head_dim 128 and pages of a multiple of 16 tokens");
+        *codes_bytes = align_up(vecs * m->dh, 256);
+        *total = *codes_bytes + vecs * 4;
+    } else {
+        *codes_bytes = vecs * m->dh * m->esz;
+        *total = *codes_bytes;
+    }
     return PT_OK;
+}
+
+pt_status pt_kv_cache_bytes_ex(const pt_model* m, int32_t num_pages, int32_t page_size, int32_t kv_dtype, size_t* bytes) {
+    if (!bytes) PT_FAIL(PT_ERR_INVALID_ARG, "null argument");
+    size_t codes = 0;
+    return kv_pool_layout(m, num_pages, page_size, kv_dtype, &codes, bytes);
+}
+
+pt_status pt_kv_cache_bytes(const pt_model* m, int32_t num_pages, int32_t page_size, size_t* bytes) {
+    return pt_kv_cache_bytes_ex(m, num_pages, page_size, PT_KV_MODEL, bytes);
 }
 
 pt_status pt_kv_cache_alloc(const pt_model* m, int32_t num_pages, int32_t page_size,
                             void* dev_pool, size_t bytes, pt_kv_cache** out) {
-    size_t need = 0;
+    return pt_kv_cache_alloc_ex(m, num_pages, page_size, PT_KV_MODEL, dev_pool, bytes, out);
+}
+
+pt_status pt_kv_cache_alloc_ex(const pt_model* m, int32_t num_pages, int32_t page_size, int32_t kv_dtype,
+                               void* dev_pool, size_t bytes, pt_kv_cache** out) {
+    size_t need = 0, codes = 0;
     if (!out || !dev_pool) PT_FAIL(PT_ERR_INVALID_ARG, "null argument");
-    pt_status s = pt_kv_cache_bytes(m, num_pages, page_size, &need);
+    pt_status s = kv_pool_layout(m, num_pages, page_size, kv_dtype, &codes, &need);
     if (s != PT_OK) return s;
     if (bytes < need) PT_FAIL(PT_ERR_BUFFER_TOO_SMALL, "KV pool: %zu < %zu bytes", bytes, need);
     if ((uintptr_t)dev_pool % 256) PT_FAIL(PT_ERR_MISALIGNED, "KV pool must be 256-byte aligned");
     pt_kv_cache* c = new (std::nothrow) pt_kv_cache();
     if (!c) PT_FAIL(PT_ERR_INVALID_ARG, "out of host memory");
     c->m = m; c->num_pages = num_pages; c->ps = page_size; c->pool = (char*)dev_pool; c->bytes = bytes;
+    c->kv_dtype = kv_dtype;
+    c->esz = kv_dtype == PT_KV_E4M3 ? 1 : m->esz;
+    c->scales = kv_dtype == PT_KV_E4M3 ? (float*)((char*)dev_pool + codes) : nullptr;
     c->page_elems = (int64_t)2 * m->cfg.kv_heads * page_size * m->dh;
     c->slab_elems = c->page_elems * num_pages;
     for (int i = 0; i < num_pages; ++i) c->free_list.push_back(i);
@@ -360,14 +399,35 @@ pt_status pt_kv_slot(const pt_kv_cache* c, int32_t track, int32_t layer, int32_t
     return PT_OK;
 }
 
+pt_status pt_kv_scale_slot(const pt_kv_cache* c, int32_t track, int32_t layer, int32_t seq, int32_t pos,
+                           int32_t kv, int32_t kv_head, int64_t* byte_offset) {
+    if (!c || !byte_offset) PT_FAIL(PT_ERR_INVALID_ARG, "null argument");
+    if (c->kv_dtype != PT_KV_E4M3) PT_FAIL(PT_ERR_STATE, "the cache holds no scales");
+    int64_t elem = 0;
+    pt_status s = pt_kv_slot(c, track, layer, seq, pos, kv, kv_head, &elem);
+    if (s != PT_OK) return s;
+    *byte_offset = ((char*)c->scales - c->pool) + (elem / c->m->dh) * 4;
+    return PT_OK;
+}
+
 /* ------------------------------------------------------------------ forward */
 
 pt_status pt_workspace_bytes(const pt_model* m, int64_t max_tokens, int32_t max_batch,
                              int32_t page_size, size_t* bytes) {
     if (!m || !bytes) PT_FAIL(PT_ERR_INVALID_ARG, "null argument");
     if (max_tokens < 1 || max_batch < 1 || max_batch > max_tokens || page_size < 8) PT_FAIL(PT_ERR_INVALID_ARG, "bad sizes");
+    return pt_workspace_bytes_ex(m, max_tokens, max_batch, page_size, PT_KV_MODEL, 0, bytes);
+}
+
+pt_status pt_workspace_bytes_ex(const pt_model* m, int64_t max_tokens, int32_t max_batch, int32_t page_size,
+                                int32_t kv_dtype, int64_t max_context, size_t* bytes) {
+    if (!m || !bytes) PT_FAIL(PT_ERR_INVALID_ARG, "null argument");
+    if (max_tokens < 1 || max_batch < 1 || max_batch > max_tokens || page_size < 8 || max_context < 0) PT_FAIL(PT_ERR_INVALID_ARG, "bad sizes");
+    if (kv_dtype != PT_KV_MODEL && kv_dtype != PT_KV_E4M3) PT_FAIL(PT_ERR_INVALID_ARG, "kv_dtype must be PT_KV_MODEL or PT_KV_E4M3");
     int maxp = (m->cfg.max_pos + page_size - 1) / page_size;
-    *bytes = carve(m, max_tokens, max_batch, maxp, nullptr, nullptr);
+    const bool fp8 = kv_dtype == PT_KV_E4M3;
+    const int64_t ctx = fp8 ? std::max<int64_t>(max_context, max_tokens + 16 * (int64_t)max_batch) : 0;
+    *bytes = carve(m, max_tokens, max_batch, maxp, fp8, ctx, nullptr, nullptr);
     return PT_OK;
 }
 
@@ -401,8 +461,18 @@ static pt_status forward(pt_model* m, pt_kv_cache* c, const void* x, int64_t x_s
     }
     if (pages_needed > c->free_list.size()) PT_FAIL(PT_ERR_CACHE_FULL, "call needs %zu new pages, %zu free", pages_needed, c->free_list.size());
     int maxp = (maxlen + c->ps - 1) / c->ps;
+    const bool fp8 = c->kv_dtype == PT_KV_E4M3;
+    if (fp8 && !m->tc) PT_FAIL(PT_ERR_UNSUPPORTED, "an E4M3 cache needs the tensor-core path");
+    // E4M3 cache, prefill: the attention kernel reads a bf16 copy of code * scale of every key of the call's sequences
+    int64_t ctx_keys = 0;
+    if (fp8 && !decode)
+        for (int b = 0; b < B; ++b) {
+            auto it = c->seqs.find(seq_ids[b]);
+            int len = it == c->seqs.end() ? 0 : it->second.len;
+            ctx_keys += ((int64_t)len + S + 15) / 16 * 16;
+        }
     Call k{};
-    size_t need_ws = carve(m, M, B, maxp, (char*)workspace, &k.w);
+    size_t need_ws = carve(m, M, B, maxp, fp8, ctx_keys, (char*)workspace, &k.w);
     if (ws_bytes < need_ws) PT_FAIL(PT_ERR_BUFFER_TOO_SMALL, "workspace: %zu < %zu bytes", ws_bytes, need_ws);
     for (int b = 0; b < B; ++b) {
         auto it = c->seqs.find(seq_ids[b]);
@@ -411,7 +481,7 @@ static pt_status forward(pt_model* m, pt_kv_cache* c, const void* x, int64_t x_s
         if (s != PT_OK) return s;
     }
     // per-call metadata, one upload
-    size_t mb = meta_bytes(M, B, maxp);
+    size_t mb = meta_bytes(M, B, maxp, fp8);
     m->meta_host.assign(mb, 0);
     char* hb = m->meta_host.data();
     char* db = (char*)workspace;
@@ -439,6 +509,32 @@ static pt_status forward(pt_model* m, pt_kv_cache* c, const void* x, int64_t x_s
             h_kvoff[r] = slab_offset(c, s.pages[pos / c->ps], 0, 0, pos % c->ps);
         }
     }
+    size_t o_stageoff = 0, o_attnoff = 0, o_start = 0, o_btattn = 0;
+    const int maxp_attn = (maxlen + 15) / 16;
+    int max_start = 0;
+    if (fp8) {
+        o_stageoff = sect((size_t)M * 8); o_attnoff = sect((size_t)M * 8); o_start = sect((size_t)B * 4);
+        o_btattn = sect((size_t)B * maxp_attn * 4);
+        int64_t* h_stage = (int64_t*)(hb + o_stageoff);
+        int64_t* h_attn = (int64_t*)(hb + o_attnoff);
+        int32_t* h_start = (int32_t*)(hb + o_start);
+        int32_t* h_bta = (int32_t*)(hb + o_btattn);
+        int32_t base = 0;                                 // first 16-token page of the sequence in the attention copy
+        for (int b = 0; b < B; ++b) {
+            const Seq& s = c->seqs[seq_ids[b]];
+            h_start[b] = s.len;
+            max_start = std::max(max_start, s.len);
+            const int np = (s.len + S + 15) / 16;
+            for (int i = 0; i < np; ++i) h_bta[(size_t)b * maxp_attn + i] = base + i;
+            for (int t = 0; t < S; ++t) {
+                const int pos = s.len + t;
+                const int64_t r = (int64_t)b * S + t;
+                h_stage[r] = r * m->dh;
+                h_attn[r] = ((int64_t)(base + pos / 16) * 2 * g.kv_heads) * 16 * m->dh + (int64_t)(pos % 16) * m->dh;
+            }
+            base += np;
+        }
+    }
     int n_items = 0, max_splits = 1;
     if (decode) plan_decode_splits(h_len, B, c->ps, (int64_t)g.T * g.kv_heads, h_items, h_nsp, &n_items, &max_splits);
     cudaStream_t st = (cudaStream_t)stream;
@@ -449,6 +545,15 @@ static pt_status forward(pt_model* m, pt_kv_cache* c, const void* x, int64_t x_s
     k.w.meta.kvlen = (const int32_t*)(db + o_len);
     k.w.meta.bt = (const int32_t*)(db + o_bt);
     k.w.meta.maxp = maxp;
+    if (fp8) {
+        k.w.meta.row_stageoff = (const int64_t*)(db + o_stageoff);
+        k.w.meta.row_attnoff = (const int64_t*)(db + o_attnoff);
+        k.w.meta.ctx_start = (const int32_t*)(db + o_start);
+        k.w.meta.bt_attn = (const int32_t*)(db + o_btattn);
+        k.w.meta.maxp_attn = maxp_attn;
+        k.w.meta.attn_pages = (int32_t)(ctx_keys / 16);
+        k.w.meta.max_start = max_start;
+    }
     k.m = m; k.c = c; k.B = B; k.S = S; k.M = (int)M; k.x = x; k.x_stride = x_stride;
     k.out = (float*)out_h; k.st = st; k.decode = decode;
     k.n_items = n_items; k.max_splits = max_splits;

@@ -93,10 +93,14 @@ struct pt_model {
 struct pt_kv_cache {
     const pt_model* m;
     int32_t num_pages, ps;
+    int32_t kv_dtype;                     // pt_kv_dtype
+    size_t esz;                           // bytes per cached element: the model's, or 1 for E4M3 codes
     char* pool;
+    float* scales;                        // E4M3: [T][L][page][K|V][kv_head][slot] behind the codes; else null
     size_t bytes;
     int64_t page_elems;                   // 2 * nkv * ps * dh
     int64_t slab_elems;                   // num_pages * page_elems : one (track, layer)
+    int64_t slab_vecs() const { return slab_elems / m->dh; }   // cached vectors (= scales) of one (track, layer)
     std::deque<int32_t> free_list;
     std::unordered_map<int32_t, pt::Seq> seqs;
 };
@@ -111,6 +115,12 @@ struct Meta {
     const int32_t* kvlen;       // [B] cached length including this call's tokens
     const int32_t* bt;          // [B][maxp] block table rows
     int32_t maxp;
+    // E4M3 caches only
+    const int64_t* row_stageoff;  // [M] row * head_dim: where the QKV epilogue puts the row's K head 0 in the staging area
+    const int64_t* row_attnoff;   // [M] prefill: offset of the row's slot (K head 0) inside a track's slab of the attention copy
+    const int32_t* bt_attn;       // [B][maxp_attn] 16-token pages of the attention copy
+    const int32_t* ctx_start;     // [B] keys cached before the call (prefill)
+    int32_t maxp_attn, attn_pages, max_start;
 };
 
 // Workspace carve-up for one call.
@@ -125,6 +135,8 @@ struct Work {
     void* z;        // [T][M][F]
     float* ssq;     // [T][M][H/kSsqTile] partial sums of squares (tc)
     float* part;    // decode split-KV partials
+    void* kv_stage; // E4M3 caches: [T][K|V][kv_head][M][dh] bf16, this call's K and V as projected
+    void* attn_kv;  // E4M3 caches, prefill: [T][page][K|V][kv_head][16][dh] bf16 copy of code * scale of every key attended to
     size_t total;
 };
 

@@ -226,6 +226,7 @@ pt_status pt_generate(pt_model* m, pt_kv_cache* c, const int32_t* dev_prompt, in
     if (s != PT_OK) return s;
     if (!c || !dev_prompt || !seq_ids || !dev_tokens_out || !workspace || B < 1 || S < 1 || n_new < 1) { set_error("bad argument"); return PT_ERR_INVALID_ARG; }
     if ((uintptr_t)workspace % 256) { set_error("workspace must be 256-byte aligned"); return PT_ERR_MISALIGNED; }
+    if (c->kv_dtype != PT_KV_MODEL) { set_error("pt_generate sizes its workspace for a cache in the model dtype: drive pt_prefill / pt_decode_step directly with an E4M3 cache"); return PT_ERR_UNSUPPORTED; }
     char *fwd, *x, *h, *hn, *logits, *tok;
     size_t fwd_bytes;
     size_t need = gen_carve(m, B, S, c->ps, (char*)workspace, &fwd, &fwd_bytes, &x, &h, &hn, &logits, &tok);

@@ -120,6 +120,7 @@ pt_status tc_forward(Call& k) {
     Work& w = k.w;
     if ((int)m->wmaps.size() != g.L) { set_error("weights not bound"); return PT_ERR_STATE; }
     const std::vector<WMaps>& wm = m->wmaps;
+    const bool fp8 = c->kv_dtype == PT_KV_E4M3;       // K and V go through a bf16 staging area into 8-bit codes
     __nv_bfloat16* pool = (__nv_bfloat16*)c->pool;
     const int64_t pool_tstride = (int64_t)g.L * c->slab_elems;
     const int tiles = (H + kSsqTile - 1) / kSsqTile;
@@ -162,6 +163,10 @@ pt_status tc_forward(Call& k) {
             p.q_out = q; p.pool_l = pool_l; p.pool_tstride = pool_tstride; p.slab_elems = c->slab_elems;
             p.row_kvoff = w.meta.row_kvoff; p.row_pos = w.meta.row_pos; p.cs = m->rope_cos(); p.sn = m->rope_sin(); p.cs16 = m->rope_cs16();
             p.nq = g.heads; p.nkv = g.kv_heads; p.dh = m->dh; p.ps = c->ps;
+            if (fp8) {          // the staging area looks like one page of M slots: [K|V][kv_head][row][dh] per track
+                p.pool_l = (__nv_bfloat16*)w.kv_stage; p.pool_tstride = (int64_t)2 * m->KVD * M; p.slab_elems = (int64_t)2 * m->KVD * M;
+                p.row_kvoff = w.meta.row_stageoff; p.ps = M;
+            }
             int bn = gemm_bn(p.N, M, T, EPI_QKV);
             p.kps = gemm_kps(bn, M, p.K, 1);
             p.pair = gemm_pair_ok(bn, M, p.N, p.T);
@@ -169,9 +174,15 @@ pt_status tc_forward(Call& k) {
             ProfScope ps(m, st, 1);
             if ((s = launch_gemm(EPI_QKV, bn, *ta, wm[l].m[0][bn_index(p.pair ? 128 : bn)][kps_index(p.kps)], p, st)) != PT_OK) return s;
         }
+        if (fp8) {
+            ProfScope ps(m, st, 6);
+            if (!k.decode && (s = launch_kv_dequant_ctx(k, l)) != PT_OK) return s;
+            if ((s = launch_kv_quant(k, l)) != PT_OK) return s;
+        }
         {
             ProfScope ps(m, st, 0);
-            if (k.decode) s = launch_decode_attn(k, q, pool_l, o);
+            if (fp8) s = k.decode ? launch_decode_attn_e4m3(k, q, l, o) : launch_flash_prefill_e4m3(k, q, o);
+            else if (k.decode) s = launch_decode_attn(k, q, pool_l, o);
             else s = launch_flash_prefill(k, q, pool_l, o);
         }
         if (s != PT_OK) return s;

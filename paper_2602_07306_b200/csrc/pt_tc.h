@@ -138,4 +138,13 @@ pt_status launch_flash_prefill_tc(const AttnP& p, int T, int dh, cudaStream_t st
 pt_status launch_flash_prefill(Call& k, const __nv_bfloat16* q, const __nv_bfloat16* pool_l, __nv_bfloat16* o);
 pt_status launch_decode_attn(Call& k, const __nv_bfloat16* q, const __nv_bfloat16* pool_l, __nv_bfloat16* o);
 
+// merges the key ranges of a split decode attention (pt_tc_attn.cu)
+pt_status launch_decode_combine(const AttnP& p, int T, int dh, cudaStream_t st);
+
+// pt_tc_kv8.cu: the E4M3 storage format of the KV cache
+pt_status launch_kv_quant(Call& k, int layer);
+pt_status launch_kv_dequant_ctx(Call& k, int layer);
+pt_status launch_flash_prefill_e4m3(Call& k, const __nv_bfloat16* q, __nv_bfloat16* o);
+pt_status launch_decode_attn_e4m3(Call& k, const __nv_bfloat16* q, int layer, __nv_bfloat16* o);
+
 }  // namespace pt

@@ -648,6 +648,17 @@ pt_status launch_decode_attn_p(const AttnP& p, int T, int dh, int n_items, int m
     return PT_OK;
 }
 
+pt_status launch_decode_combine(const AttnP& p, int T, int dh, cudaStream_t st) {
+    const dim3 grid((p.B * p.nq * 32 + 127) / 128, T);
+    cudaError_t e;
+    if (dh == 64) e = launch_dependent(k_decode_combine<64>, grid, dim3(128), (size_t)0, st, p);
+    else if (dh == 128) e = launch_dependent(k_decode_combine<128>, grid, dim3(128), (size_t)0, st, p);
+    else { set_error("no combine kernel for head_dim %d", dh); return PT_ERR_UNSUPPORTED; }
+    if (e != cudaSuccess) { set_error("k_decode_combine launch: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return PT_OK;
+}
+
 pt_status launch_decode_attn(Call& k, const __nv_bfloat16* q, const __nv_bfloat16* pool_l, __nv_bfloat16* o) {
     AttnP p = make_params(k, q, pool_l, o);
     return launch_decode_attn_p(p, k.m->cfg.T, k.m->dh, k.n_items, k.max_splits, k.st);

@@ -1,0 +1,501 @@
+// The E4M3 storage format of the KV cache (pt_kv_dtype PT_KV_E4M3): every cached vector (one token, one KV
+// head, K or V) is head_dim 8-bit codes and one power-of-two fp32 scale.
+//   k_kv_quant         this call's K and V, as the QKV GEMM left them in the bf16 staging area, into the cache:
+//                      one warp per vector finds max|v|, the scale, the codes; for a prefill it also writes
+//                      code * scale (exact in bf16: a code has four significant bits) into the bf16 copy the
+//                      prefill attention kernel reads
+//   k_kv_dequant_ctx   the keys a prefill call's sequences held before the call, code * scale into that copy
+//   k_decode_attn_e4m3 split-KV decode attention straight from the codes (see its own comment)
+#include <cuda_fp8.h>
+
+#include "pt_tc.h"
+
+namespace pt {
+
+namespace {
+
+constexpr int kDh = 128;                   // the format's kernels are written for head_dim 128
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void report(int* status, int code, int loc) {
+    if (atomicCAS(status, 0, code) == 0) status[1] = loc;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+// two codes (low byte first) -> two floats
+__device__ __forceinline__ float2 codes_to_float2(uint32_t two) {
+    const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)two, __NV_E4M3);
+    return __half22float2(*reinterpret_cast<const __half2*>(&h));
+}
+
+struct QuantP {
+    const __nv_bfloat16* stage; int64_t stage_tstride;   // [T][K|V][kv_head][M][dh]
+    uint8_t* codes_l; int64_t codes_tstride;             // this layer's slab of track 0; bytes between tracks
+    float* scales_l; int64_t scales_tstride;
+    const int64_t* row_kvoff;                            // [M] offset of the row's slot (K head 0) inside a slab, in elements
+    __nv_bfloat16* attn; int64_t attn_tstride;           // prefill: the attention copy (null for a decode step)
+    const int64_t* row_attnoff;
+    int M, nvec, ps;                                     // nvec = 2 * kv_heads vectors per row
+    int64_t slab_elems;
+    int* status;
+};
+
+__global__ void k_kv_quant(const QuantP p) {
+    grid_dep_wait();
+    grid_dep_launch();
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    const int t = blockIdx.y;
+    const int nvec = p.nvec;
+    if (warp >= p.M * nvec) return;
+    const int row = warp / nvec, kvh = warp % nvec;       // kvh = (K|V) * nkv + head
+    const uint2 raw = *reinterpret_cast<const uint2*>(p.stage + (size_t)t * p.stage_tstride + ((size_t)kvh * p.M + row) * kDh + lane * 4);
+    const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&raw.x), b = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
+    const float v0 = __low2float(a), v1 = __high2float(a), v2 = __low2float(b), v3 = __high2float(b);
+    float amax = fmaxf(fmaxf(fabsf(v0), fabsf(v1)), fmaxf(fabsf(v2), fabsf(v3)));
+#pragma unroll
+    for (int o = 16; o; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    // the smallest power of two 2^e >= 2^-100 with amax / 2^e <= 448 = 1.75 * 2^8: with amax = f * 2^x, 1 <= f < 2,
+    // e = x - 8, one more when f > 1.75
+    const uint32_t bits = __float_as_uint(amax);
+    const int xf = (int)(bits >> 23) & 0xff;
+    int e = xf == 0 ? -100 : xf - 127 - 8 + ((bits & 0x7fffffu) > 0x600000u ? 1 : 0);
+    e = max(e, -100);
+    const bool zero = amax == 0.f;
+    const float scale = zero ? 1.0f : __uint_as_float((uint32_t)(e + 127) << 23);
+    const float inv = zero ? 1.0f : __uint_as_float((uint32_t)(127 - e) << 23);
+    const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(v0 * inv, v1 * inv), __NV_SATFINITE, __NV_E4M3);
+    const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(v2 * inv, v3 * inv), __NV_SATFINITE, __NV_E4M3);
+    const int64_t off = (p.row_kvoff ? p.row_kvoff[row] : (int64_t)row * kDh) + (int64_t)kvh * p.ps * kDh;
+    if (off < 0 || off + kDh > p.slab_elems) { if (lane == 0) report(p.status, PT_ERR_DEVICE_BOUNDS, LOC_ROPE_PAGE); return; }
+    *reinterpret_cast<uint32_t*>(p.codes_l + (size_t)t * p.codes_tstride + off + lane * 4) = lo | (hi << 16);
+    if (lane == 0) p.scales_l[(size_t)t * p.scales_tstride + off / kDh] = scale;
+    if (p.attn) {
+        const float2 d0 = codes_to_float2(lo), d1 = codes_to_float2(hi);
+        uint2 o;
+        o.x = pack_bf16(d0.x * scale, d0.y * scale);
+        o.y = pack_bf16(d1.x * scale, d1.y * scale);
+        *reinterpret_cast<uint2*>(p.attn + (size_t)t * p.attn_tstride + p.row_attnoff[row] + (int64_t)kvh * 16 * kDh + lane * 4) = o;
+    }
+}
+
+struct CtxP {
+    const uint8_t* codes_l; int64_t codes_tstride;
+    const float* scales_l; int64_t scales_tstride;
+    __nv_bfloat16* attn; int64_t attn_tstride;
+    const int32_t* bt; int maxp;                          // the cache's block table
+    const int32_t* bt_attn; int maxp_attn;                // 16-token pages of the attention copy
+    const int32_t* start;                                 // [B] keys cached before the call
+    int nkv, ps, num_pages;
+    int* status;
+};
+
+__global__ void k_kv_dequant_ctx(const CtxP p) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    const int b = blockIdx.y, t = blockIdx.z;
+    const int nvec = 2 * p.nkv;
+    const int pos = warp / nvec, kvh = warp % nvec;
+    if (pos >= p.start[b]) return;
+    const int page = p.bt[(size_t)b * p.maxp + pos / p.ps];
+    if (page < 0 || page >= p.num_pages) { if (lane == 0) report(p.status, PT_ERR_DEVICE_BOUNDS, LOC_FLASH_PAGE); return; }
+    const int64_t vi = ((int64_t)page * nvec + kvh) * p.ps + pos % p.ps;
+    const uint32_t w = *reinterpret_cast<const uint32_t*>(p.codes_l + (size_t)t * p.codes_tstride + vi * kDh + lane * 4);
+    const float scale = p.scales_l[(size_t)t * p.scales_tstride + vi];
+    const float2 d0 = codes_to_float2(w & 0xffffu), d1 = codes_to_float2(w >> 16);
+    uint2 o;
+    o.x = pack_bf16(d0.x * scale, d0.y * scale);
+    o.y = pack_bf16(d1.x * scale, d1.y * scale);
+    const int64_t dst = (((int64_t)p.bt_attn[(size_t)b * p.maxp_attn + pos / 16] * nvec + kvh) * 16 + pos % 16) * kDh;
+    *reinterpret_cast<uint2*>(p.attn + (size_t)t * p.attn_tstride + dst + lane * 4) = o;
+}
+
+
+// ---- decode attention straight from the codes -------------------------------------------------------
+// Same work split as the bf16 kernel: a CTA = one (track, sequence, KV head, key range), each of its 4 warps
+// streams its own 16-token groups through a private ring (one TMA box of 16 x 128 code bytes for K, one for V,
+// two 64-byte bulk copies for their scales, all on the slot's mbarrier), the G query heads of the KV head are
+// the rows of an mma.sync m16n8k16 tile.  Codes become f16 (exact) on their way into the MMA's B fragments:
+//   scores  the contraction index of a k-step is mapped to head_dim as kappa {2q, 2q+1, 2q+8, 2q+9} <->
+//           16 ks + 4q + {0, 1, 2, 3} (q = lane % 4), so a thread's two B registers are one 32-bit load of four
+//           consecutive codes of its key's row; q is loaded in the same order.  The K scale multiplies the score.
+//   P V     a thread needs the codes of keys {2q, 2q+1, 2q+8, 2q+9} at one head_dim column: it loads four
+//           consecutive columns 32 m + 4 g + {0..3} (g = lane / 4) of those four rows and takes byte i of each for
+//           the n-tile (m, i), whose column g therefore stands for head_dim 32 m + 4 g + i; the accumulators are
+//           put back in order when they are merged.  V codes are multiplied by their scale as f16 pairs, so a
+//           cached V value must fit f16 (|v| <= 65504; below 2^-24 it flushes to zero).
+// With the 128-byte swizzle of the boxes both access patterns are free of bank conflicts.
+constexpr int kDecStages = 3;
+constexpr uint32_t kDecSpin = 1u << 24;
+constexpr int kSlotBytes = 2 * 16 * kDh;                  // K box + V box
+constexpr int kDecThreads = 128;
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                 ::"r"(dst), "l"((uint64_t)map), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mma_f16(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t codes_to_half2(uint32_t two) {
+    const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)two, __NV_E4M3);
+    return *reinterpret_cast<const uint32_t*>(&h);
+}
+__device__ __forceinline__ uint32_t pack_half2(float a, float b) {
+    const __half2 h = __floats2half2_rn(a, b);
+    return *reinterpret_cast<const uint32_t*>(&h);
+}
+// byte offset of byte `c` of row `r` inside a 16 x 128-byte box in the 128-byte swizzle
+__device__ __forceinline__ uint32_t box_off(int r, int c) { return (uint32_t)(r * 128 + ((((c >> 4) ^ (r & 7))) << 4) + (c & 15)); }
+
+struct Dec8P {
+    AttnP a;                          // q, o, bt, kvlen, items, nsplit, part ... (pool_l unused)
+    const float* scales_l; int64_t scales_tstride;
+};
+
+__global__ void __launch_bounds__(kDecThreads)
+k_decode_attn_e4m3(const __grid_constant__ CUtensorMap kvmap, const Dec8P pp) {
+    const AttnP& p = pp.a;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    float* sc_area = (float*)(smem + 4 * kDecStages * kSlotBytes);              // [warp][stage][K|V][16]
+    uint64_t* bars = (uint64_t*)(sc_area + 4 * kDecStages * 32);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    grid_dep_wait();                                          // q and this step's codes come from the kernels before it
+    grid_dep_launch();
+    const int32_t* item = p.items + (size_t)blockIdx.x * 4;
+    const int b = item[0], kstart = item[1], kcount = item[2], split = item[3];
+    const int kvh = blockIdx.y, t = blockIdx.z;
+    const int G = p.nq / p.nkv;
+    const int key_end = min(kstart + kcount, p.kvlen[b]);
+    const int npages = (key_end - kstart + 15) >> 4;          // 16-token groups of this key range
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 4 * kDecStages; ++i) mbar_init(&bars[i], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    uint8_t* ring = smem + warp * kDecStages * kSlotBytes;
+    float* wsc = sc_area + warp * kDecStages * 32;
+    uint64_t* wbar = bars + warp * kDecStages;
+    bool bad_page = false;
+    auto issue = [&](int gidx) {                              // lane 0: codes and scales of local group gidx into its slot
+        const int key0 = kstart + gidx * 16;
+        int page = p.bt[(size_t)b * p.maxp + key0 / p.ps];
+        if (page < 0 || page >= p.num_pages) { bad_page = true; page = 0; }
+        const int slot = (gidx >> 2) % kDecStages;
+        const uint32_t dst = smem_u32(ring + slot * kSlotBytes);
+        const int row_k = ((page * 2 + 0) * p.nkv + kvh) * p.ps + key0 % p.ps;   // index of the group's first vector in the slab
+        const int row_v = row_k + p.nkv * p.ps;
+        const float* sc = pp.scales_l + (size_t)t * pp.scales_tstride;
+        mbar_expect_tx(&wbar[slot], kSlotBytes + 128);
+        tma_load_3d(dst, &kvmap, &wbar[slot], 0, row_k, t);
+        tma_load_3d(dst + 16 * kDh, &kvmap, &wbar[slot], 0, row_v, t);
+        bulk_load(smem_u32(wsc + slot * 32), sc + row_k, 64, &wbar[slot]);
+        bulk_load(smem_u32(wsc + slot * 32 + 16), sc + row_v, 64, &wbar[slot]);
+    };
+
+    const int g = lane >> 2, q4 = lane & 3;
+    uint32_t qf[kDh / 16][4];
+    {
+        const __nv_bfloat16* qrow = p.q + ((size_t)t * p.M + b) * (size_t)(p.nq * kDh) + (size_t)(kvh * G + g) * kDh;
+#pragma unroll
+        for (int ks = 0; ks < kDh / 16; ++ks) {
+            qf[ks][0] = qf[ks][1] = qf[ks][2] = qf[ks][3] = 0u;
+            if (g < G) {
+                const uint2 raw = *reinterpret_cast<const uint2*>(qrow + ks * 16 + q4 * 4);
+                const float2 f0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
+                const float2 f1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
+                qf[ks][0] = pack_half2(f0.x, f0.y);
+                qf[ks][2] = pack_half2(f1.x, f1.y);
+            }
+        }
+    }
+    float o[kDh / 8][4];
+#pragma unroll
+    for (int i = 0; i < kDh / 8; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+    float m_run = -INFINITY, l_run = 0.f;
+
+    if (lane == 0)
+        for (int s = 0; s < kDecStages; ++s) { int gi = warp + 4 * s; if (gi < npages) issue(gi); }
+    bool timed_out = false;
+    int it = 0;
+    for (int gi = warp; gi < npages; gi += 4, ++it) {
+        const int slot = it % kDecStages;
+        const uint32_t parity = (it / kDecStages) & 1;
+        bool ok = false;
+        {
+            WaitClock clock;
+            for (uint32_t spin = 0; spin < kDecSpin; ++spin) {
+                if (mbar_try(&wbar[slot], parity)) { ok = true; break; }
+                if ((spin & 255) == 255 && clock.expired()) break;
+            }
+        }
+        if (!__all_sync(0xffffffffu, ok)) { timed_out = true; break; }
+        uint8_t* kb = ring + slot * kSlotBytes;
+        uint8_t* vb = kb + 16 * kDh;
+        const float* scs = wsc + slot * 32;
+        const int key0 = kstart + gi * 16;
+        const int nvalid = key_end - key0;                    // >= 1
+        if (nvalid < 16) {                                    // tail of the sequence: unused slots may hold anything
+            for (int i = lane; i < (16 - nvalid) * 8; i += 32)
+                *reinterpret_cast<uint4*>(vb + (nvalid + i / 8) * 128 + (i % 8) * 16) = make_uint4(0, 0, 0, 0);
+            __syncwarp();
+        }
+        // this thread's four keys: 2q, 2q+1, 2q+8, 2q+9 (score columns and P V contraction rows alike)
+        const float2 sk01 = *reinterpret_cast<const float2*>(scs + 2 * q4), sk89 = *reinterpret_cast<const float2*>(scs + 8 + 2 * q4);
+        const float2 sv01 = *reinterpret_cast<const float2*>(scs + 16 + 2 * q4), sv89 = *reinterpret_cast<const float2*>(scs + 24 + 2 * q4);
+        float s[2][4] = {};
+#pragma unroll
+        for (int ks = 0; ks < kDh / 16; ++ks) {
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) {
+                const uint32_t w = *reinterpret_cast<const uint32_t*>(kb + box_off(nt * 8 + g, ks * 16 + q4 * 4));
+                mma_f16(s[nt], qf[ks], codes_to_half2(w & 0xffffu), codes_to_half2(w >> 16));
+            }
+        }
+        const bool in0 = 2 * q4 < nvalid, in1 = 2 * q4 + 1 < nvalid, in8 = 8 + 2 * q4 < nvalid, in9 = 9 + 2 * q4 < nvalid;
+        s[0][0] = in0 ? s[0][0] * sk01.x * p.scale_log2 : -INFINITY;
+        s[0][1] = in1 ? s[0][1] * sk01.y * p.scale_log2 : -INFINITY;
+        s[1][0] = in8 ? s[1][0] * sk89.x * p.scale_log2 : -INFINITY;
+        s[1][1] = in9 ? s[1][1] * sk89.y * p.scale_log2 : -INFINITY;
+        float mx = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        const float mn = fmaxf(m_run, mx);
+        const float corr = exp2f(m_run - mn);
+        m_run = mn;
+        float sum = 0.f;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) { s[i][0] = exp2f(s[i][0] - mn); s[i][1] = exp2f(s[i][1] - mn); sum += s[i][0] + s[i][1]; }
+        l_run = l_run * corr + sum;
+        if (__any_sync(0xffffffffu, corr != 1.f)) {
+#pragma unroll
+            for (int i = 0; i < kDh / 8; ++i) { o[i][0] *= corr; o[i][1] *= corr; }
+        }
+        uint32_t pf[4];
+        pf[0] = pack_half2(s[0][0], s[0][1]); pf[1] = 0u;
+        pf[2] = pack_half2(s[1][0], s[1][1]); pf[3] = 0u;
+        const uint32_t hs01 = pack_half2(in0 ? sv01.x : 0.f, in1 ? sv01.y : 0.f);
+        const uint32_t hs89 = pack_half2(in8 ? sv89.x : 0.f, in9 ? sv89.y : 0.f);
+#pragma unroll
+        for (int m = 0; m < kDh / 32; ++m) {
+            const int c = 32 * m + 4 * g;
+            const uint32_t w0 = *reinterpret_cast<const uint32_t*>(vb + box_off(2 * q4, c));
+            const uint32_t w1 = *reinterpret_cast<const uint32_t*>(vb + box_off(2 * q4 + 1, c));
+            const uint32_t w2 = *reinterpret_cast<const uint32_t*>(vb + box_off(2 * q4 + 8, c));
+            const uint32_t w3 = *reinterpret_cast<const uint32_t*>(vb + box_off(2 * q4 + 9, c));
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t sel = (uint32_t)i | ((uint32_t)(4 + i) << 4);
+                uint32_t b0 = codes_to_half2(__byte_perm(w0, w1, sel) & 0xffffu);
+                uint32_t b1 = codes_to_half2(__byte_perm(w2, w3, sel) & 0xffffu);
+                asm("mul.rn.f16x2 %0, %0, %1;" : "+r"(b0) : "r"(hs01));
+                asm("mul.rn.f16x2 %0, %0, %1;" : "+r"(b1) : "r"(hs89));
+                mma_f16(o[m * 4 + i], pf, b0, b1);
+            }
+        }
+        __syncwarp();                                         // every lane is done reading the slot
+        if (lane == 0) {
+            int gn = gi + 4 * kDecStages;
+            if (gn < npages) { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); issue(gn); }
+        }
+    }
+    if (timed_out) {
+        // give the copies this warp still has in flight a bounded chance to land, then give up
+        WaitClock clock;
+        for (int s2 = 0; s2 < kDecStages; ++s2)
+            for (uint32_t spin = 0; spin < (1u << 16); ++spin) {
+                if (mbar_try(&wbar[s2], 0) || mbar_try(&wbar[s2], 1)) break;
+                if ((spin & 63) == 63 && clock.expired(100000000ull)) break;
+            }
+        if (lane == 0) report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_DECODE_PAGE);
+    }
+    if (bad_page) report(p.status, PT_ERR_DEVICE_BOUNDS, LOC_DECODE_PAGE);
+    __syncthreads();                                          // every warp has drained its ring
+
+    // merge the four warps' partial (max, sum, output) of the G query heads through shared memory; accumulator
+    // (n-tile nt, column 2q + j) holds head_dim 32 (nt / 4) + 4 (2q + j) + nt % 4
+    float* mg = reinterpret_cast<float*>(smem);
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+    if (g < G) {
+        float* dst = mg + ((size_t)warp * 8 + g) * (kDh + 2);
+#pragma unroll
+        for (int nt = 0; nt < kDh / 8; ++nt) {
+            const int d0 = 32 * (nt >> 2) + 8 * q4 + (nt & 3);
+            dst[d0] = o[nt][0]; dst[d0 + 4] = o[nt][1];
+        }
+        if (q4 == 0) { dst[kDh] = m_run; dst[kDh + 1] = l_run; }
+    }
+    __syncthreads();
+    const int ns = p.nsplit[b];
+    for (int idx = threadIdx.x; idx < G * kDh; idx += kDecThreads) {
+        const int gg = idx / kDh, d = idx % kDh;
+        float Mx = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) Mx = fmaxf(Mx, mg[((size_t)w * 8 + gg) * (kDh + 2) + kDh]);
+        float L = 0.f, acc = 0.f;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            const float* src = mg + ((size_t)w * 8 + gg) * (kDh + 2);
+            const float f = src[kDh] == -INFINITY ? 0.f : exp2f(src[kDh] - Mx);
+            L += src[kDh + 1] * f;
+            acc += src[d] * f;
+        }
+        const int head = kvh * G + gg;
+        if (ns == 1) {
+            p.o[((size_t)t * p.M + b) * (size_t)(p.nq * kDh) + (size_t)head * kDh + d] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
+        } else {
+            float* dst = p.part + ((((size_t)t * p.B + b) * p.nq + head) * p.max_splits + split) * (kDh + 2);
+            dst[d] = acc;
+            if (d == 0) { dst[kDh] = Mx; dst[kDh + 1] = L; }
+        }
+    }
+}
+
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// (code byte, vector of a slab, track) with boxes of 16 vectors x 128 bytes in the 128-byte swizzle
+pt_status make_codes_map(CUtensorMap* out, const void* base, int64_t vecs, int64_t tracks, int64_t track_stride_bytes) {
+    static EncodeFn enc = nullptr;
+    if (!enc) {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qr) == cudaSuccess && qr == cudaDriverEntryPointSuccess)
+            enc = (EncodeFn)f;
+    }
+    if (!enc) { set_error("cuTensorMapEncodeTiled is not available from this driver"); return PT_ERR_CUDA; }
+    cuuint64_t dims[3] = {(cuuint64_t)kDh, (cuuint64_t)vecs, (cuuint64_t)tracks};
+    cuuint64_t strides[2] = {(cuuint64_t)kDh, (cuuint64_t)track_stride_bytes};
+    cuuint32_t box[3] = {(cuuint32_t)kDh, 16, 1};
+    cuuint32_t es[3] = {1, 1, 1};
+    CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, es,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled (E4M3 cache) failed with code %d", (int)r); return PT_ERR_CUDA; }
+    return PT_OK;
+}
+
+}  // namespace
+
+pt_status launch_kv_quant(Call& k, int layer) {
+    const pt_model* m = k.m;
+    const pt_kv_cache* c = k.c;
+    const pt_config& g = m->cfg;
+    QuantP p{};
+    p.stage = (const __nv_bfloat16*)k.w.kv_stage; p.stage_tstride = (int64_t)2 * m->KVD * k.M;
+    p.codes_l = (uint8_t*)c->pool + (size_t)layer * c->slab_elems; p.codes_tstride = (int64_t)g.L * c->slab_elems;
+    p.scales_l = c->scales + (size_t)layer * c->slab_vecs(); p.scales_tstride = (int64_t)g.L * c->slab_vecs();
+    p.row_kvoff = k.w.meta.row_kvoff;
+    p.attn = k.decode ? nullptr : (__nv_bfloat16*)k.w.attn_kv;
+    p.attn_tstride = (int64_t)k.w.meta.attn_pages * 2 * m->KVD * 16;
+    p.row_attnoff = k.w.meta.row_attnoff;
+    p.M = k.M; p.nvec = 2 * g.kv_heads; p.ps = c->ps; p.slab_elems = c->slab_elems; p.status = m->status();
+    const unsigned blocks = (unsigned)(((size_t)k.M * 2 * g.kv_heads + 7) / 8);
+    cudaError_t e = launch_dependent(k_kv_quant, dim3(blocks, g.T), dim3(256), (size_t)0, k.st, p);
+    if (e != cudaSuccess) { set_error("k_kv_quant launch: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return PT_OK;
+}
+
+pt_status launch_kv_dequant_ctx(Call& k, int layer) {
+    const pt_model* m = k.m;
+    const pt_kv_cache* c = k.c;
+    const pt_config& g = m->cfg;
+    if (k.w.meta.max_start <= 0) return PT_OK;
+    CtxP p{};
+    p.codes_l = (const uint8_t*)c->pool + (size_t)layer * c->slab_elems; p.codes_tstride = (int64_t)g.L * c->slab_elems;
+    p.scales_l = c->scales + (size_t)layer * c->slab_vecs(); p.scales_tstride = (int64_t)g.L * c->slab_vecs();
+    p.attn = (__nv_bfloat16*)k.w.attn_kv; p.attn_tstride = (int64_t)k.w.meta.attn_pages * 2 * m->KVD * 16;
+    p.bt = k.w.meta.bt; p.maxp = k.w.meta.maxp; p.bt_attn = k.w.meta.bt_attn; p.maxp_attn = k.w.meta.maxp_attn;
+    p.start = k.w.meta.ctx_start; p.nkv = g.kv_heads; p.ps = c->ps; p.num_pages = c->num_pages; p.status = m->status();
+    const unsigned blocks = (unsigned)(((size_t)k.w.meta.max_start * 2 * g.kv_heads + 7) / 8);
+    k_kv_dequant_ctx<<<dim3(blocks, k.B, g.T), 256, 0, k.st>>>(p);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return PT_OK;
+}
+
+// Prefill attention of a call on an E4M3 cache: the tensor-memory kernel over the bf16 copy of code * scale.
+pt_status launch_flash_prefill_e4m3(Call& k, const __nv_bfloat16* q, __nv_bfloat16* o) {
+    const pt_model* m = k.m;
+    const pt_config& g = m->cfg;
+    AttnP p{};
+    p.q = q; p.o = o;
+    p.pool_l = (const __nv_bfloat16*)k.w.attn_kv; p.pool_tstride = (int64_t)k.w.meta.attn_pages * 2 * m->KVD * 16;
+    p.bt = k.w.meta.bt_attn; p.maxp = k.w.meta.maxp_attn; p.kvlen = k.w.meta.kvlen;
+    p.B = k.B; p.S = k.S; p.M = k.M; p.nq = g.heads; p.nkv = g.kv_heads; p.ps = 16; p.num_pages = k.w.meta.attn_pages;
+    p.scale_log2 = 1.4426950408889634f / sqrtf((float)m->dh);
+    p.status = m->status();
+    return launch_flash_prefill_p(p, g.T, m->dh, (g.flags & 2) != 0, k.st);
+}
+
+pt_status launch_decode_attn_e4m3(Call& k, const __nv_bfloat16* q, int layer, __nv_bfloat16* o) {
+    const pt_model* m = k.m;
+    const pt_kv_cache* c = k.c;
+    const pt_config& g = m->cfg;
+    Dec8P pp{};
+    AttnP& p = pp.a;
+    p.q = q; p.o = o; p.bt = k.w.meta.bt; p.maxp = k.w.meta.maxp; p.kvlen = k.w.meta.kvlen;
+    p.B = k.B; p.S = 1; p.M = k.M; p.nq = g.heads; p.nkv = g.kv_heads; p.ps = c->ps; p.num_pages = c->num_pages;
+    p.scale_log2 = 1.4426950408889634f / sqrtf((float)m->dh);
+    p.status = m->status();
+    p.items = k.items; p.nsplit = k.nsplit; p.part = k.w.part; p.max_splits = kMaxSplits;
+    pp.scales_l = c->scales + (size_t)layer * c->slab_vecs(); pp.scales_tstride = (int64_t)g.L * c->slab_vecs();
+    CUtensorMap kvmap;
+    pt_status s = make_codes_map(&kvmap, c->pool + (size_t)layer * c->slab_elems, c->slab_vecs(), g.T, (int64_t)g.L * c->slab_elems);
+    if (s != PT_OK) return s;
+    const int smem = 1024 + 4 * kDecStages * kSlotBytes + 4 * kDecStages * 32 * 4 + 4 * kDecStages * 8;
+    static bool done_[kMaxDevices] = {};
+    bool& done = done_[current_device()];
+    if (!done) {
+        cudaError_t e = cudaFuncSetAttribute(k_decode_attn_e4m3, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) { set_error("cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
+        done = true;
+    }
+    cudaError_t e = launch_dependent(k_decode_attn_e4m3, dim3(k.n_items, g.kv_heads, g.T), dim3(kDecThreads), (size_t)smem, k.st, kvmap, pp);
+    if (e != cudaSuccess) { set_error("k_decode_attn_e4m3 launch: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (k.max_splits > 1) return launch_decode_combine(p, g.T, m->dh, k.st);
+    return PT_OK;
+}
+
+}  // namespace pt
+
+#include "pt_kernels.h"
+
+extern "C" pt_status pt_kernel_kv_quant_e4m3(const void* src, void* codes, float* scales, int64_t n, void* status, void* stream) {
+    using namespace pt;
+    if (!src || !codes || !scales || !status) { set_error("null argument"); return PT_ERR_INVALID_ARG; }
+    if (n < 1 || n > (1 << 28)) { set_error("n outside [1, 2^28]"); return PT_ERR_INVALID_ARG; }
+    if ((uintptr_t)src % 8 || (uintptr_t)codes % 4 || (uintptr_t)scales % 4) { set_error("src must be 8-byte, codes and scales 4-byte aligned"); return PT_ERR_MISALIGNED; }
+    QuantP p{};
+    p.stage = (const __nv_bfloat16*)src; p.codes_l = (uint8_t*)codes; p.scales_l = scales;
+    p.M = (int)n; p.nvec = 1; p.ps = 1; p.slab_elems = n * 128; p.status = (int*)status;
+    k_kv_quant<<<dim3((unsigned)((n + 7) / 8), 1), 256, 0, (cudaStream_t)stream>>>(p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_error("kernel launch failed: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return PT_OK;
+}

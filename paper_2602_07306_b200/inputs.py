@@ -98,6 +98,9 @@ WORKLOADS = {
                      dtype="bf16", mode="prefill", batch=8, seq=4096),
     "cfg4": Workload("cfg4", T=4, L=48, D=6, hidden=2048, heads=16, kv_heads=4, ffn=5632,
                      dtype="bf16", mode="decode", batch=256, seq=0, ragged=(512, 4096)),
+    # The same ragged decode workload with the cache in the library's E4M3 format: the whole batch of 256 fits.
+    "cfg4_kv8": Workload("cfg4_kv8", T=4, L=48, D=6, hidden=2048, heads=16, kv_heads=4, ffn=5632,
+                         dtype="bf16", mode="decode", batch=256, seq=0, ragged=(512, 4096)),
     # The head layout of the paper's 30B PT model (Table 1: 8 tracks, 48 layers, 8 query heads and 1 KV
     # head per track, block depth D in {2, 4, 8}) at the request shapes of its latency tables (batch 1,
     # 1024 .. 63488 prompt tokens).  The paper gives neither the hidden nor the feed-forward width: 8

@@ -20,6 +20,7 @@ STATUS = {0: "PT_OK", 1: "PT_ERR_INVALID_ARG", 2: "PT_ERR_BAD_CONFIG", 3: "PT_ER
           4: "PT_ERR_BUFFER_TOO_SMALL", 5: "PT_ERR_CACHE_FULL", 6: "PT_ERR_MISALIGNED", 7: "PT_ERR_CUDA",
           8: "PT_ERR_DEVICE_BOUNDS", 9: "PT_ERR_DEVICE_TIMEOUT", 10: "PT_ERR_STATE"}
 PT_F32, PT_BF16 = 0, 1
+PT_KV_MODEL, PT_KV_E4M3 = 0, 1
 KIND = {"wq": 0, "wk": 1, "wv": 2, "wo": 3, "wg": 4, "wu": 5, "wd": 6, "g1": 7, "g2": 8}
 
 
@@ -47,6 +48,11 @@ _PROTOS = {
     "pt_model_set_track_group": (_I32, [_P, _I32, _P, _P]),
     "pt_kv_cache_bytes": (_I32, [_P, _I32, _I32, C.POINTER(_SZ)]),
     "pt_kv_cache_alloc": (_I32, [_P, _I32, _I32, _P, _SZ, C.POINTER(_P)]),
+    "pt_kv_cache_bytes_ex": (_I32, [_P, _I32, _I32, _I32, C.POINTER(_SZ)]),
+    "pt_kv_cache_alloc_ex": (_I32, [_P, _I32, _I32, _I32, _P, _SZ, C.POINTER(_P)]),
+    "pt_kv_scale_slot": (_I32, [_P, _I32, _I32, _I32, _I32, _I32, _I32, C.POINTER(_I64)]),
+    "pt_workspace_bytes_ex": (_I32, [_P, _I64, _I32, _I32, _I32, _I64, C.POINTER(_SZ)]),
+    "pt_kernel_kv_quant_e4m3": (_I32, [_P, _P, _P, _I64, _P, _P]),
     "pt_kv_cache_free": (None, [_P]),
     "pt_kv_set_free_list": (_I32, [_P, C.POINTER(_I32), _I32]),
     "pt_kv_seq_reserve": (_I32, [_P, _I32, _I32]),
@@ -212,16 +218,23 @@ class Model:
     def sync_count(self) -> int:
         return lib().pt_sync_count(self.h)
 
-    def new_cache(self, num_pages: int, page_size: int = 16, free_order=None) -> "Cache":
-        return Cache(self, num_pages, page_size, free_order)
+    def new_cache(self, num_pages: int, page_size: int = 16, free_order=None, kv_dtype: str = "model") -> "Cache":
+        """kv_dtype "model" keeps K and V in the model dtype, "e4m3" stores 8-bit codes and one scale per vector."""
+        return Cache(self, num_pages, page_size, free_order, kv_dtype=kv_dtype)
 
-    def workspace(self, tokens: int, batch: int, page_size: int):
-        if self.ws is None or tokens > self.ws_key[0] or batch > self.ws_key[1] or page_size < self.ws_key[2]:
+    def workspace(self, tokens: int, batch: int, page_size: int, kv_dtype: int = PT_KV_MODEL, context: int = 0):
+        """Workspace for calls of up to `tokens` tokens / `batch` sequences; with an E4M3 cache `context` bounds the
+        keys a prefill call attends to (sum over its sequences of the length after the call, each rounded up to 16)."""
+        key = self.ws_key + (0, 0) if len(self.ws_key) == 3 else self.ws_key
+        if (self.ws is None or tokens > key[0] or batch > key[1] or page_size < key[2] or kv_dtype > key[3] or context > key[4]):
+            tokens, batch, context = max(tokens, key[0]), max(batch, key[1]), max(context, key[4])
+            kv_dtype = max(kv_dtype, key[3])
+            page_size = min(page_size, key[2]) if key[2] else page_size
             n = _SZ()
-            check(lib().pt_workspace_bytes(self.h, tokens, batch, page_size, C.byref(n)))
+            check(lib().pt_workspace_bytes_ex(self.h, tokens, batch, page_size, kv_dtype, context, C.byref(n)))
             self.ws = None
             self.ws = self.torch.empty(n.value, dtype=self.torch.uint8, device=self.device)
-            self.ws_key = (tokens, batch, page_size)
+            self.ws_key = (tokens, batch, page_size, kv_dtype, context)
         return self.ws
 
     def set_tap(self, layer: int | None, tokens: int = 0):
@@ -244,9 +257,12 @@ class Model:
         stride = 0 if Tn == 1 and self.cfg.T > 1 else B * S * H
         if out is None:
             out = torch.empty((B, S, H), dtype=torch.float32, device=self.device)
-        ws = self.workspace(B * S, B, cache.page_size)
         ids, pids = _i32arr(seq_ids)
         assert len(ids) == B
+        ctx = 0
+        if cache.kv_dtype == PT_KV_E4M3:
+            ctx = sum((cache.length(int(s)) + S + 15) // 16 * 16 for s in ids)
+        ws = self.workspace(B * S, B, cache.page_size, cache.kv_dtype, ctx)
         with torch.cuda.device(self.device):
             check(lib().pt_prefill(self.h, cache.h, x.data_ptr(), stride, B, S, pids, out.data_ptr(),
                                    ws.data_ptr(), ws.numel(), self._stream()))
@@ -260,7 +276,7 @@ class Model:
         stride = 0 if Tn == 1 and self.cfg.T > 1 else B * H
         if out is None:
             out = torch.empty((B, H), dtype=torch.float32, device=self.device)
-        ws = self.workspace(B, B, cache.page_size)
+        ws = self.workspace(B, B, cache.page_size, cache.kv_dtype, 0)
         ids, pids = _i32arr(seq_ids)
         assert len(ids) == B
         with torch.cuda.device(self.device):
@@ -355,15 +371,25 @@ class Model:
 class Cache:
     """Paged KV cache: torch owns the pool, the library's host allocator owns the page tables."""
 
-    def __init__(self, model: Model, num_pages: int, page_size: int = 16, free_order=None, fill=None):
+    def __init__(self, model: Model, num_pages: int, page_size: int = 16, free_order=None, fill=None, kv_dtype: str = "model"):
         torch = model.torch
         self.model, self.num_pages, self.page_size = model, num_pages, page_size
+        self.kv_dtype = {"model": PT_KV_MODEL, "e4m3": PT_KV_E4M3}[kv_dtype]
         n = _SZ()
-        check(lib().pt_kv_cache_bytes(model.h, num_pages, page_size, C.byref(n)))
+        check(lib().pt_kv_cache_bytes_ex(model.h, num_pages, page_size, self.kv_dtype, C.byref(n)))
         self.bytes = n.value
-        self.pool = torch.empty(n.value // (2 if model.dtype == "bf16" else 4), dtype=model.tdtype, device=model.device)
+        if self.kv_dtype == PT_KV_E4M3:
+            # one byte buffer: the codes, then the fp32 scales (views below)
+            self.pool = torch.empty(n.value, dtype=torch.uint8, device=model.device)
+            c = model.cfg
+            vecs = c.T * c.L * num_pages * 2 * c.kv_heads * page_size
+            dh = c.hidden // c.heads
+            self.codes = self.pool[: vecs * dh]
+            self.scales = self.pool[n.value - vecs * 4:].view(torch.float32)
+        else:
+            self.pool = torch.empty(n.value // (2 if model.dtype == "bf16" else 4), dtype=model.tdtype, device=model.device)
         self.h = _P()
-        check(lib().pt_kv_cache_alloc(model.h, num_pages, page_size, self.pool.data_ptr(), n.value, C.byref(self.h)))
+        check(lib().pt_kv_cache_alloc_ex(model.h, num_pages, page_size, self.kv_dtype, self.pool.data_ptr(), n.value, C.byref(self.h)))
         if free_order is not None:
             a, p = _i32arr(free_order)
             check(lib().pt_kv_set_free_list(self.h, p, len(a)))
@@ -405,6 +431,21 @@ class Cache:
         check(lib().pt_kv_slot(self.h, t, l, seq, pos, kv, head, C.byref(v)))
         return v.value
 
+    def scale_slot(self, t: int, l: int, seq: int, pos: int, kv: int, head: int) -> int:
+        """E4M3 caches: byte offset inside the pool of the fp32 scale of the vector `slot` addresses."""
+        v = _I64()
+        check(lib().pt_kv_scale_slot(self.h, t, l, seq, pos, kv, head, C.byref(v)))
+        return v.value
+
+    def dequantized(self):
+        """E4M3 caches: code * scale of the whole pool as a float32 CUDA tensor [T, L, pages, 2, kv_heads, page, dh]."""
+        torch = self.model.torch
+        c = self.model.cfg
+        dh = c.hidden // c.heads
+        shape = (c.T, c.L, self.num_pages, 2, c.kv_heads, self.page_size)
+        codes = self.codes.view(torch.float8_e4m3fn).to(torch.float32).view(shape + (dh,))
+        return codes * self.scales.view(shape + (1,))
+
 
 def kernel_gemm_bf16(a, w, bn: int = 0, fold_tracks: bool = False):
     """a [T, M, K], w [T, N, K] bf16 CUDA tensors -> fp32 [T, M, N] ([1, M, N] when folding tracks)."""
@@ -418,6 +459,20 @@ def kernel_gemm_bf16(a, w, bn: int = 0, fold_tracks: bool = False):
         check(lib().pt_kernel_gemm_bf16(a.data_ptr(), w.data_ptr(), c.data_ptr(), T, M, N, K, bn, int(fold_tracks),
                                         status.data_ptr(), torch.cuda.current_stream().cuda_stream))
     return c, status
+
+
+def kernel_kv_quant_e4m3(src):
+    """src: bf16 CUDA tensor [n, 128] -> (codes uint8 [n, 128], scales fp32 [n], status int32[16])."""
+    import torch
+    assert src.is_cuda and src.dtype == torch.bfloat16 and src.is_contiguous() and src.shape[1] == 128
+    n = src.shape[0]
+    codes = torch.empty((n, 128), dtype=torch.uint8, device=src.device)
+    scales = torch.empty(n, dtype=torch.float32, device=src.device)
+    status = torch.zeros(16, dtype=torch.int32, device=src.device)
+    with torch.cuda.device(src.device):
+        check(lib().pt_kernel_kv_quant_e4m3(src.data_ptr(), codes.data_ptr(), scales.data_ptr(), n, status.data_ptr(),
+                                            torch.cuda.current_stream().cuda_stream))
+    return codes, scales, status
 
 
 def kernel_wait_selftest(limit_ns: int, device="cuda:0"):

@@ -24,14 +24,15 @@ from paper_2602_07306_b200 import inputs as I
 FLOOR_MARGIN = 1.10
 
 
-def _layer(h, w, pos, nq, nkv, dh, rnd):
+def _layer(h, w, pos, nq, nkv, dh, rnd, kv8=False):
     R = (lambda a: I.round_to_bf16(np.asarray(a, np.float32)).astype(np.float64)) if rnd else (lambda a: a)
+    Q8 = (lambda a: (lambda cs: cs[0] * cs[1])(O.kv_quantize(a))) if kv8 else (lambda a: a)
     S = h.shape[0]
     rinv = 1.0 / np.sqrt(np.mean(h * h, -1, keepdims=True) + 1e-6)
     a = R(h * w["g1"]) * rinv
     q = R(O.rope((a @ w["wq"].T).reshape(S, nq, dh), pos, 1e4))
-    k = R(O.rope((a @ w["wk"].T).reshape(S, nkv, dh), pos, 1e4))
-    v = R((a @ w["wv"].T).reshape(S, nkv, dh))
+    k = Q8(R(O.rope((a @ w["wk"].T).reshape(S, nkv, dh), pos, 1e4)))
+    v = Q8(R((a @ w["wv"].T).reshape(S, nkv, dh)))
     o = np.empty_like(q)
     for i in range(nq):
         j = i // (nq // nkv)
@@ -46,9 +47,11 @@ def _layer(h, w, pos, nq, nkv, dh, rnd):
 
 
 @functools.lru_cache(maxsize=None)
-def measure(T, D, H, nq, nkv, F, S=12):
+def measure(T, D, H, nq, nkv, F, S=12, kv8=False):
     """(max-rel, mean-rel) of the synced stream after one track block of depth D, T tracks, when only
-    the tensor-core operands and the cache are rounded to bf16."""
+    the tensor-core operands and the cache are rounded to bf16.  kv8: both runs cache K and V in the E4M3
+    format (the exact run quantises its exact K and V, the rounded run its bf16-rounded ones: a value near
+    a code boundary then lands on the neighbouring code, one code step - a sixteenth - away)."""
     wl = I.Workload("block", T=T, L=D, D=D, hidden=H, heads=nq, kv_heads=nkv, ffn=F, dtype="bf16",
                     mode="prefill", batch=1, seq=S)
     ws = I.WeightSource(wl)
@@ -59,19 +62,19 @@ def measure(T, D, H, nq, nkv, F, S=12):
     for l in range(D):
         for t in range(T):
             w = {k: np.asarray(v, np.float64) for k, v in ws.get(t, l).items()}
-            exact[t] = _layer(exact[t], w, pos, nq, nkv, wl.head_dim, False)
-            rounded[t] = _layer(rounded[t], w, pos, nq, nkv, wl.head_dim, True)
+            exact[t] = _layer(exact[t], w, pos, nq, nkv, wl.head_dim, False, kv8)
+            rounded[t] = _layer(rounded[t], w, pos, nq, nkv, wl.head_dim, True, kv8)
     e, r = sum(exact), sum(rounded)                           # the track-sync that closes the block
     d = np.abs(r - e)
     return float(d.max() / np.abs(e).max()), float(d.mean() / np.abs(e).mean())
 
 
-def mean_bound(wl, depth=None):
+def mean_bound(wl, depth=None, kv8=False):
     """Mean-error bound for a bf16 workload: the stated 2e-3 wherever the floor allows it, else
     FLOOR_MARGIN x the floor of the workload's own layer shape (one track block; `depth` caps the
-    block depth measured, the floor does not grow with it)."""
-    if wl.dtype != "bf16" or wl.hidden <= 512:
+    block depth measured).  With an E4M3 cache (kv8) the floor is always measured: code flips dominate it."""
+    if wl.dtype != "bf16" or (wl.hidden <= 512 and not kv8):
         return 2e-3
     D = min(wl.D, depth) if depth else wl.D
-    _, mean = measure(wl.T, D, wl.hidden, wl.heads, wl.kv_heads, wl.ffn)
+    _, mean = measure(wl.T, D, wl.hidden, wl.heads, wl.kv_heads, wl.ffn, kv8=kv8)
     return max(2e-3, FLOOR_MARGIN * mean)

@@ -158,3 +158,60 @@ def test_cache_argument_errors(lib):
     assert lib.pt_workspace_bytes(h, 0, 1, 16, C.byref(ws)) == 1
     lib.pt_kv_cache_free(c)
     lib.pt_model_destroy(h)
+
+
+def test_e4m3_cache_layout_and_scale_offsets(lib):
+    """An E4M3 pool is the one-byte codes in the usual layout followed by one fp32 scale per cached vector; the
+    scale of a vector sits at the vector's own index in that array (the oracle's pool without its last axis)."""
+    T, L, nkv, dh, pages, ps = 2, 4, 2, 128, 5, 16
+    rc, h = make(lib, T=T, L=L, D=2, hidden=256, heads=2, kv_heads=nkv, ffn=512, dtype=pt.PT_BF16)
+    assert rc == 0
+    n = C.c_size_t()
+    assert lib.pt_kv_cache_bytes_ex(h, pages, ps, pt.PT_KV_E4M3, C.byref(n)) == 0
+    vecs = T * L * pages * 2 * nkv * ps
+    assert n.value == vecs * dh + vecs * 4
+    m = C.c_size_t()
+    assert lib.pt_kv_cache_bytes_ex(h, pages, ps, pt.PT_KV_MODEL, C.byref(m)) == 0 and m.value == vecs * dh * 2
+    assert lib.pt_kv_cache_bytes_ex(h, pages, ps, 7, C.byref(m)) == 1
+    assert lib.pt_kv_cache_bytes_ex(h, pages, 8, pt.PT_KV_E4M3, C.byref(m)) == 3          # pages of 8 tokens
+    c = C.c_void_p()
+    assert lib.pt_kv_cache_alloc_ex(h, pages, ps, pt.PT_KV_E4M3, C.c_void_p(0x10000), n.value - 1, C.byref(c)) == 4
+    assert lib.pt_kv_cache_alloc_ex(h, pages, ps, pt.PT_KV_E4M3, C.c_void_p(0x10000), n.value, C.byref(c)) == 0
+    order = np.array([3, 0, 4, 1, 2], np.int32)
+    assert lib.pt_kv_set_free_list(c, order.ctypes.data_as(C.POINTER(C.c_int32)), 5) == 0
+    assert lib.pt_kv_seq_reserve(c, 9, 40) == 0
+    cfg = O.PTConfig(T=T, D=2, L=L, hidden=256, heads=2, kv_heads=nkv, ffn=512)
+    oc = O.PagedKVCache(cfg, pages, ps, order, kv_format="e4m3")
+    oc.reserve(9, 40)
+    off, soff = C.c_int64(), C.c_int64()
+    for t in range(T):
+        for l in (0, 3):
+            for pos in (0, 15, 16, 39):
+                for kv in (0, 1):
+                    for head in range(nkv):
+                        assert lib.pt_kv_slot(c, t, l, 9, pos, kv, head, C.byref(off)) == 0
+                        assert lib.pt_kv_scale_slot(c, t, l, 9, pos, kv, head, C.byref(soff)) == 0
+                        page, slot = oc.locate(9, pos)
+                        want = O.kv_slot_offset(cfg, pages, ps, t, l, page, kv, head, slot)
+                        assert off.value == want
+                        assert soff.value == vecs * dh + (want // dh) * 4
+                        # the same index addresses the oracle's scale array
+                        assert np.ravel_multi_index((t, l, page, kv, head, slot), oc.scale.shape) == want // dh
+    lib.pt_kv_cache_free(c)
+    # a cache in the model dtype holds no scales
+    assert lib.pt_kv_cache_alloc_ex(h, pages, ps, pt.PT_KV_MODEL, C.c_void_p(0x10000), m.value, C.byref(c)) == 0
+    assert lib.pt_kv_seq_reserve(c, 1, 3) == 0
+    assert lib.pt_kv_scale_slot(c, 0, 0, 1, 0, 0, 0, C.byref(soff)) == 10
+    lib.pt_kv_cache_free(c)
+    ws, ws8 = C.c_size_t(), C.c_size_t()
+    assert lib.pt_workspace_bytes_ex(h, 64, 2, ps, pt.PT_KV_MODEL, 0, C.byref(ws)) == 0
+    assert lib.pt_workspace_bytes(h, 64, 2, ps, C.byref(ws8)) == 0 and ws.value == ws8.value
+    assert lib.pt_workspace_bytes_ex(h, 64, 2, ps, pt.PT_KV_E4M3, 0, C.byref(ws8)) == 0 and ws8.value > ws.value
+    lib.pt_model_destroy(h)
+    # head_dim 64 and the plain-kernel path have no E4M3 cache
+    rc, h = make(lib, hidden=256, heads=4, kv_heads=4, dtype=pt.PT_BF16)
+    assert lib.pt_kv_cache_bytes_ex(h, pages, ps, pt.PT_KV_E4M3, C.byref(m)) == 3
+    lib.pt_model_destroy(h)
+    rc, h = make(lib, hidden=256, heads=2, kv_heads=2, dtype=pt.PT_F32)
+    assert lib.pt_kv_cache_bytes_ex(h, pages, ps, pt.PT_KV_E4M3, C.byref(m)) == 3
+    lib.pt_model_destroy(h)

@@ -470,6 +470,7 @@ def test_kv_scale_is_the_smallest_power_of_two_without_saturation():
     v[2] = 0.0; v[2, 5] = -448.0000001
     s = O.kv_scale(v)
     assert s.shape == (200, 1) and s[0, 0] == 1.0 and s[1, 0] == 1.0 and s[2, 0] == 2.0
+    assert O.kv_scale(np.array([[1e-40, 0.0]]))[0, 0] == 2.0 ** -100       # the floor of the scale
     for i in range(3, 200):
         amax = np.abs(v[i]).max()
         cands = [2.0 ** e for e in range(-60, 40) if amax / 2.0 ** e <= 448.0]
