@@ -48,6 +48,8 @@ __global__ void k_tc_prep(const __nv_bfloat16* __restrict__ x, int64_t x_stride,
 __global__ void k_track_sync(const float* __restrict__ hT, size_t tstride, int T, int T_out, float scale,
                              float* __restrict__ h_out, __nv_bfloat16* __restrict__ hb, const float* __restrict__ gain,
                              float* __restrict__ ssq, int M, int H, int tiles) {
+    grid_dep_wait();              // a dependent launch: the GEMM after it may fetch its first weight tiles while this runs
+    grid_dep_launch();
     const int groups = (H + 127) / 128;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (warp >= M * groups) return;
@@ -247,16 +249,17 @@ pt_status tc_forward(Call& k) {
             float* ssq_next = last ? nullptr : w.ssq;
             const unsigned sync_grid = (unsigned)(((size_t)M * ((H + 127) / 128) * 32 + 255) / 256);
             if (split_sync) {       // local tracks -> one stream (the final one unless other ranks still have to join)
-                k_track_sync<<<sync_grid, 256, 0, st>>>(w.hT, MH, T, T, grouped ? 1.0f : sync_scale, grouped ? w.hS : ho,
-                                                        grouped ? nullptr : hb_next, grouped ? nullptr : gain_next,
-                                                        grouped ? nullptr : ssq_next, M, H, tiles);
+                launch_dependent(k_track_sync, dim3(sync_grid), dim3(256), (size_t)0, st, (const float*)w.hT, MH, T, T, grouped ? 1.0f : sync_scale,
+                                 grouped ? w.hS : ho, grouped ? (__nv_bfloat16*)nullptr : hb_next, grouped ? (const float*)nullptr : gain_next,
+                                 grouped ? (float*)nullptr : ssq_next, M, H, tiles);
                 g_launches.fetch_add(1, std::memory_order_relaxed);
             }
             if (grouped) {
                 // w.hS holds this rank's partial sum: one all-reduce per track block, then every local track's
                 // next operand from the total
                 if (m->ar_fn(m->ar_user, w.hS, (int64_t)M * H, (void*)st) != 0) { set_error("the all-reduce hook failed at layer %d", l); return PT_ERR_CUDA; }
-                k_track_sync<<<sync_grid, 256, 0, st>>>(w.hS, 0, 1, T, sync_scale, ho, hb_next, gain_next, ssq_next, M, H, tiles);
+                launch_dependent(k_track_sync, dim3(sync_grid), dim3(256), (size_t)0, st, (const float*)w.hS, (size_t)0, 1, T, sync_scale, ho, hb_next,
+                                 gain_next, ssq_next, M, H, tiles);
                 g_launches.fetch_add(1, std::memory_order_relaxed);
             }
             if (sync) { ssq_tstride = 0; hin = ho; hin_stride = 0; }

@@ -113,12 +113,16 @@ __global__ void k_kv_dequant_ctx(const CtxP p) {
 
 // ---- decode attention straight from the codes -------------------------------------------------------
 // Same work split as the bf16 kernel: a CTA = one (track, sequence, KV head, key range), each of its 4 warps
-// streams its own 16-token groups through a private ring (one TMA box of 16 x 128 code bytes for K, one for V,
-// two 64-byte bulk copies for their scales, all on the slot's mbarrier), the G query heads of the KV head are
-// the rows of an mma.sync m16n8k16 tile.  Codes become f16 (exact) on their way into the MMA's B fragments:
-//   scores  the contraction index of a k-step is mapped to head_dim as kappa {2q, 2q+1, 2q+8, 2q+9} <->
-//           16 ks + 4q + {0, 1, 2, 3} (q = lane % 4), so a thread's two B registers are one 32-bit load of four
-//           consecutive codes of its key's row; q is loaded in the same order.  The K scale multiplies the score.
+// streams its own 16-token groups through a private ring, the G query heads of the KV head are the rows of an
+// mma.sync m16n8k16 tile.  An SM starts a TMA copy only every 80 cycles or so whatever its size (with a K box, a V
+// box and two 64-byte bulk copies of scales per group this kernel ran at 3.7 TB/s, the rate of four copies per
+// 4.2 KB), so a group is ONE copy: a 5-D box that takes the K block and, nkv blocks further, the V block of the
+// page in one go (element stride nkv in the (K|V, head) dimension); the 32 scales come as 32 four-byte cp.async
+// copies, one per lane.  Codes become f16 (exact) on their way into the MMA's B fragments:
+//   scores  the contraction indices kappa {2q, 2q+1, 2q+8, 2q+9} (q = lane % 4) of k-steps 2kk and 2kk+1 are mapped
+//           to head_dim 32 kk + 8q + {0..3} and + {4..7}, so a thread's four B registers of two k-steps are one
+//           64-bit load of eight consecutive codes of its key's row; q is loaded in the same order.  The K scale
+//           multiplies the score.
 //   P V     a thread needs the codes of keys {2q, 2q+1, 2q+8, 2q+9} at one head_dim column: it loads four
 //           consecutive columns 32 m + 4 g + {0..3} (g = lane / 4) of those four rows and takes byte i of each for
 //           the n-tile (m, i), whose column g therefore stands for head_dim 32 m + 4 g + i; the accumulators are
@@ -142,21 +146,27 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
                  : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2) {
-    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-                 ::"r"(dst), "l"((uint64_t)map), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar)) : "memory");
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2, int c3, int c4) {
+    asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+                 ::"r"(dst), "l"((uint64_t)map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint64_t* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
 }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 __device__ __forceinline__ void mma_f16(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
-__device__ __forceinline__ uint32_t codes_to_half2(uint32_t two) {
-    const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)two, __NV_E4M3);
-    return *reinterpret_cast<const uint32_t*>(&h);
+// four codes (a 32-bit word, low byte first) -> two f16 pairs
+__device__ __forceinline__ void codes4_to_half(uint32_t w, uint32_t& lo, uint32_t& hi) {
+    asm("{\n .reg .b16 a, b;\n mov.b32 {a, b}, %2;\n cvt.rn.f16x2.e4m3x2 %0, a;\n cvt.rn.f16x2.e4m3x2 %1, b;\n}" : "=r"(lo), "=r"(hi) : "r"(w));
+}
+__device__ __forceinline__ float ex2f(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 __device__ __forceinline__ uint32_t pack_half2(float a, float b) {
     const __half2 h = __floats2half2_rn(a, b);
@@ -170,7 +180,7 @@ struct Dec8P {
     const float* scales_l; int64_t scales_tstride;
 };
 
-__global__ void __launch_bounds__(kDecThreads)
+__global__ void __launch_bounds__(kDecThreads, 4)
 k_decode_attn_e4m3(const __grid_constant__ CUtensorMap kvmap, const Dec8P pp) {
     const AttnP& p = pp.a;
     extern __shared__ uint8_t smem_raw[];
@@ -198,45 +208,61 @@ k_decode_attn_e4m3(const __grid_constant__ CUtensorMap kvmap, const Dec8P pp) {
     float* wsc = sc_area + warp * kDecStages * 32;
     uint64_t* wbar = bars + warp * kDecStages;
     bool bad_page = false;
-    auto issue = [&](int gidx) {                              // lane 0: codes and scales of local group gidx into its slot
+    // all lanes: lane 0 starts the copy of the codes of local group gidx into its slot, every lane fetches one scale
+    // (lanes 0-15 those of K, 16-31 those of V); one cp.async group per call, so groups complete in issue order
+    auto issue = [&](int gidx) {
         const int key0 = kstart + gidx * 16;
         int page = p.bt[(size_t)b * p.maxp + key0 / p.ps];
         if (page < 0 || page >= p.num_pages) { bad_page = true; page = 0; }
         const int slot = (gidx >> 2) % kDecStages;
-        const uint32_t dst = smem_u32(ring + slot * kSlotBytes);
-        const int row_k = ((page * 2 + 0) * p.nkv + kvh) * p.ps + key0 % p.ps;   // index of the group's first vector in the slab
-        const int row_v = row_k + p.nkv * p.ps;
-        const float* sc = pp.scales_l + (size_t)t * pp.scales_tstride;
-        mbar_expect_tx(&wbar[slot], kSlotBytes + 128);
-        tma_load_3d(dst, &kvmap, &wbar[slot], 0, row_k, t);
-        tma_load_3d(dst + 16 * kDh, &kvmap, &wbar[slot], 0, row_v, t);
-        bulk_load(smem_u32(wsc + slot * 32), sc + row_k, 64, &wbar[slot]);
-        bulk_load(smem_u32(wsc + slot * 32 + 16), sc + row_v, 64, &wbar[slot]);
+        if (lane == 0) {
+            mbar_expect_tx(&wbar[slot], kSlotBytes);
+            tma_load_5d(smem_u32(ring + slot * kSlotBytes), &kvmap, &wbar[slot], 0, key0 % p.ps, kvh, page, t);
+        }
+        const int64_t vec = ((int64_t)(page * 2 + (lane >> 4)) * p.nkv + kvh) * p.ps + key0 % p.ps + (lane & 15);
+        cp_async4(smem_u32(wsc + slot * 32 + lane), pp.scales_l + (size_t)t * pp.scales_tstride + vec);
+        cp_async_commit();
     };
 
     const int g = lane >> 2, q4 = lane & 3;
+    // q fragments: k-steps 2kk and 2kk+1 take head_dim 32 kk + 8 q + {0..3} and + {4..7}
     uint32_t qf[kDh / 16][4];
     {
         const __nv_bfloat16* qrow = p.q + ((size_t)t * p.M + b) * (size_t)(p.nq * kDh) + (size_t)(kvh * G + g) * kDh;
 #pragma unroll
-        for (int ks = 0; ks < kDh / 16; ++ks) {
-            qf[ks][0] = qf[ks][1] = qf[ks][2] = qf[ks][3] = 0u;
+        for (int kk = 0; kk < kDh / 32; ++kk) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) { qf[2 * kk + h][0] = qf[2 * kk + h][1] = qf[2 * kk + h][2] = qf[2 * kk + h][3] = 0u; }
             if (g < G) {
-                const uint2 raw = *reinterpret_cast<const uint2*>(qrow + ks * 16 + q4 * 4);
-                const float2 f0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
-                const float2 f1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
-                qf[ks][0] = pack_half2(f0.x, f0.y);
-                qf[ks][2] = pack_half2(f1.x, f1.y);
+                const uint4 raw = *reinterpret_cast<const uint4*>(qrow + kk * 32 + q4 * 8);
+                const uint32_t wds[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const float2 f0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wds[2 * h]));
+                    const float2 f1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wds[2 * h + 1]));
+                    qf[2 * kk + h][0] = pack_half2(f0.x, f0.y);
+                    qf[2 * kk + h][2] = pack_half2(f1.x, f1.y);
+                }
             }
         }
     }
+    // byte offsets inside a slot, fixed for the thread (the swizzle's XOR is folded in once):
+    //   K: row g (+8 for the second n-tile), the 8 bytes at head_dim 32 kk + 8 q
+    //   V: rows 2q + j (+8), the 4 bytes at head_dim 32 m + 4 g
+    uint32_t koff[kDh / 32], voff[kDh / 32][2];
+#pragma unroll
+    for (int kk = 0; kk < kDh / 32; ++kk) koff[kk] = box_off(g, 32 * kk + 8 * q4);
+#pragma unroll
+    for (int m = 0; m < kDh / 32; ++m)
+#pragma unroll
+        for (int j = 0; j < 2; ++j) voff[m][j] = 16 * kDh + box_off(2 * q4 + j, 32 * m + 4 * g);
     float o[kDh / 8][4];
 #pragma unroll
     for (int i = 0; i < kDh / 8; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
     float m_run = -INFINITY, l_run = 0.f;
 
-    if (lane == 0)
-        for (int s = 0; s < kDecStages; ++s) { int gi = warp + 4 * s; if (gi < npages) issue(gi); }
+#pragma unroll
+    for (int s = 0; s < kDecStages; ++s) { int gi = warp + 4 * s; if (gi < npages) issue(gi); else cp_async_commit(); }
     bool timed_out = false;
     int it = 0;
     for (int gi = warp; gi < npages; gi += 4, ++it) {
@@ -251,43 +277,50 @@ k_decode_attn_e4m3(const __grid_constant__ CUtensorMap kvmap, const Dec8P pp) {
             }
         }
         if (!__all_sync(0xffffffffu, ok)) { timed_out = true; break; }
-        uint8_t* kb = ring + slot * kSlotBytes;
-        uint8_t* vb = kb + 16 * kDh;
+        cp_async_wait<kDecStages - 1>();                      // this group's scales (the groups after it may still be in flight)
+        __syncwarp();
+        const uint32_t sb = smem_u32(ring + slot * kSlotBytes);
         const float* scs = wsc + slot * 32;
-        const int key0 = kstart + gi * 16;
-        const int nvalid = key_end - key0;                    // >= 1
+        const int nvalid = key_end - (kstart + gi * 16);      // >= 1
         if (nvalid < 16) {                                    // tail of the sequence: unused slots may hold anything
+            uint8_t* vb = ring + slot * kSlotBytes + 16 * kDh;
             for (int i = lane; i < (16 - nvalid) * 8; i += 32)
                 *reinterpret_cast<uint4*>(vb + (nvalid + i / 8) * 128 + (i % 8) * 16) = make_uint4(0, 0, 0, 0);
             __syncwarp();
         }
         // this thread's four keys: 2q, 2q+1, 2q+8, 2q+9 (score columns and P V contraction rows alike)
-        const float2 sk01 = *reinterpret_cast<const float2*>(scs + 2 * q4), sk89 = *reinterpret_cast<const float2*>(scs + 8 + 2 * q4);
-        const float2 sv01 = *reinterpret_cast<const float2*>(scs + 16 + 2 * q4), sv89 = *reinterpret_cast<const float2*>(scs + 24 + 2 * q4);
+        float2 sk01 = *reinterpret_cast<const float2*>(scs + 2 * q4), sk89 = *reinterpret_cast<const float2*>(scs + 8 + 2 * q4);
+        float2 sv01 = *reinterpret_cast<const float2*>(scs + 16 + 2 * q4), sv89 = *reinterpret_cast<const float2*>(scs + 24 + 2 * q4);
         float s[2][4] = {};
 #pragma unroll
-        for (int ks = 0; ks < kDh / 16; ++ks) {
+        for (int kk = 0; kk < kDh / 32; ++kk) {
 #pragma unroll
             for (int nt = 0; nt < 2; ++nt) {
-                const uint32_t w = *reinterpret_cast<const uint32_t*>(kb + box_off(nt * 8 + g, ks * 16 + q4 * 4));
-                mma_f16(s[nt], qf[ks], codes_to_half2(w & 0xffffu), codes_to_half2(w >> 16));
+                uint32_t w0, w1, b0, b1, b2, b3;
+                asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(w0), "=r"(w1) : "r"(sb + koff[kk] + nt * 1024));
+                codes4_to_half(w0, b0, b1);
+                codes4_to_half(w1, b2, b3);
+                mma_f16(s[nt], qf[2 * kk], b0, b1);
+                mma_f16(s[nt], qf[2 * kk + 1], b2, b3);
             }
         }
-        const bool in0 = 2 * q4 < nvalid, in1 = 2 * q4 + 1 < nvalid, in8 = 8 + 2 * q4 < nvalid, in9 = 9 + 2 * q4 < nvalid;
-        s[0][0] = in0 ? s[0][0] * sk01.x * p.scale_log2 : -INFINITY;
-        s[0][1] = in1 ? s[0][1] * sk01.y * p.scale_log2 : -INFINITY;
-        s[1][0] = in8 ? s[1][0] * sk89.x * p.scale_log2 : -INFINITY;
-        s[1][1] = in9 ? s[1][1] * sk89.y * p.scale_log2 : -INFINITY;
+        s[0][0] *= sk01.x * p.scale_log2; s[0][1] *= sk01.y * p.scale_log2;
+        s[1][0] *= sk89.x * p.scale_log2; s[1][1] *= sk89.y * p.scale_log2;
+        if (nvalid < 16) {
+            if (2 * q4 >= nvalid) { s[0][0] = -INFINITY; sv01.x = 0.f; }
+            if (2 * q4 + 1 >= nvalid) { s[0][1] = -INFINITY; sv01.y = 0.f; }
+            if (2 * q4 + 8 >= nvalid) { s[1][0] = -INFINITY; sv89.x = 0.f; }
+            if (2 * q4 + 9 >= nvalid) { s[1][1] = -INFINITY; sv89.y = 0.f; }
+        }
         float mx = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
         const float mn = fmaxf(m_run, mx);
-        const float corr = exp2f(m_run - mn);
+        const float corr = ex2f(m_run - mn);
         m_run = mn;
-        float sum = 0.f;
-#pragma unroll
-        for (int i = 0; i < 2; ++i) { s[i][0] = exp2f(s[i][0] - mn); s[i][1] = exp2f(s[i][1] - mn); sum += s[i][0] + s[i][1]; }
-        l_run = l_run * corr + sum;
+        s[0][0] = ex2f(s[0][0] - mn); s[0][1] = ex2f(s[0][1] - mn);
+        s[1][0] = ex2f(s[1][0] - mn); s[1][1] = ex2f(s[1][1] - mn);
+        l_run = l_run * corr + ((s[0][0] + s[0][1]) + (s[1][0] + s[1][1]));
         if (__any_sync(0xffffffffu, corr != 1.f)) {
 #pragma unroll
             for (int i = 0; i < kDh / 8; ++i) { o[i][0] *= corr; o[i][1] *= corr; }
@@ -295,31 +328,35 @@ k_decode_attn_e4m3(const __grid_constant__ CUtensorMap kvmap, const Dec8P pp) {
         uint32_t pf[4];
         pf[0] = pack_half2(s[0][0], s[0][1]); pf[1] = 0u;
         pf[2] = pack_half2(s[1][0], s[1][1]); pf[3] = 0u;
-        const uint32_t hs01 = pack_half2(in0 ? sv01.x : 0.f, in1 ? sv01.y : 0.f);
-        const uint32_t hs89 = pack_half2(in8 ? sv89.x : 0.f, in9 ? sv89.y : 0.f);
+        const uint32_t hs01 = pack_half2(sv01.x, sv01.y), hs89 = pack_half2(sv89.x, sv89.y);
 #pragma unroll
         for (int m = 0; m < kDh / 32; ++m) {
-            const int c = 32 * m + 4 * g;
-            const uint32_t w0 = *reinterpret_cast<const uint32_t*>(vb + box_off(2 * q4, c));
-            const uint32_t w1 = *reinterpret_cast<const uint32_t*>(vb + box_off(2 * q4 + 1, c));
-            const uint32_t w2 = *reinterpret_cast<const uint32_t*>(vb + box_off(2 * q4 + 8, c));
-            const uint32_t w3 = *reinterpret_cast<const uint32_t*>(vb + box_off(2 * q4 + 9, c));
+            uint32_t w0, w1, w2, w3;
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w0) : "r"(sb + voff[m][0]));
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w1) : "r"(sb + voff[m][1]));
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w2) : "r"(sb + voff[m][0] + 1024));
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w3) : "r"(sb + voff[m][1] + 1024));
+            // bytes (i, i + 1) of two rows side by side: [r0.b_i, r1.b_i, r0.b_i+1, r1.b_i+1]
+            const uint32_t a01 = __byte_perm(w0, w1, 0x5140), a23 = __byte_perm(w0, w1, 0x7362);
+            const uint32_t c01 = __byte_perm(w2, w3, 0x5140), c23 = __byte_perm(w2, w3, 0x7362);
+            uint32_t b0[4], b1[4];
+            codes4_to_half(a01, b0[0], b0[1]); codes4_to_half(a23, b0[2], b0[3]);
+            codes4_to_half(c01, b1[0], b1[1]); codes4_to_half(c23, b1[2], b1[3]);
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const uint32_t sel = (uint32_t)i | ((uint32_t)(4 + i) << 4);
-                uint32_t b0 = codes_to_half2(__byte_perm(w0, w1, sel) & 0xffffu);
-                uint32_t b1 = codes_to_half2(__byte_perm(w2, w3, sel) & 0xffffu);
-                asm("mul.rn.f16x2 %0, %0, %1;" : "+r"(b0) : "r"(hs01));
-                asm("mul.rn.f16x2 %0, %0, %1;" : "+r"(b1) : "r"(hs89));
-                mma_f16(o[m * 4 + i], pf, b0, b1);
+                asm("mul.rn.f16x2 %0, %0, %1;" : "+r"(b0[i]) : "r"(hs01));
+                asm("mul.rn.f16x2 %0, %0, %1;" : "+r"(b1[i]) : "r"(hs89));
+                mma_f16(o[m * 4 + i], pf, b0[i], b1[i]);
             }
         }
         __syncwarp();                                         // every lane is done reading the slot
-        if (lane == 0) {
-            int gn = gi + 4 * kDecStages;
+        {
+            const int gn = gi + 4 * kDecStages;
             if (gn < npages) { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); issue(gn); }
+            else cp_async_commit();                           // keeps "all but the last kDecStages - 1 groups" meaning this group's successor
         }
     }
+    cp_async_wait<0>();
     if (timed_out) {
         // give the copies this warp still has in flight a bounded chance to land, then give up
         WaitClock clock;
@@ -377,8 +414,9 @@ typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void
                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// (code byte, vector of a slab, track) with boxes of 16 vectors x 128 bytes in the 128-byte swizzle
-pt_status make_codes_map(CUtensorMap* out, const void* base, int64_t vecs, int64_t tracks, int64_t track_stride_bytes) {
+// (code byte, slot, (K|V, head), page, track): a box is the 16 x 128 code bytes of one 16-token group of a K block and,
+// through the element stride nkv of the third dimension, of the V block of the same head
+pt_status make_codes_map(CUtensorMap* out, const void* base, int ps, int nkv, int64_t pages, int64_t tracks, int64_t track_stride_bytes) {
     static EncodeFn enc = nullptr;
     if (!enc) {
         void* f = nullptr;
@@ -387,11 +425,12 @@ pt_status make_codes_map(CUtensorMap* out, const void* base, int64_t vecs, int64
             enc = (EncodeFn)f;
     }
     if (!enc) { set_error("cuTensorMapEncodeTiled is not available from this driver"); return PT_ERR_CUDA; }
-    cuuint64_t dims[3] = {(cuuint64_t)kDh, (cuuint64_t)vecs, (cuuint64_t)tracks};
-    cuuint64_t strides[2] = {(cuuint64_t)kDh, (cuuint64_t)track_stride_bytes};
-    cuuint32_t box[3] = {(cuuint32_t)kDh, 16, 1};
-    cuuint32_t es[3] = {1, 1, 1};
-    CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, es,
+    if (nkv > 8) { set_error("an E4M3 cache supports up to 8 KV heads per track"); return PT_ERR_UNSUPPORTED; }
+    cuuint64_t dims[5] = {(cuuint64_t)kDh, (cuuint64_t)ps, (cuuint64_t)(2 * nkv), (cuuint64_t)pages, (cuuint64_t)tracks};
+    cuuint64_t strides[4] = {(cuuint64_t)kDh, (cuuint64_t)ps * kDh, (cuuint64_t)2 * nkv * ps * kDh, (cuuint64_t)track_stride_bytes};
+    cuuint32_t box[5] = {(cuuint32_t)kDh, 16, (cuuint32_t)(nkv + 1), 1, 1};
+    cuuint32_t es[5] = {1, 1, (cuuint32_t)nkv, 1, 1};
+    CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 5, const_cast<void*>(base), dims, strides, box, es,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled (E4M3 cache) failed with code %d", (int)r); return PT_ERR_CUDA; }
@@ -464,7 +503,7 @@ pt_status launch_decode_attn_e4m3(Call& k, const __nv_bfloat16* q, int layer, __
     p.items = k.items; p.nsplit = k.nsplit; p.part = k.w.part; p.max_splits = kMaxSplits;
     pp.scales_l = c->scales + (size_t)layer * c->slab_vecs(); pp.scales_tstride = (int64_t)g.L * c->slab_vecs();
     CUtensorMap kvmap;
-    pt_status s = make_codes_map(&kvmap, c->pool + (size_t)layer * c->slab_elems, c->slab_vecs(), g.T, (int64_t)g.L * c->slab_elems);
+    pt_status s = make_codes_map(&kvmap, c->pool + (size_t)layer * c->slab_elems, c->ps, g.kv_heads, c->num_pages, g.T, (int64_t)g.L * c->slab_elems);
     if (s != PT_OK) return s;
     const int smem = 1024 + 4 * kDecStages * kSlotBytes + 4 * kDecStages * 32 * 4 + 4 * kDecStages * 8;
     static bool done_[kMaxDevices] = {};

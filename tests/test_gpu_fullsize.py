@@ -133,29 +133,45 @@ def test_prefill_full_size_sampled_prefixes_match_oracle(mid_model):
     torch.cuda.empty_cache()
 
 
+def _seq_kv(cache, wl, t, pages):
+    """What attention reads for track t on the given pages (a CUDA index tensor), all layers:
+    float32 numpy [L, pages, K|V, head, slot, dh] - the cached values, or code * scale of an E4M3 cache -
+    and the scales [L, pages, K|V, head, slot] (None for a cache in the model dtype)."""
+    import torch
+    shape = (wl.T, wl.L, cache.num_pages, 2, wl.kv_heads, wl.page_size)
+    if cache.kv_dtype:
+        codes = cache.codes.view(shape + (wl.head_dim,))[t][:, pages].view(torch.float8_e4m3fn).to(torch.float32)
+        sc = cache.scales.view(shape)[t][:, pages]
+        return (codes * sc.unsqueeze(-1)).cpu().numpy(), sc.cpu().numpy()
+    return cache.pool.view(shape + (wl.head_dim,))[t][:, pages].float().cpu().numpy(), None
+
+
 def _inject(cache, wl, seq, n, ocache, oseq):
     """Copy the first n cached tokens of device sequence `seq` into sequence `oseq` of the oracle's cache."""
     import torch
     ocache.reserve(oseq, n)
     ocache.length[oseq] = n
     pages = torch.tensor(cache.block_table(seq)[: -(-n // wl.page_size)], device=cache.pool.device)
-    pool = cache.pool.view(wl.T, wl.L, cache.num_pages, 2, wl.kv_heads, wl.page_size, wl.head_dim)
     opages = np.asarray(ocache.block_table[oseq])
     for t in range(wl.T):
-        blk = pool[t][:, pages].float().cpu().numpy()                 # [L, pages, K|V, head, slot, dh]
+        blk, sc = _seq_kv(cache, wl, t, pages)                         # [L, pages, K|V, head, slot, dh]
         if n % wl.page_size:
             blk[:, -1, :, :, n % wl.page_size:, :] = 0.0               # slots past the sequence's end were never written
         ocache.pool[t][:, opages] = blk
+        if sc is not None:
+            if n % wl.page_size:
+                sc[:, -1, :, :, n % wl.page_size:] = 1.0
+            ocache.scale[t][:, opages] = sc
 
 
-def _fill_and_decode(model, wl, lens, own, x_own, rows, xd_rows, seed, sub_tokens=16384):
+def _fill_and_decode(model, wl, lens, own, x_own, rows, xd_rows, seed, sub_tokens=16384, kv8=False):
     """Fill the cache of a full-size batch by prefills of N(0, 1) prompts (sequence `own` gets the NumPy-drawn
     prompt x_own [T, 1, len, H]), then run ONE decode step over the whole batch in which the rows `rows` get the
     NumPy-drawn inputs xd_rows [T, len(rows), H].  Returns (cache, output [B, H], tap [L, 2, T, B, H])."""
     import torch
     B, ps, T, H = len(lens), wl.page_size, wl.T, wl.hidden
     pages = int(sum(-(-(int(n) + 1) // ps) for n in lens))
-    cache = model.new_cache(pages, ps)
+    cache = model.new_cache(pages, ps, kv_dtype="e4m3" if kv8 else "model")
     g = torch.Generator(device=model.device).manual_seed(seed)
     order = np.argsort(-np.asarray(lens), kind="stable")
     i = 0
@@ -184,16 +200,19 @@ def _fill_and_decode(model, wl, lens, own, x_own, rows, xd_rows, seed, sub_token
     return cache, got, tap
 
 
-def _decode_against_oracle(model, wl, ws, lens, own, injected, seed, tag, sub_tokens=16384):
+def _decode_against_oracle(model, wl, ws, lens, own, injected, seed, tag, sub_tokens=16384, kv8=False):
+    """kv8: the cache holds E4M3 codes on both sides.  The device quantises the K and V its bf16 GEMM made, the
+    oracle its exact ones, so cached values may sit one code step apart: the mean bound comes from the floor
+    measured with that format, the cached values are held to one code step, a layer delta to 6e-2."""
     import torch
     T, L, ps = wl.T, wl.L, wl.page_size
-    mean_tol = Hp.mean_bound(wl)
+    mean_tol = Hp.mean_bound(wl, kv8=kv8)
     rows = [own, injected]
     x_own = I.prefill_inputs(wl, batch=1, seq=int(lens[own]), salt=200)
     xd_rows = I.decode_inputs(wl, batch=2, step=0)
-    cache, got, tap = _fill_and_decode(model, wl, lens, own, x_own, rows, xd_rows, seed, sub_tokens)
+    cache, got, tap = _fill_and_decode(model, wl, lens, own, x_own, rows, xd_rows, seed, sub_tokens, kv8)
     cfg = Hp.oracle_cfg(wl)
-    ocache = O.PagedKVCache(cfg, sum(-(-(int(lens[r]) + 1) // ps) for r in rows), ps)
+    ocache = O.PagedKVCache(cfg, sum(-(-(int(lens[r]) + 1) // ps) for r in rows), ps, kv_format="e4m3" if kv8 else "model")
     O.pt_prefill(cfg, Hp.Prefetch(ws, T, L), x_own, ocache, [0])            # the oracle's own cache for `own`
     # the K/V the device cached for `own` against the oracle's: every track and layer, all whole pages (the tail
     # page has unwritten slots), accumulated track by track
@@ -201,18 +220,22 @@ def _decode_against_oracle(model, wl, ws, lens, own, injected, seed, tag, sub_to
     full = n_own // ps
     pages = torch.tensor(cache.block_table(own)[:full], device=cache.pool.device)
     opages = np.asarray(ocache.block_table[0][:full])
-    pool = cache.pool.view(T, L, cache.num_pages, 2, wl.kv_heads, ps, wl.head_dim)
     dmax = dsum = rmax = rsum = 0.0
     for t in range(T):
         want = ocache.pool[t][:, opages]
-        d = np.abs(pool[t][:, pages].float().cpu().numpy() - want)
+        have, sc = _seq_kv(cache, wl, t, pages)
+        d = np.abs(have - want)
+        if kv8:      # never further apart than the largest code step (32 units of the larger of the two scales)
+            assert np.all(d <= 32.0 * np.maximum(sc, ocache.scale[t][:, opages])[..., None] * (1 + 1e-6))
         dmax, dsum = max(dmax, float(d.max())), dsum + float(d.sum())
         rmax, rsum = max(rmax, float(np.abs(want).max())), rsum + float(np.abs(want).sum())
-        del d, want
+        del d, want, have
     mx, mean = dmax / rmax, dsum / rsum
-    Hp.record(f"{tag}: cached K/V of the own-cache sequence ({full * ps} tokens, all tracks and layers)", mx, mean, 2e-2, 2 * mean_tol)
-    # a cached value carries its own bf16 rounding on top of its projection's operand rounding: the mean bound is doubled
-    assert mx <= 2e-2 and mean <= 2 * mean_tol, f"cached K/V: max-rel {mx:.3e}, mean-rel {mean:.3e}"
+    # bf16 cache: a cached value carries its own bf16 rounding on top of its projection's operand rounding, so the
+    # mean bound is doubled; E4M3 cache: one code step of a value near the top of its binade is 32 / 224 of it
+    kv_mx, kv_mean = (32.0 / 224.0, 1e-2) if kv8 else (2e-2, 2 * mean_tol)
+    Hp.record(f"{tag}: cached K/V of the own-cache sequence ({full * ps} tokens, all tracks and layers)", mx, mean, kv_mx, kv_mean)
+    assert mx <= kv_mx and mean <= kv_mean, f"cached K/V: max-rel {mx:.3e}, mean-rel {mean:.3e}"
     _inject(cache, wl, injected, int(lens[injected]), ocache, 1)
     taps = {}
     ref = O.pt_decode_step(cfg, Hp.Prefetch(ws, T, L), xd_rows, ocache, [0, 1], taps)
@@ -221,24 +244,25 @@ def _decode_against_oracle(model, wl, ws, lens, own, injected, seed, tag, sub_to
         Hp.assert_close(out[i], ref[i], wl.dtype, f"{tag}: decode output of sequence {r}", mean_tol=mean_tol,
                         log=f"{tag}: decode output, sequence {r} (KV {int(lens[r])}, {kind})")
     tp = tap[:, :, :, rows].cpu().numpy()
-    _check_taps(wl, tp, taps, 2, 1, mean_tol)                              # every layer's stream and both deltas
+    _check_taps(wl, tp, taps, 2, 1, mean_tol, delta_tol=6e-2 if kv8 else None)     # every layer's stream and both deltas
     for l in _tap_layers(wl) + [L - 1]:
         mx, mean = Hp.rel_errs(tp[l, 1], taps["h"][l].reshape(T, 2, wl.hidden))
         Hp.record(f"{tag}: layer {l} stream after the layer (both sequences)", mx, mean, 2e-2, mean_tol)
     cache.close()
-    del cache, tap, pool, pages
+    del cache, tap, pages
     torch.cuda.empty_cache()
 
 
-def test_decode_against_oracle_machinery_on_a_small_model():
+@pytest.mark.parametrize("kv8", [False, True])
+def test_decode_against_oracle_machinery_on_a_small_model(kv8):
     """The same own-cache / device-cache comparison on a model the oracle runs in a second."""
-    wl = I.Workload("small-decode", T=3, L=6, D=3, hidden=256, heads=4, kv_heads=2, ffn=352, dtype="bf16",
-                    mode="decode", batch=5, seq=0, ragged=(40, 200))
+    wl = I.Workload("small-decode", T=3, L=6, D=3, hidden=256, heads=2 if kv8 else 4, kv_heads=1 if kv8 else 2, ffn=352,
+                    dtype="bf16", mode="decode", batch=5, seq=0, ragged=(40, 200))
     ws = I.WeightSource(wl)
     model = Hp.make_model(wl, ws, max_pos=256)
     lens = I.kv_lengths(wl)
     _decode_against_oracle(model, wl, ws, lens, own=int(np.argmin(lens)), injected=int(np.argmax(lens)), seed=5,
-                           tag="small ragged decode", sub_tokens=256)
+                           tag="small ragged decode" + (" (e4m3 cache)" if kv8 else ""), sub_tokens=256, kv8=kv8)
     model.close()
 
 
@@ -250,29 +274,57 @@ def test_decode_full_size_matches_oracle_cfg2(mid_model):
     _decode_against_oracle(model, wl, ws, I.kv_lengths(wl), own=37, injected=3, seed=7, tag="cfg2 decode batch 64 at KV 2048")
 
 
-def test_decode_full_size_matches_oracle_cfg4_ragged_gqa():
+@pytest.fixture(scope="module")
+def wide_model():
+    """The T=4, L=48 GQA model of the ragged decode workload with its seeded weights."""
+    import torch
+    torch.cuda.empty_cache()
+    wl = I.WORKLOADS["cfg4"]
+    ws = I.WeightSource(wl)
+    m = Hp.make_model(wl, Hp.Prefetch(ws, wl.T, wl.L), max_pos=int(I.kv_lengths(wl).max()) + 16)
+    yield wl, ws, m
+    m.close()
+
+
+def _largest_batch(wl, lens_all, bytes_per_element, reserve_gib):
+    """The largest prefix (a multiple of 16) of the workload's sequences whose pages fit the free device memory."""
+    import torch
+    page_bytes = wl.T * wl.L * 2 * wl.kv_heads * wl.page_size * (wl.head_dim * bytes_per_element + (4 if bytes_per_element == 1 else 0))
+    pages_of = (lens_all.astype(np.int64) + 1 + wl.page_size - 1) // wl.page_size
+    budget = torch.cuda.mem_get_info()[0] - (reserve_gib << 30)
+    B = wl.batch
+    while B > 16 and int(pages_of[:B].sum()) * page_bytes > budget:
+        B -= 16
+    return B if int(pages_of[:B].sum()) * page_bytes <= budget else 0
+
+
+def test_decode_full_size_matches_oracle_cfg4_ragged_gqa(wide_model):
     """The wide GQA model at its full width and depth with the seeded weights and the seeded ragged lengths; the
     batch is the largest prefix of the 256 sequences whose pages fit the device, as in the benchmark.  The
     oracle's own-cache sequence is the shortest of the batch, the device-cache one the longest."""
     import torch
-    wl = I.WORKLOADS["cfg4"]
-    lens_all = I.kv_lengths(wl)
+    wl, ws, model = wide_model
     torch.cuda.empty_cache()
-    page_bytes = wl.T * wl.L * 2 * wl.kv_heads * wl.page_size * wl.head_dim * 2
-    pages_of = (lens_all.astype(np.int64) + 1 + wl.page_size - 1) // wl.page_size
-    weight_bytes = wl.T * wl.L * wl.params_per_track_layer() * 2
-    budget = torch.cuda.mem_get_info()[0] - weight_bytes - (14 << 30)
-    B = wl.batch
-    while B > 16 and int(pages_of[:B].sum()) * page_bytes > budget:
-        B -= 16
-    if int(pages_of[:B].sum()) * page_bytes > budget:
+    lens_all = I.kv_lengths(wl)
+    B = _largest_batch(wl, lens_all, 2, 14)
+    if not B:
         pytest.skip("not enough free device memory for 16 sequences")
-    ws = I.WeightSource(wl)
-    model = Hp.make_model(wl, Hp.Prefetch(ws, wl.T, wl.L), max_pos=int(lens_all.max()) + 16)
     lens = lens_all[:B]
     _decode_against_oracle(model, wl, ws, lens, own=int(np.argmin(lens)), injected=int(np.argmax(lens)), seed=9,
                            tag=f"cfg4 ragged GQA decode batch {B}", sub_tokens=8192)
-    model.close()
+
+
+def test_decode_full_size_matches_oracle_cfg4_whole_batch_e4m3_cache(wide_model):
+    """The same workload with the cache in the E4M3 format: all 256 sequences fit."""
+    import torch
+    wl, ws, model = wide_model
+    torch.cuda.empty_cache()
+    lens_all = I.kv_lengths(wl)
+    B = _largest_batch(wl, lens_all, 1, 14)
+    if B < wl.batch:
+        pytest.skip(f"only {B} of {wl.batch} sequences fit the free device memory")
+    _decode_against_oracle(model, wl, ws, lens_all, own=int(np.argmin(lens_all)), injected=int(np.argmax(lens_all)), seed=9,
+                           tag=f"cfg4 ragged GQA decode batch {B}, e4m3 cache", sub_tokens=8192, kv8=True)
 
 
 def test_wide_gqa_architecture_at_reduced_depth_matches_oracle():
