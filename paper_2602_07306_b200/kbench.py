@@ -5,6 +5,7 @@
     python -m paper_2602_07306_b200.kbench layer --T 8 --B 2 --S 4096 --H 1024 --nq 8 --nkv 8 --F 2816
     python -m paper_2602_07306_b200.kbench generate --B 1 --S 1024 --new 64 [--depth 2|4|8]
     python -m paper_2602_07306_b200.kbench gemm --T 8 --M 32768 --N 3072 --K 1024 [--bn 256] [--fold]
+    python -m paper_2602_07306_b200.kbench step --T 4 --B 64 --len 2048 --H 2048 --nq 16 --nkv 4 --F 5632 [--kv8 1]
 
 Prints one JSON line: average device time per launch (CUDA events on the launching stream,
 after warm-up) and the achieved GB/s (decode: K/V bytes read) or TFLOP/s (gemm).  Small cases of
@@ -122,6 +123,46 @@ def layer(a):
     print(json.dumps({"kernel": "layer", "per_launch": res, "args": vars(a)}))
 
 
+def step(a):
+    """Decode steps of a small model (L = D = --layers) of the given width over a cache filled by real prefills, with
+    the cache in the model dtype or (--kv8 1) in the E4M3 format: per-category device time per launch, and the
+    achieved rate of the attention kernel over the bytes of the cached vectors it reads."""
+    dev = torch.device("cuda:0")
+    m = pt.Model(T=a.T, D=a.layers, L=a.layers, hidden=a.H, heads=a.nq, kv_heads=a.nkv, ffn=a.F, dtype="bf16",
+                 max_pos=a.len + 16, device=dev)
+    m.init_random(0)
+    dh = a.H // a.nq
+    cache = m.new_cache(a.B * (-(-(a.len + 1) // a.ps)), a.ps, kv_dtype="e4m3" if a.kv8 else "model")
+    g = torch.Generator(device=dev).manual_seed(0)
+    sub = max(1, 8192 // a.len)
+    for i in range(0, a.B, sub):
+        ids = list(range(i, min(a.B, i + sub)))
+        x = torch.randn((a.T, len(ids), a.len, a.H), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        m.prefill(cache, x, ids)
+    xd = torch.randn((a.T, a.B, a.H), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    out = torch.empty((a.B, a.H), dtype=torch.float32, device=dev)
+    ids = list(range(a.B))
+
+    def one():
+        m.decode_step(cache, xd, ids, out)
+        for s_ in ids:
+            cache.truncate(s_, a.len)
+    for _ in range(a.warmup):
+        one()
+    torch.cuda.synchronize()
+    m.profile(True)
+    for _ in range(a.iters):
+        one()
+    torch.cuda.synchronize()
+    prof = m.profile_read()
+    assert m.device_status() == (0, 0)
+    vec = dh + 4 if a.kv8 else 2 * dh
+    byts = a.T * 2 * a.nkv * vec * a.B * (a.len + 1)
+    res = {k: v[0] / max(v[1], 1) for k, v in prof.items() if v[1]}
+    print(json.dumps({"kernel": "decode_step", "ms_per_launch": res, "attention_GBps": byts / res["attention"] / 1e6,
+                      "attention_bytes": byts, "args": vars(a)}))
+
+
 def generate(a):
     """Greedy generation at the head layout of the paper's 30B model (inputs.WORKLOADS["pt30b_prefill"]): time
     to the first token (embed + prefill + LM head + choice) and time per further token, batch a.B."""
@@ -206,12 +247,15 @@ def main():
     gn = sub.add_parser("generate")
     for k, v in dict(B=1, S=1024, new=64, vocab=32000, depth=0, iters=3, warmup=1).items():
         gn.add_argument("--" + k, type=int, default=v)
+    sp = sub.add_parser("step")
+    for k, v in dict(T=4, B=64, len=2048, H=2048, nq=16, nkv=4, F=5632, ps=16, layers=2, kv8=0, iters=10, warmup=3).items():
+        sp.add_argument("--" + k, type=int, default=v)
     gm = sub.add_parser("gemm")
     for k, v in dict(T=8, M=4096, N=3072, K=1024, bn=0, iters=20, warmup=3).items():
         gm.add_argument("--" + k, type=int, default=v)
     gm.add_argument("--fold", action="store_true")
     a = ap.parse_args()
-    {"decode": decode, "gemm": gemm, "prefill": prefill, "layer": layer, "generate": generate}[a.cmd](a)
+    {"decode": decode, "gemm": gemm, "prefill": prefill, "layer": layer, "generate": generate, "step": step}[a.cmd](a)
 
 
 if __name__ == "__main__":
