@@ -255,7 +255,9 @@ pt_status pt_generate(pt_model* m, pt_kv_cache* c, const int32_t* dev_prompt, in
  * fp32 values at `dev_buf` (device) by their sum over all ranks, enqueued on `stream` (e.g. an NCCL
  * all-reduce), and return 0; any other return value fails the forward call with PT_ERR_CUDA.  With
  * sync_op = MEAN the mean is taken over world_tracks.  Every rank passes the same batch; x holds the
- * rank's own tracks.  fn == NULL or world_tracks == 0 returns the model to the single-GPU schedule.
+ * rank's own tracks.  While `fn`'s work runs on `stream`, the library pulls the weights of the next layer's
+ * first projection into L2 on a stream of its own (created on first use, joined into `stream` before the
+ * forward call's work on it ends), so that the next track block does not start from HBM latency.  fn == NULL or world_tracks == 0 returns the model to the single-GPU schedule.
  * bf16 models on the tensor-core path only. */
 typedef int32_t (*pt_allreduce_fn)(void* user, void* dev_buf, int64_t count, void* stream);
 pt_status pt_model_set_track_group(pt_model* m, int32_t world_tracks, pt_allreduce_fn fn, void* user);

@@ -157,6 +157,8 @@ pt_status pt_model_create(const pt_config* cfg, pt_model** out) {
 void pt_model_destroy(pt_model* m) {
     if (!m) return;
     for (auto& e : m->prof_ev) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
+    if (m->side_event) cudaEventDestroy(m->side_event);
+    if (m->side_stream) cudaStreamDestroy(m->side_stream);
     delete m;
 }
 

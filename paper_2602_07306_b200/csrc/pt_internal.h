@@ -67,6 +67,10 @@ struct pt_model {
     int world_tracks = 0;                  // > 0: this model holds cfg.T of world_tracks tracks (pt_model_set_track_group)
     pt_allreduce_fn ar_fn = nullptr;
     void* ar_user = nullptr;
+    // track groups: a side stream and an event (created on first use, destroyed with the model) on which the next
+    // layer's first weights are pulled into L2 while the all-reduce of a track-sync runs on the call's stream
+    cudaStream_t side_stream = nullptr;
+    cudaEvent_t side_event = nullptr;
     int tap_layer = -2;
     float* tap_buf = nullptr;
     std::vector<char> meta_host;          // staging for the per-call metadata upload

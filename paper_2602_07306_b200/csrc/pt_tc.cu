@@ -82,6 +82,13 @@ __global__ void k_track_sync(const float* __restrict__ hT, size_t tstride, int T
     if (ssq && (lane & 15) == 0 && tile < tiles) ssq[(size_t)row * tiles + tile] = s;
 }
 
+// Asks L2 for `bytes` bytes from `base` (128-byte lines, a grid-stride loop of prefetch hints: nothing is read into the SM).
+__global__ void k_l2_prefetch(const char* __restrict__ base, size_t bytes) {
+    const size_t lines = (bytes + 127) / 128;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < lines; i += (size_t)gridDim.x * blockDim.x)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(base + i * 128));
+}
+
 inline int kps_index(int kps) { return kps == 4 ? 2 : (kps == 2 ? 1 : 0); }
 
 }  // namespace
@@ -256,7 +263,22 @@ pt_status tc_forward(Call& k) {
             }
             if (grouped) {
                 // w.hS holds this rank's partial sum: one all-reduce per track block, then every local track's
-                // next operand from the total
+                // next operand from the total.  While the all-reduce runs on the call's stream, a side stream pulls the
+                // weights of the next layer's QKV projection (at most 48 MB of them) into L2, so that the first GEMM of
+                // the next track block does not start from HBM latency: the side stream only waits for the sync GEMM
+                // (an event), nothing waits for it.
+                if (!last) {
+                    if (!m->side_stream && (cudaStreamCreateWithFlags(&m->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
+                                            cudaEventCreateWithFlags(&m->side_event, cudaEventDisableTiming) != cudaSuccess)) {
+                        set_error("side stream for the weight prefetch: %s", cudaGetErrorString(cudaGetLastError()));
+                        return PT_ERR_CUDA;
+                    }
+                    const size_t wbytes = std::min<size_t>(m->wqkv_layer() * 2, (size_t)48 << 20);
+                    cudaEventRecord(m->side_event, st);
+                    cudaStreamWaitEvent(m->side_stream, m->side_event, 0);
+                    k_l2_prefetch<<<148, 256, 0, m->side_stream>>>(m->wbuf + m->off_wqkv + (size_t)(l + 1) * m->wqkv_layer() * 2, wbytes);
+                    g_launches.fetch_add(1, std::memory_order_relaxed);
+                }
                 if (m->ar_fn(m->ar_user, w.hS, (int64_t)M * H, (void*)st) != 0) { set_error("the all-reduce hook failed at layer %d", l); return PT_ERR_CUDA; }
                 launch_dependent(k_track_sync, dim3(sync_grid), dim3(256), (size_t)0, st, (const float*)w.hS, (size_t)0, 1, T, sync_scale, ho, hb_next,
                                  gain_next, ssq_next, M, H, tiles);
@@ -266,6 +288,10 @@ pt_status tc_forward(Call& k) {
             else { ssq_tstride = (size_t)M * tiles; hin = w.hT; hin_stride = MH; }
         }
         tap_copy(k, l, 1, hin, hin_stride);
+    }
+    if (m->ar_fn && m->side_stream) {      // the call's stream ends after the side stream's last prefetch: a wait on it covers both
+        cudaEventRecord(m->side_event, m->side_stream);
+        cudaStreamWaitEvent(st, m->side_event, 0);
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_error("kernel launch failed: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }

@@ -34,20 +34,29 @@ def _full_and_inputs(sync_op, L=4, D=2):
 def test_one_rank_with_identity_hook_equals_the_plain_schedule_and_syncs_L_over_D_times(sync_op):
     import torch
     wl, ws, x, xd = _full_and_inputs(sync_op)
+    from paper_2602_07306_b200 import pt
     outs = []
     calls = []
+    launches = []
     for hooked in (False, True):
         m = Hp.make_model(wl, ws, sync_op=sync_op, max_pos=512)
         if hooked:
             m.set_track_group(wl.T, lambda t: calls.append(t.numel()))
         cache = m.new_cache(2 * 20, 16)
-        p = m.prefill(cache, Hp.to_dev(m, x), [0, 1]).cpu().numpy()
+        xdev = Hp.to_dev(m, x)
+        n0 = pt.lib().pt_launch_count()
+        p = m.prefill(cache, xdev, [0, 1]).cpu().numpy()
+        launches.append(pt.lib().pt_launch_count() - n0)
         n_prefill = len(calls)
         d = m.decode_step(cache, Hp.to_dev(m, xd), [0, 1]).cpu().numpy()
         torch.cuda.synchronize()
         assert m.device_status() == (0, 0)
         outs.append((p, d))
         m.close()
+    # with a track group a prefill launches, per track block, the kernel that spreads the reduced stream and - except
+    # after the last block - the side-stream prefetch of the next layer's QKV weights that runs under the all-reduce
+    syncs = wl.L // wl.D
+    assert launches[1] - launches[0] == syncs + (syncs - 1)
     # one all-reduce per track block: L/D per forward, against 2L for tensor parallelism
     assert n_prefill == wl.L // wl.D and len(calls) == 2 * (wl.L // wl.D)
     assert calls[0] == 2 * 300 * wl.hidden and calls[-1] == 2 * wl.hidden
