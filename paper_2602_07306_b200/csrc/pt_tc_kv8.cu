@@ -129,6 +129,11 @@ __global__ void k_kv_dequant_ctx(const CtxP p) {
 //           put back in order when they are merged.  V codes are multiplied by their scale as f16 pairs, so a
 //           cached V value must fit f16 (|v| <= 65504; below 2^-24 it flushes to zero).
 // With the 128-byte swizzle of the boxes both access patterns are free of bank conflicts.
+// Tried and dropped: both products on mma.sync m16n8k32 with E4M3 operands (q and the probabilities split into two
+// E4M3 numbers hi + lo / 16 carried by rows g and g + 8 of the 16-row tile, K and V codes fed to the MMA as they
+// are, V transposed by byte permutes).  Results matched the oracle, but on this architecture the compiler lowers
+// that MMA to conversions plus f16 MMAs (the profiler shows the HMMA pipe and as many instructions as here):
+// 2314 GB/s against 2985 on the same case.  The 8-bit tensor path of this chip is tcgen05 only.
 constexpr int kDecStages = 3;
 constexpr uint32_t kDecSpin = 1u << 24;
 constexpr int kSlotBytes = 2 * 16 * kDh;                  // K box + V box
