@@ -87,7 +87,10 @@ typedef struct {
                            cross-check; the fp32 dtype always uses them)
                            bit 1: prefill attention on the warp-level mma.sync kernel
                            instead of the tensor-memory (tcgen05) one (diagnostic; that
-                           kernel also serves head_dim 32 and 8-token pages)           */
+                           kernel also serves head_dim 32 and 8-token pages)
+                           bit 2: decode attention of an E4M3 cache on the warp-level mma.sync
+                           kernel (codes converted to f16) instead of the tcgen05 one
+                           (diagnostic)                                                  */
 } pt_config;
 
 typedef struct pt_model pt_model;

@@ -146,5 +146,7 @@ pt_status launch_kv_quant(Call& k, int layer);
 pt_status launch_kv_dequant_ctx(Call& k, int layer);
 pt_status launch_flash_prefill_e4m3(Call& k, const __nv_bfloat16* q, __nv_bfloat16* o);
 pt_status launch_decode_attn_e4m3(Call& k, const __nv_bfloat16* q, int layer, __nv_bfloat16* o);
+// pt_tc_kv8_dec.cu: the same on tcgen05 (the default; the mma.sync kernel serves config flag bit 2)
+pt_status launch_decode_attn_e4m3_tc(Call& k, const __nv_bfloat16* q, int layer, __nv_bfloat16* o);
 
 }  // namespace pt

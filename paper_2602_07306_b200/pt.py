@@ -120,13 +120,13 @@ class Model:
     """A PT model with its packed weights on one CUDA device (torch owns the memory)."""
 
     def __init__(self, *, T, D, L, hidden, heads, kv_heads, ffn, dtype="bf16", rope_base=10000.0,
-                 rms_eps=1e-6, sync_op="sum", max_pos=4096, simt=False, device="cuda:0"):
+                 rms_eps=1e-6, sync_op="sum", max_pos=4096, simt=False, flags=0, device="cuda:0"):
         import torch
         self.torch = torch
         self.device = torch.device(device)
         self.cfg = pt_config(T, D, L, hidden, heads, kv_heads, ffn, rope_base, rms_eps,
                              PT_BF16 if dtype == "bf16" else PT_F32, 1 if sync_op == "mean" else 0,
-                             max_pos, 1 if simt else 0)
+                             max_pos, (1 if simt else 0) | int(flags))
         self.dtype = dtype
         self.tdtype = torch.bfloat16 if dtype == "bf16" else torch.float32
         self.h = _P()

@@ -10,11 +10,11 @@ def oracle_cfg(wl, sync_op="sum"):
                       ffn=wl.ffn, rope_base=wl.rope_base, rms_eps=wl.rms_eps, sync_op=sync_op)
 
 
-def make_model(wl, ws, sync_op="sum", max_pos=4096, simt=False):
+def make_model(wl, ws, sync_op="sum", max_pos=4096, simt=False, flags=0):
     from paper_2602_07306_b200 import pt
     m = pt.Model(T=wl.T, D=wl.D, L=wl.L, hidden=wl.hidden, heads=wl.heads, kv_heads=wl.kv_heads, ffn=wl.ffn,
                  dtype=wl.dtype, rope_base=wl.rope_base, rms_eps=wl.rms_eps, sync_op=sync_op,
-                 max_pos=max_pos, simt=simt)
+                 max_pos=max_pos, simt=simt, flags=flags)
     m.load(ws)
     return m
 

@@ -47,7 +47,7 @@ def test_quantiser_matches_the_oracle_bit_for_bit():
     np.testing.assert_array_equal(got, want_codes)
 
 
-def run_kv8_case(wl, *, B, chunks, decode_steps, ps=16, shuffle=True, sync_op="sum", lens_extra=0):
+def run_kv8_case(wl, *, B, chunks, decode_steps, ps=16, shuffle=True, sync_op="sum", flags=0):
     import torch
     ws = I.WeightSource(wl, gain_jitter=0.1)
     cfg = Hp.oracle_cfg(wl, sync_op)
@@ -56,7 +56,7 @@ def run_kv8_case(wl, *, B, chunks, decode_steps, ps=16, shuffle=True, sync_op="s
     pages = B * (-(-total // ps)) + 2
     order = I.free_list_permutation(pages, seed=11) if shuffle else None
     seq_ids = [3 + 2 * b for b in range(B)]
-    model = Hp.make_model(wl, ws, sync_op=sync_op, max_pos=max(64, total))
+    model = Hp.make_model(wl, ws, sync_op=sync_op, max_pos=max(64, total), flags=flags)
     cache = model.new_cache(pages, ps, order, kv_dtype="e4m3")
     cache.pool.zero_()
     ocache = O.PagedKVCache(cfg, pages, ps, order, kv_format="e4m3")
@@ -84,7 +84,7 @@ def run_kv8_case(wl, *, B, chunks, decode_steps, ps=16, shuffle=True, sync_op="s
         torch.cuda.synchronize()
         assert model.device_status() == (0, 0)
         Hp.assert_close(got.cpu().numpy(), ref, wl.dtype, f"decode step {step}", mean_tol=mean_tol,
-                        log=f"e4m3 cache, {wl.name}: decode step {step} at KV {S + step}")
+                        log=f"e4m3 cache, {wl.name}{' (mma.sync kernel)' if flags & 4 else ''}: decode step {step} at KV {S + step}")
         worst = max(worst, _check_taps(wl, tap.cpu().numpy(), taps, B, 1, mean_tol, delta_tol=DELTA_TOL))
     Hp.record(f"e4m3 cache, {wl.name}: largest error of a layer delta on its own scale", worst, float("nan"), DELTA_TOL, float("nan"))
     model.set_tap(None)
@@ -118,14 +118,22 @@ def _wl(name, T, L, D, H, nq, nkv, F):
                       batch=1, seq=64, seed=0)
 
 
-def test_e4m3_cache_chunked_prefill_and_decode_mha():
-    run_kv8_case(_wl("kv8-mha", 2, 4, 2, 256, 2, 2, 352), B=3, chunks=[24, 1, 23], decode_steps=3)
+# Decode attention of an E4M3 cache has two kernels: the tcgen05 one (codes straight into 8-bit MMAs, keys on the M
+# dimension; the default) and the mma.sync one (codes converted to f16; config flag bit 2).  Both run every case.
+KERNELS = pytest.mark.parametrize("flags", [0, 4], ids=["tcgen05", "mma_sync"])
 
 
-def test_e4m3_cache_gqa4_pages_of_32_tokens():
-    run_kv8_case(_wl("kv8-gqa4", 2, 2, 1, 512, 4, 1, 176), B=2, chunks=[40, 30], decode_steps=2, ps=32)
+@KERNELS
+def test_e4m3_cache_chunked_prefill_and_decode_mha(flags):
+    run_kv8_case(_wl("kv8-mha", 2, 4, 2, 256, 2, 2, 352), B=3, chunks=[24, 1, 23], decode_steps=3, flags=flags)
 
 
-def test_e4m3_cache_gqa8_long_sequences_split_over_key_ranges():
+@KERNELS
+def test_e4m3_cache_gqa4_pages_of_32_tokens(flags):
+    run_kv8_case(_wl("kv8-gqa4", 2, 2, 1, 512, 4, 1, 176), B=2, chunks=[40, 30], decode_steps=2, ps=32, flags=flags)
+
+
+@KERNELS
+def test_e4m3_cache_gqa8_long_sequences_split_over_key_ranges(flags):
     # 700 cached keys and few sequences: the decode step splits every sequence over several key ranges
-    run_kv8_case(_wl("kv8-gqa8", 2, 2, 2, 1024, 8, 1, 256), B=2, chunks=[512, 188], decode_steps=2, sync_op="mean")
+    run_kv8_case(_wl("kv8-gqa8", 2, 2, 2, 1024, 8, 1, 256), B=2, chunks=[512, 188], decode_steps=2, sync_op="mean", flags=flags)
