@@ -17,7 +17,7 @@
 // and one named barrier per tile.  The reference maximum is raised only when it grows by more than 2^8 (the
 // accumulator is then rescaled in tensor memory), so rescales are rare.
 // Roles: warp 0 streams K and V tiles page by page with TMA (one 16 x 128-byte box per page and K|V) through
-// three-stage rings; warp 1 issues the MMAs (scores of tile j+1 before P V of tile j: S^T is double-buffered in
+// three-stage rings; warp 1 issues the MMAs (the scores of tile j+2 right behind P V of tile j: S^T is double-buffered in
 // tensor memory, P in shared memory); warps 2-5 are the softmax threads.  Every mbarrier wait is bounded; the named
 // barrier is executed exactly once per tile and twice at the end by every softmax warp whatever happened before.
 #include <cuda_fp8.h>
@@ -30,7 +30,7 @@ namespace {
 
 constexpr int kDh = 128;
 constexpr int kThreads = 192;
-constexpr int kStages = 3;
+constexpr int kStages = 2;
 constexpr int kTile = 128 * kDh;            // bytes of a K or V tile: 128 keys x 128 code bytes
 constexpr int kQBytes = 16 * kDh;           // q (and one P buffer): 16 rows of 128 bytes
 constexpr uint32_t kSpin = 1u << 26;
@@ -149,7 +149,7 @@ struct Dec8TcP {
 
 constexpr int kSmem = 1024 + 2 * kStages * kTile + kQBytes + 2 * kQBytes + 2 * 4 * 12 * 4 + 8 * 4 + B_COUNT * 8 + 64;
 
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 3)
 k_decode_attn_e4m3_tc(const __grid_constant__ CUtensorMap kvmap, const Dec8TcP pp) {
     const AttnP& p = pp.a;
     extern __shared__ uint8_t smem_raw[];
@@ -253,9 +253,9 @@ k_decode_attn_e4m3_tc(const __grid_constant__ CUtensorMap kvmap, const Dec8TcP p
         // is free, so q is guarded by its own arrival on B_PFULL + 1 (see there)
         wait(B_PFULL + 1, 0u, LOC_FLASH_QFULL);
         if (n_tiles > 0) qk(0);
+        if (n_tiles > 1) qk(1);
         for (int j = 0; j < n_tiles && ok; ++j) {
             const int s = j % kStages, bb = j & 1;
-            if (j + 1 < n_tiles) qk(j + 1);
             // P buffer bb: the q hand-over used one phase of B_PFULL + 1, so that barrier runs one phase ahead
             wait(B_PFULL + bb, ((uint32_t)(j >> 1) + (bb ? 1u : 0u)) & 1u, LOC_FLASH_PFULL);
             wait(B_VFULL + s, (uint32_t)(j / kStages) & 1u, LOC_FLASH_VFULL);
@@ -266,6 +266,7 @@ k_decode_attn_e4m3_tc(const __grid_constant__ CUtensorMap kvmap, const Dec8TcP p
                 mma_f8(tmem_base + 32, desc_mnmajor(va + ks * 4096), desc_kmajor(pa + ks * 32), idesc_pv, j > 0 || ks != 0);
             tc_commit(&bars[B_PEMPTY + bb]);
             tc_commit(&bars[B_VEMPTY + s]);
+            if (j + 2 < n_tiles) qk(j + 2);                    // scores run two tiles ahead of the softmax threads
         }
         __syncwarp();
     } else {
