@@ -5,7 +5,7 @@
     python -m paper_2602_07306_b200.kbench layer --T 8 --B 2 --S 4096 --H 1024 --nq 8 --nkv 8 --F 2816
     python -m paper_2602_07306_b200.kbench generate --B 1 --S 1024 --new 64 [--depth 2|4|8]
     python -m paper_2602_07306_b200.kbench gemm --T 8 --M 32768 --N 3072 --K 1024 [--bn 256] [--fold]
-    python -m paper_2602_07306_b200.kbench step --T 4 --B 64 --len 2048 --H 2048 --nq 16 --nkv 4 --F 5632 [--kv8 1]
+    python -m paper_2602_07306_b200.kbench step --T 4 --B 64 --len 2048 --H 2048 --nq 16 --nkv 4 --F 5632 [--kv8 1 [--mma_sync 1]]
 
 Prints one JSON line: average device time per launch (CUDA events on the launching stream,
 after warm-up) and the achieved GB/s (decode: K/V bytes read) or TFLOP/s (gemm).  Small cases of
@@ -129,7 +129,7 @@ def step(a):
     achieved rate of the attention kernel over the bytes of the cached vectors it reads."""
     dev = torch.device("cuda:0")
     m = pt.Model(T=a.T, D=a.layers, L=a.layers, hidden=a.H, heads=a.nq, kv_heads=a.nkv, ffn=a.F, dtype="bf16",
-                 max_pos=a.len + 16, device=dev)
+                 max_pos=a.len + 16, flags=4 if a.mma_sync else 0, device=dev)
     m.init_random(0)
     dh = a.H // a.nq
     cache = m.new_cache(a.B * (-(-(a.len + 1) // a.ps)), a.ps, kv_dtype="e4m3" if a.kv8 else "model")
@@ -248,7 +248,7 @@ def main():
     for k, v in dict(B=1, S=1024, new=64, vocab=32000, depth=0, iters=3, warmup=1).items():
         gn.add_argument("--" + k, type=int, default=v)
     sp = sub.add_parser("step")
-    for k, v in dict(T=4, B=64, len=2048, H=2048, nq=16, nkv=4, F=5632, ps=16, layers=2, kv8=0, iters=10, warmup=3).items():
+    for k, v in dict(T=4, B=64, len=2048, H=2048, nq=16, nkv=4, F=5632, ps=16, layers=2, kv8=0, mma_sync=0, iters=10, warmup=3).items():
         sp.add_argument("--" + k, type=int, default=v)
     gm = sub.add_parser("gemm")
     for k, v in dict(T=8, M=4096, N=3072, K=1024, bn=0, iters=20, warmup=3).items():
