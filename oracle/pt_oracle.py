@@ -16,7 +16,8 @@ consistent choice is valid): rotary pairs are (j, j + dh/2); query head i reads
 KV head i // G; the all-reduce of Algorithm 1 is a SUM (MEAN is available as an
 option); "Set h_i = h" of Algorithm 1 is read as inside the if-block (its own
 comment says it follows the all-reduce); the optional FP8 storage format of the KV
-cache (E4M3 codes with one power-of-two scale per cached vector).
+cache (E4M3 codes with one power-of-two scale per cached vector); the PT-MoE feed-forward
+(linear router, top-k by logit with the lower index winning ties, softmax over the chosen logits).
 
 Shapes: T tracks, L layers, D track-block depth, H per-track hidden, nq / nkv
 query / KV heads per track, dh = H / nq, G = nq / nkv, F feed-forward width.
@@ -41,6 +42,8 @@ class PTConfig:
     rope_base: float = 10000.0
     rms_eps: float = 1e-6
     sync_op: str = "sum"          # "sum" (the all-reduce of Algorithm 1) or "mean"
+    experts: int = 0              # > 0: every track's feed-forward is a mixture of this many experts of width ffn (PT-MoE)
+    top_k: int = 0                # experts evaluated per token
 
     def __post_init__(self):
         if self.T < 1 or self.L < 1 or self.D < 1:
@@ -54,6 +57,8 @@ class PTConfig:
             raise ValueError("head_dim must be even for rotary pairs")
         if self.sync_op not in ("sum", "mean"):
             raise ValueError("sync_op")
+        if self.experts < 0 or (self.experts > 0 and not 1 <= self.top_k <= self.experts) or (self.experts == 0 and self.top_k):
+            raise ValueError("top_k must lie in [1, experts]")
 
     @property
     def head_dim(self) -> int:
@@ -126,6 +131,34 @@ def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, qpos: np.ndarray) -> 
         p = np.exp(s)
         p = p / np.sum(p, axis=-1, keepdims=True)
         out[:, i, :] = p @ vh
+    return out
+
+
+def moe_gates(logits: np.ndarray, top_k: int) -> np.ndarray:
+    """Routing weights of a mixture-of-experts layer: for every row of logits[..., E] the top_k largest
+    logits (the lower index wins a tie) get softmax weights among themselves, all others 0."""
+    logits = np.asarray(logits, np.float64)
+    E = logits.shape[-1]
+    # stable sort of -logits: equal logits keep index order, so the lower index ranks first
+    order = np.argsort(-logits, axis=-1, kind="stable")
+    chosen = order[..., :top_k]
+    sel = np.take_along_axis(logits, chosen, axis=-1)
+    w = np.exp(sel - sel.max(axis=-1, keepdims=True))
+    w = w / w.sum(axis=-1, keepdims=True)
+    gates = np.zeros(logits.shape)
+    np.put_along_axis(gates, chosen, w, axis=-1)
+    return gates
+
+
+def moe_ffn(c: np.ndarray, wr: np.ndarray, wg: np.ndarray, wu: np.ndarray, wd: np.ndarray, top_k: int) -> np.ndarray:
+    """PT-MoE feed-forward of one track (the paper names it in one sentence - an MoE layer inside each track -
+    and defines nothing else; declared here): router logits c wr^T over E experts, moe_gates, and
+    sum_e gate_e * (silu(c wg[e]^T) * (c wu[e]^T)) wd[e]^T.  wr [E, H], wg / wu [E, F, H], wd [E, H, F]."""
+    gates = moe_gates(c @ wr.T, top_k)
+    out = np.zeros(c.shape)
+    for e in range(wr.shape[0]):
+        y = (silu(c @ wg[e].T) * (c @ wu[e].T)) @ wd[e].T
+        out = out + gates[..., e:e + 1] * y
     return out
 
 
@@ -267,7 +300,12 @@ def _layer(cfg: PTConfig, w: dict, h: np.ndarray, cache: PagedKVCache, t: int, l
     attn_delta = o.reshape(B, S, nq * dh) @ W["wo"].T
     h = h + attn_delta
     c = rmsnorm(h, W["g2"], cfg.rms_eps)
-    ffn_delta = (silu(c @ W["wg"].T) * (c @ W["wu"].T)) @ W["wd"].T
+    if cfg.experts:
+        ffn_delta = moe_ffn(c, W["wr"], W["wg"], W["wu"], W["wd"], cfg.top_k)
+        if taps is not None:
+            taps.setdefault("router_logits", {})[(t, l)] = c @ W["wr"].T
+    else:
+        ffn_delta = (silu(c @ W["wg"].T) * (c @ W["wu"].T)) @ W["wd"].T
     if taps is not None:
         taps.setdefault("attn_delta", {})[(t, l)] = attn_delta
         taps.setdefault("ffn_delta", {})[(t, l)] = ffn_delta

@@ -17,7 +17,7 @@ from dataclasses import dataclass, field
 import numpy as np
 
 # tensor kinds, also the draw order inside one (track, layer)
-KINDS = ("wq", "wk", "wv", "wo", "wg", "wu", "wd", "g1", "g2")
+KINDS = ("wq", "wk", "wv", "wo", "wg", "wu", "wd", "g1", "g2", "wr")     # wr: the router of a PT-MoE layer (only with experts > 0)
 _KIND_ID = {k: i for i, k in enumerate(KINDS)}
 _KIND_X = 100        # prefill inputs
 _KIND_XDEC = 101     # decode inputs
@@ -69,6 +69,8 @@ class Workload:
     rope_base: float = 10000.0
     rms_eps: float = 1e-6
     seed: int = 0
+    experts: int = 0      # > 0: PT-MoE - every track's feed-forward is a mixture of `experts` experts of width ffn
+    top_k: int = 0
 
     @property
     def head_dim(self) -> int:
@@ -76,14 +78,15 @@ class Workload:
 
     def weight_shape(self, kind: str) -> tuple:
         H, dh, F = self.hidden, self.head_dim, self.ffn
+        E = (self.experts,) if self.experts else ()
         return {
             "wq": (self.heads * dh, H), "wk": (self.kv_heads * dh, H), "wv": (self.kv_heads * dh, H),
-            "wo": (H, self.heads * dh), "wg": (F, H), "wu": (F, H), "wd": (H, F),
-            "g1": (H,), "g2": (H,),
+            "wo": (H, self.heads * dh), "wg": E + (F, H), "wu": E + (F, H), "wd": E + (H, F),
+            "g1": (H,), "g2": (H,), "wr": (max(self.experts, 1), H),
         }[kind]
 
     def params_per_track_layer(self) -> int:
-        H, dh, F = self.hidden, self.head_dim, self.ffn
+        H, dh, F = self.hidden, self.head_dim, self.ffn * max(self.experts, 1)
         return 2 * H * self.heads * dh + 2 * H * self.kv_heads * dh + 3 * H * F
 
 
@@ -122,8 +125,9 @@ class WeightSource:
     """
 
     def __init__(self, wl: Workload, seed: int | None = None, std: float = 0.02,
-                 gain_jitter: float = 0.0, zero: tuple = ()):
+                 gain_jitter: float = 0.0, zero: tuple = (), router_std: float | None = None):
         self.wl, self.std, self.gain_jitter, self.zero = wl, std, gain_jitter, tuple(zero)
+        self.router_std = std if router_std is None else router_std
         self.seed = wl.seed if seed is None else seed
 
     def one(self, t: int, l: int, kind: str) -> np.ndarray:
@@ -135,12 +139,14 @@ class WeightSource:
             w = np.ones(shape, np.float32)
             if self.gain_jitter:
                 w = w + np.float32(self.gain_jitter) * g.standard_normal(shape, dtype=np.float32)
+        elif kind == "wr":
+            return g.standard_normal(shape, dtype=np.float32) * np.float32(self.router_std)    # the router stays fp32
         else:
             w = g.standard_normal(shape, dtype=np.float32) * np.float32(self.std)
         return round_to_bf16(w) if self.wl.dtype == "bf16" else w
 
     def get(self, t: int, l: int) -> dict:
-        return {k: self.one(t, l, k) for k in KINDS}
+        return {k: self.one(t, l, k) for k in KINDS if k != "wr" or self.wl.experts}
 
 
 def prefill_inputs(wl: Workload, batch: int | None = None, seq: int | None = None,

@@ -7,7 +7,8 @@ from paper_2602_07306_b200 import inputs as I
 
 def oracle_cfg(wl, sync_op="sum"):
     return O.PTConfig(T=wl.T, D=wl.D, L=wl.L, hidden=wl.hidden, heads=wl.heads, kv_heads=wl.kv_heads,
-                      ffn=wl.ffn, rope_base=wl.rope_base, rms_eps=wl.rms_eps, sync_op=sync_op)
+                      ffn=wl.ffn, rope_base=wl.rope_base, rms_eps=wl.rms_eps, sync_op=sync_op,
+                      experts=wl.experts, top_k=wl.top_k)
 
 
 def make_model(wl, ws, sync_op="sum", max_pos=4096, simt=False, flags=0):

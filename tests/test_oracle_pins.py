@@ -518,3 +518,82 @@ def test_fp8_cache_quantises_what_it_stores_and_nothing_else():
     np.testing.assert_allclose(rest, got[:, 10:S - 1], rtol=1e-12, atol=1e-13)
     last = O.pt_decode_step(cfg, ws, x[:, :, S - 1], c8b, [0, 1])
     np.testing.assert_allclose(last, got[:, S - 1], rtol=1e-12, atol=1e-13)
+
+
+# ---------------------------------------------------------------- PT-MoE feed-forward
+
+def test_moe_gates_by_hand_and_against_torch():
+    # a hand-checked row: logits 1, 3, 3, 0 with top-2: experts 1 and 2 tie for the top, both chosen, half each
+    g = O.moe_gates(np.array([[1.0, 3.0, 3.0, 0.0]]), 2)
+    np.testing.assert_allclose(g, [[0.0, 0.5, 0.5, 0.0]])
+    # a tie at the boundary of the choice: the lower index wins
+    g = O.moe_gates(np.array([[2.0, 5.0, 2.0, 2.0]]), 2)
+    e = np.exp(2.0 - 5.0)
+    np.testing.assert_allclose(g, [[e / (1 + e), 1 / (1 + e), 0.0, 0.0]])
+    rng = np.random.default_rng(0)
+    logits = rng.standard_normal((50, 7, 6))
+    for k in (1, 2, 6):
+        got = O.moe_gates(logits, k)
+        tl = torch.from_numpy(logits)
+        vals, idx = torch.topk(tl, k, dim=-1)
+        want = torch.zeros_like(tl).scatter(-1, idx, torch.softmax(vals, dim=-1)).numpy()
+        np.testing.assert_allclose(got, want, rtol=1e-13, atol=1e-15)
+        assert np.all((got > 0).sum(-1) == k) and np.allclose(got.sum(-1), 1.0)
+
+
+def test_moe_ffn_special_cases():
+    rng = np.random.default_rng(1)
+    H, F, E, n = 16, 24, 4, 9
+    c = rng.standard_normal((n, H))
+    wr = rng.standard_normal((E, H))
+    wg, wu, wd = rng.standard_normal((E, F, H)) * 0.3, rng.standard_normal((E, F, H)) * 0.3, rng.standard_normal((E, H, F)) * 0.3
+    dense = lambda e: (O.silu(c @ wg[e].T) * (c @ wu[e].T)) @ wd[e].T
+    # one expert: the plain feed-forward, whatever the router says
+    np.testing.assert_allclose(O.moe_ffn(c, wr[:1], wg[:1], wu[:1], wd[:1], 1), dense(0), rtol=1e-13)
+    # identical experts: the gates sum to one, so the mixture is that expert
+    same = lambda a: np.repeat(a[:1], E, axis=0)
+    np.testing.assert_allclose(O.moe_ffn(c, wr, same(wg), same(wu), same(wd), 2), dense(0), rtol=1e-12)
+    # all experts chosen: a softmax mixture of every expert, written out
+    p = torch.softmax(torch.from_numpy(c @ wr.T), dim=-1).numpy()
+    np.testing.assert_allclose(O.moe_ffn(c, wr, wg, wu, wd, E), sum(p[:, e:e + 1] * dense(e) for e in range(E)), rtol=1e-12)
+    # top-1 by brute force, token by token
+    want = np.stack([dense(int(np.argmax(c[i] @ wr.T)))[i] for i in range(n)])
+    np.testing.assert_allclose(O.moe_ffn(c, wr, wg, wu, wd, 1), want, rtol=1e-12)
+    # renumbering the experts (router rows and expert weights together) changes nothing
+    perm = np.array([2, 0, 3, 1])
+    np.testing.assert_allclose(O.moe_ffn(c, wr[perm], wg[perm], wu[perm], wd[perm], 2), O.moe_ffn(c, wr, wg, wu, wd, 2), rtol=1e-12)
+
+
+def test_moe_stack_reduces_to_the_dense_stack_with_one_expert_and_keeps_algorithm_1s_invariants():
+    base = dict(T=2, L=4, D=2, hidden=32, heads=4, kv_heads=2, ffn=48, dtype="f32", mode="prefill", batch=2, seq=12, seed=3)
+    wl1 = I.Workload("moe1", experts=1, top_k=1, **base)
+    wl0 = I.Workload("dense", **base)
+    ws1, ws0 = I.WeightSource(wl1, std=0.2), I.WeightSource(wl0, std=0.2)
+    x = I.prefill_inputs(wl0)
+    cfg0 = O.PTConfig(T=2, D=2, L=4, hidden=32, heads=4, kv_heads=2, ffn=48)
+    cfg1 = O.PTConfig(T=2, D=2, L=4, hidden=32, heads=4, kv_heads=2, ffn=48, experts=1, top_k=1)
+
+    class One:                                    # the dense weights, presented as one expert
+        def get(self, t, l):
+            w = dict(ws0.get(t, l))
+            for k in ("wg", "wu", "wd"):
+                w[k] = w[k][None]
+            w["wr"] = ws1.get(t, l)["wr"]
+            return w
+    a = O.pt_prefill(cfg0, ws0, x, O.PagedKVCache(cfg0, 8, 16), [0, 1])
+    b = O.pt_prefill(cfg1, One(), x, O.PagedKVCache(cfg1, 8, 16), [0, 1])
+    np.testing.assert_allclose(a, b, rtol=1e-12, atol=1e-13)
+    # four experts, top-2: decode equals a prefill row, and the sync count is still L / D
+    wl4 = I.Workload("moe4", experts=4, top_k=2, **base)
+    ws4 = I.WeightSource(wl4, std=0.2, router_std=0.5)
+    cfg4 = O.PTConfig(T=2, D=2, L=4, hidden=32, heads=4, kv_heads=2, ffn=48, experts=4, top_k=2)
+    taps = {}
+    full = O.pt_prefill(cfg4, ws4, x, O.PagedKVCache(cfg4, 8, 16), [0, 1], taps)
+    assert taps["syncs"] == 2 and taps["router_logits"][(1, 3)].shape == (2, 12, 4)
+    cache = O.PagedKVCache(cfg4, 8, 16)
+    O.pt_prefill(cfg4, ws4, x[:, :, :11], cache, [0, 1])
+    last = O.pt_decode_step(cfg4, ws4, x[:, :, 11], cache, [0, 1])
+    np.testing.assert_allclose(last, full[:, 11], rtol=1e-12, atol=1e-13)
+    assert np.abs(full - a).max() > 1e-3          # and it is not the dense stack
+    with pytest.raises(ValueError):
+        O.PTConfig(T=2, D=2, L=4, hidden=32, heads=4, kv_heads=2, ffn=48, experts=4, top_k=5)
