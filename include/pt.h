@@ -65,7 +65,8 @@ typedef enum { PT_KV_MODEL = 0, PT_KV_E4M3 = 1 } pt_kv_dtype;
 typedef enum {
     PT_WQ = 0, PT_WK = 1, PT_WV = 2, PT_WO = 3, PT_WG = 4, PT_WU = 5, PT_WD = 6,
     PT_G1 = 7, /* RMSNorm gain before attention */
-    PT_G2 = 8  /* RMSNorm gain before the feed-forward */
+    PT_G2 = 8, /* RMSNorm gain before the feed-forward */
+    PT_WR = 9  /* router of a PT-MoE layer: [experts][hidden], always fp32 */
 } pt_weight_kind;
 
 /* Architecture of a PT stack: Algorithm 1's n (= T), L, D; heads per track as in Table 1. */
@@ -91,6 +92,17 @@ typedef struct {
                            bit 2: decode attention of an E4M3 cache on the warp-level mma.sync
                            kernel (codes converted to f16) instead of the tcgen05 one
                            (diagnostic)                                                  */
+    int32_t experts;    /* 0: the plain SwiGLU feed-forward.  > 0 (at most 16; bf16 models on the
+                           tensor-core path): PT-MoE - the feed-forward of every track and layer is a
+                           mixture of `experts` SwiGLU experts of width ffn each.  The paper names the
+                           combination in one sentence (Section 2.2, "Contrast with MoE": an MoE layer
+                           inside each track) and defines nothing else; this library's definition: router
+                           logits = rmsnorm(h; g2) Wr^T, the top_k largest logits (the lower index wins a
+                           tie) get softmax weights among themselves, the layer's output is the weighted
+                           sum of the chosen experts' outputs.  Every expert is evaluated for every
+                           token and weighted afterwards (unchosen experts by zero): the result is the
+                           mixture's, the routing sparsity is not exploited                         */
+    int32_t top_k;      /* experts chosen per token, 1 .. experts (0 with experts == 0)              */
 } pt_config;
 
 typedef struct pt_model pt_model;
@@ -117,9 +129,13 @@ pt_status pt_model_bind_weights(pt_model* m, void* dev_buf, size_t bytes);
 
 /* Copy one weight tensor of (track, layer) into the packed buffer.  `dev_src` (device) is
  * [out, in] row-major in the model dtype (y = x W^T); gains are [hidden] in fp32.
- * Asynchronous on `stream`. */
+ * Asynchronous on `stream`.  With experts > 0, PT_WR takes the router [experts][hidden] in fp32 and
+ * PT_WG / PT_WU / PT_WD go through pt_model_set_expert_weight instead. */
 pt_status pt_model_set_weight(pt_model* m, int32_t track, int32_t layer, int32_t kind,
                               const void* dev_src, void* stream);
+/* The same for one expert's PT_WG, PT_WU ([ffn, hidden]) or PT_WD ([hidden, ffn]) of a PT-MoE model. */
+pt_status pt_model_set_expert_weight(pt_model* m, int32_t track, int32_t layer, int32_t expert, int32_t kind,
+                                     const void* dev_src, void* stream);
 
 /* Number of track-sync points of one forward pass: L / D (Section 2.2). */
 int32_t pt_sync_count(const pt_model* m);

@@ -54,14 +54,15 @@ static size_t carve(const pt_model* m, int64_t M, int B, int maxp, bool fp8, int
     void* a = take(TMH * m->esz);
     void* qkv = take((size_t)c.T * M * m->Nqkv * m->esz);
     void* o = take((size_t)c.T * M * m->QD * m->esz);
-    void* gu = m->tc ? nullptr : take((size_t)c.T * M * 2 * c.ffn * m->esz);
-    void* z = take((size_t)c.T * M * c.ffn * m->esz);
+    void* gu = m->tc ? nullptr : take((size_t)c.T * M * 2 * m->Ftot * m->esz);
+    void* z = take((size_t)c.T * M * m->Ftot * m->esz);
+    float* gates = m->E ? (float*)take((size_t)c.T * M * m->E * 4) : nullptr;
     float* ssq = m->tc ? (float*)take((size_t)c.T * M * ((c.hidden + kSsqTile - 1) / kSsqTile) * 4) : nullptr;
     float* part = m->tc ? (float*)take((size_t)c.T * B * kMaxSplits * c.heads * (m->dh + 2) * 4) : nullptr;
     void* kv_stage = fp8 ? take((size_t)c.T * 2 * m->KVD * M * 2) : nullptr;
     void* attn_kv = fp8 && ctx_keys > 0 ? take((size_t)c.T * 2 * m->KVD * (size_t)ctx_keys * 2) : nullptr;
     if (w) {
-        w->kv_stage = kv_stage; w->attn_kv = attn_kv;
+        w->kv_stage = kv_stage; w->attn_kv = attn_kv; w->gates = gates;
         w->hT = hT; w->hS = hS; w->a = a; w->qkv = qkv; w->o = o; w->gu = gu; w->z = z;
         w->ssq = ssq; w->part = part; w->total = off;
         (void)meta;
@@ -127,6 +128,10 @@ pt_status pt_model_create(const pt_config* cfg, pt_model** out) {
     if (c.ffn % 16) PT_FAIL(PT_ERR_UNSUPPORTED, "ffn must be a multiple of 16");
     if (c.hidden % 16) PT_FAIL(PT_ERR_UNSUPPORTED, "hidden must be a multiple of 16");
     if (c.heads / c.kv_heads > 8) PT_FAIL(PT_ERR_UNSUPPORTED, "more than 8 query heads per KV head");
+    if (c.experts < 0 || (c.experts == 0 && c.top_k != 0) || (c.experts > 0 && (c.top_k < 1 || c.top_k > c.experts)))
+        PT_FAIL(PT_ERR_BAD_CONFIG, "top_k must lie in [1, experts] (and be 0 without experts)");
+    if (c.experts > 16) PT_FAIL(PT_ERR_UNSUPPORTED, "more than 16 experts");
+    if (c.experts > 0 && (c.dtype != PT_BF16 || (c.flags & 1))) PT_FAIL(PT_ERR_UNSUPPORTED, "PT-MoE needs a bf16 model on the tensor-core path");
     pt_model* m = new (std::nothrow) pt_model();
     if (!m) PT_FAIL(PT_ERR_INVALID_ARG, "out of host memory");
     m->cfg = c;
@@ -137,6 +142,8 @@ pt_status pt_model_create(const pt_config* cfg, pt_model** out) {
     m->Nqkv = m->QD + 2 * m->KVD;
     m->esz = c.dtype == PT_BF16 ? 2 : 4;
     m->tc = c.dtype == PT_BF16 && !(c.flags & 1);
+    m->E = c.experts;
+    m->Ftot = std::max(c.experts, 1) * c.ffn;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes, 256); return o; };
     m->off_wqkv = take(m->wqkv_layer() * c.L * m->esz);
@@ -148,6 +155,7 @@ pt_status pt_model_create(const pt_config* cfg, pt_model** out) {
     m->off_cos = take((size_t)c.max_pos * (dh / 2) * 4);
     m->off_sin = take((size_t)c.max_pos * (dh / 2) * 4);
     m->off_cs16 = take((size_t)c.max_pos * (dh / 2) * 4);
+    m->off_wr = take((size_t)c.L * c.T * m->E * c.hidden * 4);
     m->off_status = take(kStatusWords * 4);
     m->total_bytes = off;
     *out = m;
@@ -239,9 +247,17 @@ pt_status pt_model_set_weight(pt_model* m, int32_t track, int32_t layer, int32_t
     if (!m || !dev_src) PT_FAIL(PT_ERR_INVALID_ARG, "null argument");
     if (!m->wbuf) PT_FAIL(PT_ERR_STATE, "pt_model_bind_weights has not been called");
     const pt_config& c = m->cfg;
-    if (track < 0 || track >= c.T || layer < 0 || layer >= c.L || kind < 0 || kind > PT_G2)
+    if (track < 0 || track >= c.T || layer < 0 || layer >= c.L || kind < 0 || kind > PT_WR)
         PT_FAIL(PT_ERR_INVALID_ARG, "track/layer/kind out of range");
     cudaStream_t st = (cudaStream_t)stream;
+    if (kind == PT_WR) {
+        if (!m->E) PT_FAIL(PT_ERR_INVALID_ARG, "the model has no router (experts == 0)");
+        float* dst = (float*)(m->wbuf + m->off_wr) + ((size_t)layer * c.T + track) * m->E * c.hidden;
+        PT_CUDA(cudaMemcpyAsync(dst, dev_src, (size_t)m->E * c.hidden * 4, cudaMemcpyDeviceToDevice, st));
+        return PT_OK;
+    }
+    if (m->E && (kind == PT_WG || kind == PT_WU || kind == PT_WD))
+        PT_FAIL(PT_ERR_INVALID_ARG, "a PT-MoE model takes its feed-forward weights expert by expert: pt_model_set_expert_weight");
     if (kind == PT_G1 || kind == PT_G2) {
         float* dst = (float*)(m->wbuf + (kind == PT_G1 ? m->off_g1 : m->off_g2)) + ((size_t)layer * c.T + track) * c.hidden;
         PT_CUDA(cudaMemcpyAsync(dst, dev_src, (size_t)c.hidden * 4, cudaMemcpyDeviceToDevice, st));
@@ -254,11 +270,27 @@ pt_status pt_model_set_weight(pt_model* m, int32_t track, int32_t layer, int32_t
         case PT_WO:
             base = m->wbuf + m->off_wo + ((size_t)layer * c.T + track) * c.hidden * m->QD * m->esz; break;
         case PT_WG: case PT_WU:
-            base = m->wbuf + m->off_wgu + ((size_t)layer * c.T + track) * 2 * c.ffn * c.hidden * m->esz; break;
+            base = m->wbuf + m->off_wgu + ((size_t)layer * c.T + track) * 2 * m->Ftot * c.hidden * m->esz; break;
         default:
-            base = m->wbuf + m->off_wd + ((size_t)layer * c.T + track) * c.hidden * c.ffn * m->esz; break;
+            base = m->wbuf + m->off_wd + ((size_t)layer * c.T + track) * c.hidden * m->Ftot * m->esz; break;
     }
     launch_pack(m, kind, dev_src, base, st);
+    PT_CUDA(cudaGetLastError());
+    return PT_OK;
+}
+
+pt_status pt_model_set_expert_weight(pt_model* m, int32_t track, int32_t layer, int32_t expert, int32_t kind,
+                                     const void* dev_src, void* stream) {
+    if (!m || !dev_src) PT_FAIL(PT_ERR_INVALID_ARG, "null argument");
+    if (!m->wbuf) PT_FAIL(PT_ERR_STATE, "pt_model_bind_weights has not been called");
+    const pt_config& c = m->cfg;
+    if (!m->E) PT_FAIL(PT_ERR_INVALID_ARG, "the model has no experts");
+    if (track < 0 || track >= c.T || layer < 0 || layer >= c.L || expert < 0 || expert >= m->E)
+        PT_FAIL(PT_ERR_INVALID_ARG, "track/layer/expert out of range");
+    if (kind != PT_WG && kind != PT_WU && kind != PT_WD) PT_FAIL(PT_ERR_INVALID_ARG, "kind must be PT_WG, PT_WU or PT_WD");
+    char* base = kind == PT_WD ? m->wbuf + m->off_wd + ((size_t)layer * c.T + track) * c.hidden * m->Ftot * m->esz
+                               : m->wbuf + m->off_wgu + ((size_t)layer * c.T + track) * 2 * m->Ftot * c.hidden * m->esz;
+    launch_pack(m, kind, dev_src, base, (cudaStream_t)stream, expert);
     PT_CUDA(cudaGetLastError());
     return PT_OK;
 }

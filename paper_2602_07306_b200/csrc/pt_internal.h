@@ -57,10 +57,11 @@ inline int current_device() {
 struct pt_model {
     pt_config cfg;
     int dh, G, QD, KVD, Nqkv;             // head_dim, heads/kv_heads, nq*dh, nkv*dh, QD+2*KVD
+    int E, Ftot;                          // experts of a PT-MoE layer (0: plain feed-forward) and the packed width max(E, 1) * ffn
     size_t esz;                           // bytes per element of the model dtype
     bool tc;                              // bf16 tensor-core path (else SIMT)
     // byte offsets inside the bound weight buffer; matrices are [L][T][rows][cols]
-    size_t off_wqkv, off_wo, off_wgu, off_wd, off_g1, off_g2, off_cos, off_sin, off_cs16, off_status, total_bytes;
+    size_t off_wqkv, off_wo, off_wgu, off_wd, off_g1, off_g2, off_cos, off_sin, off_cs16, off_wr, off_status, total_bytes;
     char* wbuf = nullptr;
     char* lm_buf = nullptr;                // embedding table, LM head, final gain (pt_lm_bind)
     int lm_vocab = 0;
@@ -83,8 +84,10 @@ struct pt_model {
 
     size_t wqkv_layer() const { return (size_t)cfg.T * Nqkv * cfg.hidden; }     // elements
     size_t wo_layer() const { return (size_t)cfg.T * cfg.hidden * QD; }
-    size_t wgu_layer() const { return (size_t)cfg.T * 2 * cfg.ffn * cfg.hidden; }
-    size_t wd_layer() const { return (size_t)cfg.T * cfg.hidden * cfg.ffn; }
+    size_t wgu_layer() const { return (size_t)cfg.T * 2 * Ftot * cfg.hidden; }
+    size_t wd_layer() const { return (size_t)cfg.T * cfg.hidden * Ftot; }
+    // PT-MoE: fp32 router [L][T][E][hidden]
+    const float* router(int l) const { return (const float*)(wbuf + off_wr) + (size_t)l * cfg.T * E * cfg.hidden; }
     int* status() const { return (int*)(wbuf + off_status); }
     const float* gain(int which, int l) const {
         return (const float*)(wbuf + (which ? off_g2 : off_g1)) + (size_t)l * cfg.T * cfg.hidden;
@@ -140,6 +143,7 @@ struct Work {
     float* ssq;     // [T][M][H/kSsqTile] partial sums of squares (tc)
     float* part;    // decode split-KV partials
     void* kv_stage; // E4M3 caches: [T][K|V][kv_head][M][dh] bf16, this call's K and V as projected
+    float* gates;   // PT-MoE: [T][M][E] routing weights of the current layer (0 for the experts a token did not choose)
     void* attn_kv;  // E4M3 caches, prefill: [T][page][K|V][kv_head][16][dh] bf16 copy of code * scale of every key attended to
     size_t total;
 };
@@ -184,7 +188,7 @@ void plan_decode_splits(const int32_t* lens, int B, int ps, int64_t units, int32
 
 // pt_simt.cu
 pt_status simt_forward(Call& k);
-void launch_pack(const pt_model* m, int kind, const void* src, void* dst_matrix_base, cudaStream_t st);
+void launch_pack(const pt_model* m, int kind, const void* src, void* dst_matrix_base, cudaStream_t st, int expert = 0);
 
 // pt_tc.cu (bf16 tensor-core path)
 pt_status tc_build_weight_maps(pt_model* m);

@@ -22,32 +22,36 @@ __device__ __forceinline__ void report(int* status, int code, int loc) {
 // ---- weight packing: rows of one [rows, cols] source matrix go to mapped rows of the packed matrix.
 // kind: PT_WQ/PT_WK/PT_WV -> rows offset inside [Nqkv, H]; PT_WG/PT_WU -> interleaved in groups
 // of 16 rows (gate rows 32g..32g+15, up rows 32g+16..32g+31); others -> identity.
+// A PT-MoE model packs its experts side by side: expert e's gate/up rows follow those of expert e - 1 (row_off),
+// its down-projection columns sit at e * ffn of rows that are Ftot wide (dst_cols, col_off).
 template <class E>
-__global__ void k_pack(const E* __restrict__ src, E* __restrict__ dst, int rows, int cols, int row_off, int interleave) {
+__global__ void k_pack(const E* __restrict__ src, E* __restrict__ dst, int rows, int cols, int row_off, int interleave,
+                       int dst_cols, int col_off) {
     size_t n = (size_t)rows * cols;
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
         int r = (int)(i / cols), c = (int)(i % cols);
-        int dr = interleave ? (r / 16) * 32 + (interleave - 1) * 16 + r % 16 : r + row_off;
-        dst[(size_t)dr * cols + c] = src[i];
+        int dr = (interleave ? (r / 16) * 32 + (interleave - 1) * 16 + r % 16 : r) + row_off;
+        dst[(size_t)dr * dst_cols + col_off + c] = src[i];
     }
 }
 
-void launch_pack(const pt_model* m, int kind, const void* src, void* dst, cudaStream_t st) {
+void launch_pack(const pt_model* m, int kind, const void* src, void* dst, cudaStream_t st, int expert) {
     const pt_config& c = m->cfg;
-    int rows, cols, row_off = 0, il = 0;
+    int rows, cols, row_off = 0, il = 0, dst_cols = 0, col_off = 0;
     switch (kind) {
         case PT_WQ: rows = m->QD; cols = c.hidden; break;
         case PT_WK: rows = m->KVD; cols = c.hidden; row_off = m->QD; break;
         case PT_WV: rows = m->KVD; cols = c.hidden; row_off = m->QD + m->KVD; break;
         case PT_WO: rows = c.hidden; cols = m->QD; break;
-        case PT_WG: rows = c.ffn; cols = c.hidden; il = 1; break;
-        case PT_WU: rows = c.ffn; cols = c.hidden; il = 2; break;
-        default: rows = c.hidden; cols = c.ffn; break;
+        case PT_WG: rows = c.ffn; cols = c.hidden; il = 1; row_off = expert * 2 * c.ffn; break;
+        case PT_WU: rows = c.ffn; cols = c.hidden; il = 2; row_off = expert * 2 * c.ffn; break;
+        default: rows = c.hidden; cols = c.ffn; dst_cols = m->Ftot; col_off = expert * c.ffn; break;
     }
+    if (!dst_cols) dst_cols = cols;
     size_t n = (size_t)rows * cols;
     int grid = (int)std::min<size_t>((n + 255) / 256, 148 * 8);
-    if (m->esz == 2) k_pack<<<grid, 256, 0, st>>>((const __nv_bfloat16*)src, (__nv_bfloat16*)dst, rows, cols, row_off, il);
-    else k_pack<<<grid, 256, 0, st>>>((const float*)src, (float*)dst, rows, cols, row_off, il);
+    if (m->esz == 2) k_pack<<<grid, 256, 0, st>>>((const __nv_bfloat16*)src, (__nv_bfloat16*)dst, rows, cols, row_off, il, dst_cols, col_off);
+    else k_pack<<<grid, 256, 0, st>>>((const float*)src, (float*)dst, rows, cols, row_off, il, dst_cols, col_off);
     LAUNCH_COUNT();
 }
 

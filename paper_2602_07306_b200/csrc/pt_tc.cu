@@ -89,6 +89,64 @@ __global__ void k_l2_prefetch(const char* __restrict__ base, size_t bytes) {
         asm volatile("prefetch.global.L2 [%0];" ::"l"(base + i * 128));
 }
 
+// PT-MoE routing weights of one layer: one warp per (token, track).  The normalised stream is the gain-scaled bf16
+// copy times 1/rms (the operand the gate/up GEMM sees); the router itself is fp32.  logits[e] = c . Wr[e]; the top_k
+// largest logits (the lower index wins a tie) get softmax weights among themselves, every other expert 0.
+__global__ void k_moe_route(const __nv_bfloat16* __restrict__ hb, const float* __restrict__ ssq, int tiles, float eps,
+                            const float* __restrict__ wr, float* __restrict__ gates, int M, int H, int E, int top_k) {
+    grid_dep_wait();
+    grid_dep_launch();
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    const int t = blockIdx.y;
+    if (warp >= M) return;
+    const size_t row = (size_t)t * M + warp;
+    float ss = 0.f;
+    for (int i = lane; i < tiles; i += 32) ss += ssq[row * tiles + i];
+#pragma unroll
+    for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    const float rinv = 1.0f / sqrtf(ss / (float)H + eps);
+    float logit[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) logit[e] = 0.f;
+    const __nv_bfloat16* hr = hb + row * H;
+    const float* w = wr + (size_t)t * E * H;
+    for (int c = lane * 2; c < H; c += 64) {
+        const float2 hv = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(hr + c));
+#pragma unroll
+        for (int e = 0; e < 16; ++e)
+            if (e < E) {
+                const float2 wv = *reinterpret_cast<const float2*>(w + (size_t)e * H + c);
+                logit[e] = fmaf(hv.x, wv.x, fmaf(hv.y, wv.y, logit[e]));
+            }
+    }
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+#pragma unroll
+        for (int o = 16; o; o >>= 1) logit[e] += __shfl_xor_sync(0xffffffffu, logit[e], o);
+        logit[e] *= rinv;
+    }
+    // every lane holds all logits: choose top_k (lowest index among equals first), softmax over the chosen
+    unsigned chosen = 0;
+    float top = 0.f;
+    for (int k = 0; k < top_k; ++k) {
+        int best = -1;
+        float bv = 0.f;
+#pragma unroll
+        for (int e = 0; e < 16; ++e)
+            if (e < E && !((chosen >> e) & 1u) && (best < 0 || logit[e] > bv)) { best = e; bv = logit[e]; }
+        chosen |= 1u << best;
+        if (k == 0) top = bv;
+    }
+    float sum = 0.f, wgt[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) { wgt[e] = ((chosen >> e) & 1u) ? __expf(logit[e] - top) : 0.f; sum += wgt[e]; }
+    const float inv = 1.0f / sum;
+    float mine = 0.f;
+#pragma unroll
+    for (int e = 0; e < 16; ++e) mine = lane == e ? wgt[e] * inv : mine;
+    if (lane < E) gates[row * E + lane] = mine;
+}
+
 inline int kps_index(int kps) { return kps == 4 ? 2 : (kps == 2 ? 1 : 0); }
 
 }  // namespace
@@ -108,7 +166,7 @@ pt_status tc_build_weight_maps(pt_model* m) {
                 if (bn * kps > 256) continue;
                 const void* base[4] = {wqkv + (size_t)l * m->wqkv_layer(), wo + (size_t)l * m->wo_layer(),
                                        wgu + (size_t)l * m->wgu_layer(), wd + (size_t)l * m->wd_layer()};
-                const int64_t kk[4] = {c.hidden, m->QD, c.hidden, c.ffn}, nn[4] = {m->Nqkv, c.hidden, 2 * c.ffn, c.hidden};
+                const int64_t kk[4] = {c.hidden, m->QD, c.hidden, m->Ftot}, nn[4] = {m->Nqkv, c.hidden, 2 * m->Ftot, c.hidden};
                 for (int i = 0; i < 4; ++i) {
                     if (kps > 1 && (kk[i] % 64 || (kk[i] / 64) % kps)) continue;
                     pt_status s = make_w_map(&v[l].m[i][b][kp], base[i], kk[i], nn[i], c.T, bn, kps);
@@ -123,7 +181,7 @@ pt_status tc_forward(Call& k) {
     pt_model* m = k.m;
     pt_kv_cache* c = k.c;
     const pt_config& g = m->cfg;
-    const int T = g.T, M = k.M, H = g.hidden, F = g.ffn;
+    const int T = g.T, M = k.M, H = g.hidden, F = m->Ftot;        // with experts: all of a track's experts side by side
     const size_t MH = (size_t)M * H;
     cudaStream_t st = k.st;
     Work& w = k.w;
@@ -210,9 +268,16 @@ pt_status tc_forward(Call& k) {
             ssq_tstride = (size_t)M * tiles;
         }
         tap_copy(k, l, 0, w.hT, MH);
-        {   // gate/up + SwiGLU
+        if (m->E) {   // PT-MoE: the routing weights of this layer, from the operand and statistics the out-projection just wrote
+            ProfScope ps(m, st, 6);
+            launch_dependent(k_moe_route, dim3((M * 32 + 255) / 256, T), dim3(256), (size_t)0, st, (const __nv_bfloat16*)hb, (const float*)w.ssq, tiles,
+                             g.rms_eps, m->router(l), w.gates, M, H, m->E, g.top_k);
+            g_launches.fetch_add(1, std::memory_order_relaxed);
+        }
+        {   // gate/up + SwiGLU (PT-MoE: every expert's, each column block weighted by its expert's routing weight)
             GemmP p = base;
             p.N = 2 * F; p.K = H;
+            p.gates = w.gates; p.n_experts = m->E; p.expert_cols = 2 * g.ffn;
             p.ssq_in = w.ssq; p.ssq_in_tstride = ssq_tstride; p.ssq_tiles = tiles;
             p.z_out = z;
             int bn = gemm_bn(p.N, M, T, EPI_SWIGLU);

@@ -38,6 +38,8 @@ struct GemmP {
     int nq, nkv, dh, ps;
     // EPI_SWIGLU
     __nv_bfloat16* z_out;   // [T][M][N/2]
+    const float* gates;     // PT-MoE: [T][M][n_experts] weights; accumulator columns [e * expert_cols, (e + 1) * expert_cols) belong to expert e
+    int n_experts, expert_cols;
     // EPI_RESID
     const float* h_in; size_t h_in_tstride; int n_sum; float scale;
     float* h_out; size_t h_out_tstride;

@@ -224,13 +224,18 @@ __device__ __forceinline__ bool epi_swiglu(const GemmP& p, uint32_t taddr, int t
 #pragma unroll
         for (int g4 = 0; g4 < 4; ++g4) tc_ld16(taddr + c + g4 * 16, gu + g4 * 16);
         tc_wait_ld();
+        // PT-MoE: the 64 columns of a unit belong to one expert (its block is a multiple of 32 columns wide and starts on one)
+        float wgt = 1.0f;
+        if (p.gates && row_ok) wgt = p.gates[((size_t)t * p.M + row) * p.n_experts + (n0 + c) / p.expert_cols];
 #pragma unroll
         for (int g2 = 0; g2 < 2; ++g2) {
             float z[16];
+            if (p.gates && g2 == 1 && row_ok && ((n0 + c + 32) / p.expert_cols) != ((n0 + c) / p.expert_cols) && n0 + c + 32 < p.N)
+                wgt = p.gates[((size_t)t * p.M + row) * p.n_experts + (n0 + c + 32) / p.expert_cols];
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
                 const float gv = gu[g2 * 32 + i] * rinv, uv = gu[g2 * 32 + 16 + i] * rinv;
-                z[i] = __fdividef(gv, 1.0f + __expf(-gv)) * uv;
+                z[i] = __fdividef(gv, 1.0f + __expf(-gv)) * uv * wgt;
             }
             const int zc = ((n0 + c) >> 1) + g2 * 16;      // first output column of this group
             if (row_ok && zc < F) store16_bf16(p.z_out + ((size_t)t * p.M + row) * F + zc, z);

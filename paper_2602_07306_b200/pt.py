@@ -21,7 +21,7 @@ STATUS = {0: "PT_OK", 1: "PT_ERR_INVALID_ARG", 2: "PT_ERR_BAD_CONFIG", 3: "PT_ER
           8: "PT_ERR_DEVICE_BOUNDS", 9: "PT_ERR_DEVICE_TIMEOUT", 10: "PT_ERR_STATE"}
 PT_F32, PT_BF16 = 0, 1
 PT_KV_MODEL, PT_KV_E4M3 = 0, 1
-KIND = {"wq": 0, "wk": 1, "wv": 2, "wo": 3, "wg": 4, "wu": 5, "wd": 6, "g1": 7, "g2": 8}
+KIND = {"wq": 0, "wk": 1, "wv": 2, "wo": 3, "wg": 4, "wu": 5, "wd": 6, "g1": 7, "g2": 8, "wr": 9}
 
 
 class PtError(RuntimeError):
@@ -34,7 +34,8 @@ class pt_config(C.Structure):
     _fields_ = [("T", C.c_int32), ("D", C.c_int32), ("L", C.c_int32), ("hidden", C.c_int32),
                 ("heads", C.c_int32), ("kv_heads", C.c_int32), ("ffn", C.c_int32),
                 ("rope_base", C.c_float), ("rms_eps", C.c_float), ("dtype", C.c_int32),
-                ("sync_op", C.c_int32), ("max_pos", C.c_int32), ("flags", C.c_int32)]
+                ("sync_op", C.c_int32), ("max_pos", C.c_int32), ("flags", C.c_int32),
+                ("experts", C.c_int32), ("top_k", C.c_int32)]
 
 
 _P, _I32, _I64, _SZ = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
@@ -44,6 +45,7 @@ _PROTOS = {
     "pt_model_weight_bytes": (_I32, [_P, C.POINTER(_SZ)]),
     "pt_model_bind_weights": (_I32, [_P, _P, _SZ]),
     "pt_model_set_weight": (_I32, [_P, _I32, _I32, _I32, _P, _P]),
+    "pt_model_set_expert_weight": (_I32, [_P, _I32, _I32, _I32, _I32, _P, _P]),
     "pt_sync_count": (_I32, [_P]),
     "pt_model_set_track_group": (_I32, [_P, _I32, _P, _P]),
     "pt_kv_cache_bytes": (_I32, [_P, _I32, _I32, C.POINTER(_SZ)]),
@@ -120,13 +122,13 @@ class Model:
     """A PT model with its packed weights on one CUDA device (torch owns the memory)."""
 
     def __init__(self, *, T, D, L, hidden, heads, kv_heads, ffn, dtype="bf16", rope_base=10000.0,
-                 rms_eps=1e-6, sync_op="sum", max_pos=4096, simt=False, flags=0, device="cuda:0"):
+                 rms_eps=1e-6, sync_op="sum", max_pos=4096, simt=False, flags=0, experts=0, top_k=0, device="cuda:0"):
         import torch
         self.torch = torch
         self.device = torch.device(device)
         self.cfg = pt_config(T, D, L, hidden, heads, kv_heads, ffn, rope_base, rms_eps,
                              PT_BF16 if dtype == "bf16" else PT_F32, 1 if sync_op == "mean" else 0,
-                             max_pos, (1 if simt else 0) | int(flags))
+                             max_pos, (1 if simt else 0) | int(flags), experts, top_k)
         self.dtype = dtype
         self.tdtype = torch.bfloat16 if dtype == "bf16" else torch.float32
         self.h = _P()
@@ -162,10 +164,14 @@ class Model:
         torch = self.torch
         if isinstance(w, np.ndarray):
             w = torch.from_numpy(np.ascontiguousarray(w))
-        want = torch.float32 if kind in ("g1", "g2") else self.tdtype
+        want = torch.float32 if kind in ("g1", "g2", "wr") else self.tdtype
         w = w.to(device=self.device, dtype=want).contiguous()
         with torch.cuda.device(self.device):
-            check(lib().pt_model_set_weight(self.h, t, l, KIND[kind], w.data_ptr(), self._stream()))
+            if self.cfg.experts and kind in ("wg", "wu", "wd"):       # PT-MoE: [experts, ...], one call per expert
+                for e in range(self.cfg.experts):
+                    check(lib().pt_model_set_expert_weight(self.h, t, l, e, KIND[kind], w[e].data_ptr(), self._stream()))
+            else:
+                check(lib().pt_model_set_weight(self.h, t, l, KIND[kind], w.data_ptr(), self._stream()))
             torch.cuda.current_stream().synchronize()      # w may be freed after return
 
     def load(self, source) -> None:
@@ -188,8 +194,15 @@ class Model:
             for l in range(c.L):
                 for t in range(c.T):
                     for k, shp in shapes.items():
-                        w = (torch.randn(shp, generator=g, device=self.device, dtype=torch.float32) * std).to(self.tdtype)
-                        check(lib().pt_model_set_weight(self.h, t, l, KIND[k], w.data_ptr(), self._stream()))
+                        for e in range(c.experts if c.experts and k in ("wg", "wu", "wd") else 1):
+                            w = (torch.randn(shp, generator=g, device=self.device, dtype=torch.float32) * std).to(self.tdtype)
+                            if c.experts and k in ("wg", "wu", "wd"):
+                                check(lib().pt_model_set_expert_weight(self.h, t, l, e, KIND[k], w.data_ptr(), self._stream()))
+                            else:
+                                check(lib().pt_model_set_weight(self.h, t, l, KIND[k], w.data_ptr(), self._stream()))
+                    if c.experts:
+                        wr = torch.randn((c.experts, c.hidden), generator=g, device=self.device, dtype=torch.float32) * std
+                        check(lib().pt_model_set_weight(self.h, t, l, KIND["wr"], wr.data_ptr(), self._stream()))
                     for k in ("g1", "g2"):
                         check(lib().pt_model_set_weight(self.h, t, l, KIND[k], ones.data_ptr(), self._stream()))
             torch.cuda.synchronize()

@@ -15,7 +15,7 @@ def make_model(wl, ws, sync_op="sum", max_pos=4096, simt=False, flags=0):
     from paper_2602_07306_b200 import pt
     m = pt.Model(T=wl.T, D=wl.D, L=wl.L, hidden=wl.hidden, heads=wl.heads, kv_heads=wl.kv_heads, ffn=wl.ffn,
                  dtype=wl.dtype, rope_base=wl.rope_base, rms_eps=wl.rms_eps, sync_op=sync_op,
-                 max_pos=max_pos, simt=simt, flags=flags)
+                 max_pos=max_pos, simt=simt, flags=flags, experts=wl.experts, top_k=wl.top_k)
     m.load(ws)
     return m
 

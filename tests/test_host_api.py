@@ -24,7 +24,7 @@ def lib():
 
 def make(lib, **kw):
     base = dict(T=2, D=2, L=4, hidden=128, heads=4, kv_heads=4, ffn=512, rope_base=1e4, rms_eps=1e-6,
-                dtype=pt.PT_F32, sync_op=0, max_pos=256, flags=0)
+                dtype=pt.PT_F32, sync_op=0, max_pos=256, flags=0, experts=0, top_k=0)
     base.update(kw)
     cfg = pt.pt_config(**base)
     h = C.c_void_p()
@@ -53,6 +53,13 @@ def test_config_validation(lib):
     assert make(lib, hidden=96, heads=4)[0] == 3  # head_dim 24 unsupported
     assert make(lib, ffn=100)[0] == 3
     assert lib.pt_model_create(None, None) == 1
+    # PT-MoE: top_k in [1, experts]; bf16 models on the tensor-core path only; at most 16 experts
+    assert make(lib, dtype=pt.PT_BF16, experts=4, top_k=2)[0] == pt.PT_OK
+    assert make(lib, dtype=pt.PT_BF16, experts=4, top_k=5)[0] == 2
+    assert make(lib, dtype=pt.PT_BF16, experts=4, top_k=0)[0] == 2
+    assert make(lib, dtype=pt.PT_BF16, experts=0, top_k=1)[0] == 2
+    assert make(lib, dtype=pt.PT_BF16, experts=17, top_k=1)[0] == 3
+    assert make(lib, dtype=pt.PT_F32, experts=2, top_k=1)[0] == 3
 
 
 def test_sync_count_is_L_over_D(lib):
