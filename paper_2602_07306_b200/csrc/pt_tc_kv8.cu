@@ -5,7 +5,8 @@
 //                      code * scale (exact in bf16: a code has four significant bits) into the bf16 copy the
 //                      prefill attention kernel reads
 //   k_kv_dequant_ctx   the keys a prefill call's sequences held before the call, code * scale into that copy
-//   k_decode_attn_e4m3 split-KV decode attention straight from the codes (see its own comment)
+//   k_decode_attn_e4m3 split-KV decode attention from the codes on mma.sync (config flag bit 2; the default kernel is the
+//                      tcgen05 one in pt_tc_kv8_dec.cu)
 #include <cuda_fp8.h>
 
 #include "pt_tc.h"
@@ -114,10 +115,8 @@ __global__ void k_kv_dequant_ctx(const CtxP p) {
 // ---- decode attention straight from the codes -------------------------------------------------------
 // Same work split as the bf16 kernel: a CTA = one (track, sequence, KV head, key range), each of its 4 warps
 // streams its own 16-token groups through a private ring, the G query heads of the KV head are the rows of an
-// mma.sync m16n8k16 tile.  An SM starts a TMA copy only every 80 cycles or so whatever its size (with a K box, a V
-// box and two 64-byte bulk copies of scales per group this kernel ran at 3.7 TB/s, the rate of four copies per
-// 4.2 KB), so a group is ONE copy: a 5-D box that takes the K block and, nkv blocks further, the V block of the
-// page in one go (element stride nkv in the (K|V, head) dimension); the 32 scales come as 32 four-byte cp.async
+// mma.sync m16n8k16 tile.  A group arrives as ONE copy: a 5-D box that takes the K block and, nkv blocks further, the V
+// block of the page in one go (element stride nkv in the (K|V, head) dimension); the 32 scales come as 32 four-byte cp.async
 // copies, one per lane.  Codes become f16 (exact) on their way into the MMA's B fragments:
 //   scores  the contraction indices kappa {2q, 2q+1, 2q+8, 2q+9} (q = lane % 4) of k-steps 2kk and 2kk+1 are mapped
 //           to head_dim 32 kk + 8q + {0..3} and + {4..7}, so a thread's four B registers of two k-steps are one

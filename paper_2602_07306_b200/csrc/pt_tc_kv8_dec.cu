@@ -17,7 +17,7 @@
 // and one named barrier per tile.  The reference maximum is raised only when it grows by more than 2^8 (the
 // accumulator is then rescaled in tensor memory), so rescales are rare.
 // Roles: warp 0 streams K and V tiles page by page with TMA (one 16 x 128-byte box per page and K|V) through
-// three-stage rings; warp 1 issues the MMAs (the scores of tile j+2 right behind P V of tile j: S^T is double-buffered in
+// two-stage rings (so that three CTAs fit an SM: the kernel is bound by the latency of its copies, more CTAs hide it); warp 1 issues the MMAs (the scores of tile j+2 right behind P V of tile j: S^T is double-buffered in
 // tensor memory, P in shared memory); warps 2-5 are the softmax threads.  Every mbarrier wait is bounded; the named
 // barrier is executed exactly once per tile and twice at the end by every softmax warp whatever happened before.
 #include <cuda_fp8.h>
