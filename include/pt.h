@@ -99,9 +99,12 @@ typedef struct {
                            inside each track) and defines nothing else; this library's definition: router
                            logits = rmsnorm(h; g2) Wr^T, the top_k largest logits (the lower index wins a
                            tie) get softmax weights among themselves, the layer's output is the weighted
-                           sum of the chosen experts' outputs.  Every expert is evaluated for every
-                           token and weighted afterwards (unchosen experts by zero): the result is the
-                           mixture's, the routing sparsity is not exploited                         */
+                           sum of the chosen experts' outputs.  Prefill calls of 512 rows or more copy
+                           every token's row to the row groups of the experts it chose and evaluate only
+                           those (a grouped GEMM over (track, expert)); smaller calls and decode steps
+                           evaluate every expert for every token and weight afterwards (unchosen experts by
+                           zero) - the same result, and a decode batch streams every expert's weights
+                           either way                                                                */
     int32_t top_k;      /* experts chosen per token, 1 .. experts (0 with experts == 0)              */
 } pt_config;
 

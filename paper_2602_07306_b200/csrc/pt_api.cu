@@ -57,12 +57,23 @@ static size_t carve(const pt_model* m, int64_t M, int B, int maxp, bool fp8, int
     void* gu = m->tc ? nullptr : take((size_t)c.T * M * 2 * m->Ftot * m->esz);
     void* z = take((size_t)c.T * M * m->Ftot * m->esz);
     float* gates = m->E ? (float*)take((size_t)c.T * M * m->E * 4) : nullptr;
+    MoeWork mw{};
+    if (m->E && moe_sparse_ok(m, (int)std::min<int64_t>(M, 1 << 30), false)) {
+        const size_t R = (size_t)moe_rows(m, M);
+        mw.pos = (int32_t*)take((size_t)c.T * M * m->E * 4);
+        mw.tile_expert = (int32_t*)take((size_t)c.T * (R / 128) * 4);
+        mw.xperm = (__nv_bfloat16*)take((size_t)c.T * R * c.hidden * 2);
+        mw.ssq_perm = (float*)take((size_t)c.T * R * ((c.hidden + kSsqTile - 1) / kSsqTile) * 4);
+        mw.gperm = (float*)take((size_t)c.T * R * 4);
+        mw.zperm = (__nv_bfloat16*)take((size_t)c.T * R * c.ffn * 2);
+        mw.yperm = (float*)take((size_t)c.T * R * c.hidden * 4);
+    }
     float* ssq = m->tc ? (float*)take((size_t)c.T * M * ((c.hidden + kSsqTile - 1) / kSsqTile) * 4) : nullptr;
     float* part = m->tc ? (float*)take((size_t)c.T * B * kMaxSplits * c.heads * (m->dh + 2) * 4) : nullptr;
     void* kv_stage = fp8 ? take((size_t)c.T * 2 * m->KVD * M * 2) : nullptr;
     void* attn_kv = fp8 && ctx_keys > 0 ? take((size_t)c.T * 2 * m->KVD * (size_t)ctx_keys * 2) : nullptr;
     if (w) {
-        w->kv_stage = kv_stage; w->attn_kv = attn_kv; w->gates = gates;
+        w->kv_stage = kv_stage; w->attn_kv = attn_kv; w->gates = gates; w->moe = mw;
         w->hT = hT; w->hS = hS; w->a = a; w->qkv = qkv; w->o = o; w->gu = gu; w->z = z;
         w->ssq = ssq; w->part = part; w->total = off;
         (void)meta;

@@ -130,6 +130,18 @@ struct Meta {
     int32_t maxp_attn, attn_pages, max_start;
 };
 
+// PT-MoE with permuted tokens: R = moe_rows() rows per track, every (token, chosen expert) one row, experts in runs of
+// 128-row tiles.
+struct MoeWork {
+    int32_t* pos;            // [T][M][E] row of (token, expert), -1 where the token did not choose the expert
+    int32_t* tile_expert;    // [T][R / 128]
+    __nv_bfloat16* xperm;    // [T][R][H] operand rows
+    float* ssq_perm;         // [T][R][H / kSsqTile]
+    float* gperm;            // [T][R] routing weight of the row
+    __nv_bfloat16* zperm;    // [T][R][ffn]
+    float* yperm;            // [T][R][H]
+};
+
 // Workspace carve-up for one call.
 struct Work {
     Meta meta;
@@ -143,6 +155,7 @@ struct Work {
     float* ssq;     // [T][M][H/kSsqTile] partial sums of squares (tc)
     float* part;    // decode split-KV partials
     void* kv_stage; // E4M3 caches: [T][K|V][kv_head][M][dh] bf16, this call's K and V as projected
+    MoeWork moe;    // PT-MoE, permuted-token path (prefill calls of 512 rows or more)
     float* gates;   // PT-MoE: [T][M][E] routing weights of the current layer (0 for the experts a token did not choose)
     void* attn_kv;  // E4M3 caches, prefill: [T][page][K|V][kv_head][16][dh] bf16 copy of code * scale of every key attended to
     size_t total;
@@ -189,6 +202,10 @@ void plan_decode_splits(const int32_t* lens, int B, int ps, int64_t units, int32
 // pt_simt.cu
 pt_status simt_forward(Call& k);
 void launch_pack(const pt_model* m, int kind, const void* src, void* dst_matrix_base, cudaStream_t st, int expert = 0);
+
+// pt_tc_moe.cu
+bool moe_sparse_ok(const pt_model* m, int M, bool decode);
+int64_t moe_rows(const pt_model* m, int64_t M);
 
 // pt_tc.cu (bf16 tensor-core path)
 pt_status tc_build_weight_maps(pt_model* m);

@@ -274,6 +274,16 @@ pt_status tc_forward(Call& k) {
                              g.rms_eps, m->router(l), w.gates, M, H, m->E, g.top_k);
             g_launches.fetch_add(1, std::memory_order_relaxed);
         }
+        if (moe_sparse_ok(m, M, k.decode)) {   // PT-MoE on permuted tokens: only the chosen experts are evaluated
+            const bool sync = (l + 1) % g.D == 0, last = l + 1 == g.L;
+            float* ho = last ? k.out : w.hS;
+            const float sync_scale = g.sync_op ? 1.0f / (float)T : 1.0f;
+            if ((s = moe_sparse_ffn(k, l, sync, last, sync_scale, w.hT, MH, sync ? ho : w.hT, sync ? 0 : MH)) != PT_OK) return s;
+            if (sync) { ssq_tstride = 0; hin = ho; hin_stride = 0; }
+            else { ssq_tstride = (size_t)M * tiles; hin = w.hT; hin_stride = MH; }
+            tap_copy(k, l, 1, hin, hin_stride);
+            continue;
+        }
         {   // gate/up + SwiGLU (PT-MoE: every expert's, each column block weighted by its expert's routing weight)
             GemmP p = base;
             p.N = 2 * F; p.K = H;

@@ -23,6 +23,9 @@ struct GemmP {
     uint32_t w_kb_bytes;    // shared-memory bytes one k-block of W takes
     int stages;             // ring depth
     int w_static;           // W is written by no kernel of the stream: its first tiles may be fetched before grid_dep_wait()
+    // grouped rows (PT-MoE with permuted tokens; one-CTA kernel with kps = 1 only): row tile mt of track t multiplies with
+    // expert tile_expert[t * tiles_m + mt]'s weights, found w_row_per_expert rows / w_k_per_expert columns further in W
+    const int32_t* tile_expert; int w_row_per_expert, w_k_per_expert;
     int* status;
     // RMSNorm applied as a per-row scale: rinv = rsqrt(sum(ssq_in[row][:]) / K + eps)
     const float* ssq_in; size_t ssq_in_tstride; int ssq_tiles; float eps;
@@ -139,6 +142,11 @@ pt_status launch_flash_prefill_tc(const AttnP& p, int T, int dh, cudaStream_t st
 // pt_tc_attn.cu
 pt_status launch_flash_prefill(Call& k, const __nv_bfloat16* q, const __nv_bfloat16* pool_l, __nv_bfloat16* o);
 pt_status launch_decode_attn(Call& k, const __nv_bfloat16* q, const __nv_bfloat16* pool_l, __nv_bfloat16* o);
+
+// pt_tc_moe.cu: the feed-forward of a PT-MoE layer with permuted tokens, from the stream after the attention residual
+// (h_in) to what the dense path's down GEMM leaves (h_out, the next operand and statistics, the track-sync when `sync`)
+pt_status moe_sparse_ffn(Call& k, int l, bool sync, bool last, float sync_scale, const float* h_in, size_t h_in_tstride,
+                         float* h_out, size_t h_out_tstride);
 
 // merges the key ranges of a split decode attention (pt_tc_attn.cu)
 pt_status launch_decode_combine(const AttnP& p, int T, int dh, cudaStream_t st);

@@ -531,6 +531,10 @@ gemm_tc(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensor
                 int nt, mt, t;
                 tile_coords(p, tile, nt, mt, t);
                 if (kps == 1) {
+                    // grouped rows: this row tile's expert shifts the W coordinates (the table is written by a kernel of
+                    // the stream, so such launches never prefetch W before the wait: npre is 0)
+                    const int ex = p.tile_expert ? p.tile_expert[t * p.tiles_m + mt] : 0;
+                    const int w_row = nt * BN + ex * p.w_row_per_expert, w_k = ex * p.w_k_per_expert;
                     for (int kb = 0; kb < kblocks; ++kb) {
                         const int tt = p.kt > 1 ? kb / kpb : t;
                         const int k0 = (p.kt > 1 ? kb % kpb : kb) * BK;
@@ -541,7 +545,7 @@ gemm_tc(const __grid_constant__ CUtensorMap ta, const __grid_constant__ CUtensor
                             if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_GEMM_EMPTY_WAIT); *abort_flag = 1; break; }
                             mbar_expect_tx(&full[s], stage_tx);
                             tma_load_3d(sa, &ta, &full[s], k0, mt * BM, tt);
-                            tma_load_3d(sa + a_bytes, &tb, &full[s], k0, nt * BN, tt);
+                            tma_load_3d(sa + a_bytes, &tb, &full[s], k0 + w_k, w_row, tt);
                         }
                         if (++s == stages) { s = 0; ph ^= 1; }
                     }

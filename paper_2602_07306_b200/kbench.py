@@ -93,7 +93,8 @@ def layer(a):
     --layers 2 the track block is two layers deep, so the first layer's down GEMM is the plain one (gemm_down)."""
     from paper_2602_07306_b200 import inputs as I
     dev = torch.device("cuda:0")
-    m = pt.Model(T=a.T, D=a.layers, L=a.layers, hidden=a.H, heads=a.nq, kv_heads=a.nkv, ffn=a.F, dtype="bf16", max_pos=a.S, device=dev)
+    m = pt.Model(T=a.T, D=a.layers, L=a.layers, hidden=a.H, heads=a.nq, kv_heads=a.nkv, ffn=a.F, dtype="bf16", max_pos=a.S,
+                 experts=a.experts, top_k=a.top_k, device=dev)
     m.init_random(0)
     cache = m.new_cache(a.B * (-(-a.S // a.ps)), a.ps)
     g = torch.Generator(device=dev).manual_seed(0)
@@ -115,9 +116,10 @@ def layer(a):
     prof = m.profile_read()
     assert m.device_status() == (0, 0)
     tok = a.B * a.S
+    kx = max(a.top_k, 1)          # PT-MoE: a token's feed-forward flops are those of its top_k experts
     fl = {"gemm_qkv": 2.0 * a.T * tok * a.H * (a.nq + 2 * a.nkv) * (a.H // a.nq), "gemm_out": 2.0 * a.T * tok * a.H * a.H,
-          "gemm_gate_up": 4.0 * a.T * tok * a.H * a.F, "gemm_down_sync": 2.0 * a.T * tok * a.H * a.F,
-          "gemm_down": 2.0 * a.T * tok * a.H * a.F}
+          "gemm_gate_up": 4.0 * a.T * tok * a.H * a.F * kx, "gemm_down_sync": 2.0 * a.T * tok * a.H * a.F * kx,
+          "gemm_down": 2.0 * a.T * tok * a.H * a.F * kx}
     res = {k: {"ms": v[0] / max(v[1], 1), "TFLOPs": fl[k] / (v[0] / max(v[1], 1)) / 1e9 if k in fl and v[1] else None}
            for k, v in prof.items() if v[1]}
     print(json.dumps({"kernel": "layer", "per_launch": res, "args": vars(a)}))
@@ -242,7 +244,7 @@ def main():
     for k, v in dict(T=8, B=8, S=4096, start=0, nq=8, nkv=8, dh=128, ps=16, impl=0, iters=10, warmup=3).items():
         pf.add_argument("--" + k, type=int, default=v)
     ly = sub.add_parser("layer")
-    for k, v in dict(T=8, B=2, S=4096, H=1024, nq=8, nkv=8, F=2816, ps=16, layers=1, iters=3, warmup=1).items():
+    for k, v in dict(T=8, B=2, S=4096, H=1024, nq=8, nkv=8, F=2816, ps=16, layers=1, experts=0, top_k=0, iters=3, warmup=1).items():
         ly.add_argument("--" + k, type=int, default=v)
     gn = sub.add_parser("generate")
     for k, v in dict(B=1, S=1024, new=64, vocab=32000, depth=0, iters=3, warmup=1).items():

@@ -142,3 +142,57 @@ def test_moe_with_one_expert_is_the_dense_model_bit_for_bit():
         m.close()
     np.testing.assert_array_equal(outs[0], outs[1])
 
+
+
+# ---- the permuted-token path (prefill calls of 512 rows or more evaluate only the chosen experts)
+
+def test_moe_sparse_all_experts_two_layers_with_a_sync():
+    wl = _moe_wl("sparse-all3", 3, 3, T=2, L=2, D=2, H=256, nq=4, nkv=2, F=176)
+    ws = I.WeightSource(wl, gain_jitter=0.1, router_std=0.05)
+    import torch
+    cfg = Hp.oracle_cfg(wl)
+    B, S = 2, 300                                                  # 600 rows: the permuted path
+    x = I.prefill_inputs(wl, batch=B, seq=S)
+    taps = {}
+    ref = O.pt_prefill(cfg, ws, x, O.PagedKVCache(cfg, 40, 16), [0, 1], taps)
+    model = Hp.make_model(wl, ws, max_pos=320)
+    tap = model.set_tap(-1, B * S)
+    got = model.prefill(model.new_cache(40, 16), Hp.to_dev(model, x), [0, 1])
+    torch.cuda.synchronize()
+    assert model.device_status() == (0, 0)
+    Hp.assert_close(got.cpu().numpy(), ref, wl.dtype, "permuted-token path, all experts", log="PT-MoE permuted tokens, all 3 experts, 600 rows: prefill")
+    _check_taps(wl, tap.cpu().numpy(), taps, B, S)
+    model.set_tap(None)
+    model.close()
+
+
+def test_moe_sparse_top2_of_4_row_by_row_and_against_the_dense_masked_path():
+    import torch
+    wl = _moe_wl("sparse-top2of4", 4, 2, T=2, L=1, D=1, seed=2)
+    ws = I.WeightSource(wl, gain_jitter=0.1, router_std=0.3)
+    cfg = Hp.oracle_cfg(wl)
+    B, S = 2, 320
+    x = I.prefill_inputs(wl, batch=B, seq=S)
+    taps = {}
+    ref = O.pt_prefill(cfg, ws, x, O.PagedKVCache(cfg, 40, 16), [0, 1], taps)
+    model = Hp.make_model(wl, ws, max_pos=320)
+    from paper_2602_07306_b200 import pt
+    xd = Hp.to_dev(model, x)
+    n0 = pt.lib().pt_launch_count()
+    sparse = model.prefill(model.new_cache(40, 16), xd, [0, 1]).cpu().numpy()           # 640 rows at once
+    # input prep + [QKV, attention, out-projection, router, plan, dispatch, gate/up, down, combine]
+    assert pt.lib().pt_launch_count() - n0 == 1 + 9
+    cache = model.new_cache(40, 16)                                                     # 2 x 160 rows per call: every expert for every token
+    dense = np.concatenate([model.prefill(cache, xd[:, :, :160].contiguous(), [0, 1]).cpu().numpy(),
+                            model.prefill(cache, xd[:, :, 160:].contiguous(), [0, 1]).cpu().numpy()], axis=1)
+    torch.cuda.synchronize()
+    assert model.device_status() == (0, 0)
+    model.close()
+    # one layer: both paths route from the same operand, so they take the same decisions; they differ in summation order only
+    mx, mean = Hp.rel_errs(sparse, dense)
+    Hp.record("PT-MoE top 2 of 4, one layer, 640 rows: permuted-token path against the dense-masked path", mx, mean, 1e-3, 1e-4)
+    assert mx <= 1e-3 and mean <= 1e-4
+    safe = token_margins(taps, wl.top_k) > MARGIN
+    assert safe.mean() > 0.9
+    Hp.assert_close(sparse[safe], ref[safe], wl.dtype, "tokens with a clear routing decision",
+                    log=f"PT-MoE permuted tokens, top 2 of 4, one layer: {int(safe.sum())} of {safe.size} tokens with a routing margin above {MARGIN}")
