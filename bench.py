@@ -405,6 +405,9 @@ class _Cached:
         return self.w[(t, l)]
 
 
+_SAMPLE_WEIGHTS = {}          # the sample's weights are drawn once per process, outside every timed call
+
+
 def oracle_sample(wl, budget_s=20.0):
     """Time the CPU oracle, as it stands, on a bounded sample of the workload: the first track
     block (D of the L layers, all T tracks) on a few rows / a shorter prompt; tokens/s is scaled by
@@ -414,18 +417,26 @@ def oracle_sample(wl, budget_s=20.0):
     cores = len(os.sched_getaffinity(0))
     sub = dataclasses.replace(wl, L=wl.D)
     cfg = O.PTConfig(T=sub.T, D=sub.D, L=sub.L, hidden=sub.hidden, heads=sub.heads, kv_heads=sub.kv_heads, ffn=sub.ffn)
-    ws = _Cached(I.WeightSource(sub), sub.T, sub.L)
+    key = (sub.name, sub.T, sub.L, sub.hidden, sub.ffn, sub.seed)
+    if key not in _SAMPLE_WEIGHTS:
+        _SAMPLE_WEIGHTS[key] = _Cached(I.WeightSource(sub), sub.T, sub.L)
+    ws = _SAMPLE_WEIGHTS[key]
     scale = wl.D / wl.L
     if wl.mode == "decode":
         rows = 2
         lens = I.kv_lengths(wl, batch=rows)
         pages = int(sum((int(n) + 1 + 15) // 16 for n in lens))
-        cache = O.PagedKVCache(cfg, pages, 16)
-        rng = np.random.default_rng(0)
-        for b in range(rows):                     # synthetic cache contents: timing does not depend on them
-            cache.reserve(b, int(lens[b]))
-            cache.length[b] = int(lens[b])
-        cache.pool[...] = rng.standard_normal(cache.pool.shape)
+        ckey = key + ("cache",)
+        if ckey not in _SAMPLE_WEIGHTS:               # the pre-filled cache too is built once, outside the timed calls
+            cache = O.PagedKVCache(cfg, pages, 16)
+            rng = np.random.default_rng(0)
+            for b in range(rows):                     # synthetic cache contents: timing does not depend on them
+                cache.reserve(b, int(lens[b]) + 1)
+            cache.pool[...] = rng.standard_normal(cache.pool.shape)
+            _SAMPLE_WEIGHTS[ckey] = cache
+        cache = _SAMPLE_WEIGHTS[ckey]
+        for b in range(rows):
+            cache.length[b] = int(lens[b])            # every timed step decodes at the same KV lengths
         x = I.decode_inputs(sub, batch=rows)
         t0 = time.perf_counter()
         O.pt_decode_step(cfg, ws, x, cache, list(range(rows)))
