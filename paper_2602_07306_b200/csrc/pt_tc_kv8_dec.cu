@@ -191,13 +191,16 @@ k_decode_attn_e4m3_tc(const __grid_constant__ CUtensorMap kvmap, const Dec8TcP p
     const uint32_t tmem_base = *tmem_slot;                    // S^T buffers at columns 0 and 16, O^T at column 32
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------------ TMA producer.  K and V advance on their own
+        // counters: a K tile is requested the moment its stage is free (two tiles before its scores are issued) and never
+        // queues behind the wait for a V stage, which frees a tile later.  One bounded polling loop serves both.
         bool bad_page = false;
-        for (int j = 0; j < n_tiles; ++j) {
-            const int s = j % kStages;
-            const uint32_t ph = (uint32_t)(j / kStages) & 1u;
+        int jk = 0, jv = 0;
+        WaitClock clock;
+        uint32_t idle = 0;
+        auto rows_of = [&](int j, int& ng) {                       // lane < ng: first vector of the lane's 16-key group of tile j
             const int key0 = kstart + j * 128;
-            const int ng = min(8, (key_end - key0 + 15) >> 4);    // 16-key groups of this tile that hold keys
+            ng = min(8, (key_end - key0 + 15) >> 4);
             int row_k = 0;
             if (lane < ng) {
                 const int key = key0 + lane * 16;
@@ -205,25 +208,45 @@ k_decode_attn_e4m3_tc(const __grid_constant__ CUtensorMap kvmap, const Dec8TcP p
                 if (page < 0 || page >= p.num_pages) { bad_page = true; page = 0; }
                 row_k = (page * 2 * p.nkv + kvh) * p.ps + key % p.ps;
             }
-            const uint32_t bytes = (uint32_t)ng * 16u * kDh;
-            if (!mbar_wait(&bars[B_KEMPTY + s], ph ^ 1u, abort_flag, true)) { if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_FLASH_KEMPTY); *abort_flag = 1; } break; }
-            if (lane == 0) mbar_expect_tx(&bars[B_KFULL + s], bytes);
-            __syncwarp();
-            if (lane < ng) tma_load_3d(smem_u32(sk + s * kTile + lane * 2048), &kvmap, &bars[B_KFULL + s], 0, row_k, t);
-            if (!mbar_wait(&bars[B_VEMPTY + s], ph ^ 1u, abort_flag, true)) { if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_FLASH_VEMPTY); *abort_flag = 1; } break; }
-            const bool partial = key0 + 128 > key_end;             // rows past the last key must read as zero
-            uint64_t* vbar = partial ? &bars[B_VRAW] : &bars[B_VFULL + s];
-            if (lane == 0) mbar_expect_tx(vbar, bytes);
-            __syncwarp();
-            if (lane < ng) tma_load_3d(smem_u32(sv + s * kTile + lane * 2048), &kvmap, vbar, 0, row_k + p.nkv * p.ps, t);
-            if (partial) {                                         // at most once per CTA: its last tile
-                if (!mbar_wait(&bars[B_VRAW], 0u, abort_flag)) { if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_FLASH_VRAW); *abort_flag = 1; } break; }
-                const int nvalid = key_end - key0;
-                for (int idx = lane; idx < (128 - nvalid) * 8; idx += 32)
-                    *reinterpret_cast<uint4*>(sv + s * kTile + (nvalid + idx / 8) * 128 + (idx % 8) * 16) = make_uint4(0, 0, 0, 0);
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            return row_k;
+        };
+        while (jk < n_tiles || jv < n_tiles) {
+            bool progressed = false;
+            if (jk < n_tiles && __any_sync(0xffffffffu, mbar_try(&bars[B_KEMPTY + jk % kStages], ((uint32_t)(jk / kStages) & 1u) ^ 1u))) {
+                const int s = jk % kStages;
+                int ng;
+                const int row_k = rows_of(jk, ng);
+                if (lane == 0) mbar_expect_tx(&bars[B_KFULL + s], (uint32_t)ng * 16u * kDh);
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&bars[B_VFULL + s]);
+                if (lane < ng) tma_load_3d(smem_u32(sk + s * kTile + lane * 2048), &kvmap, &bars[B_KFULL + s], 0, row_k, t);
+                ++jk; progressed = true;
+            }
+            if (jv < n_tiles && __any_sync(0xffffffffu, mbar_try(&bars[B_VEMPTY + jv % kStages], ((uint32_t)(jv / kStages) & 1u) ^ 1u))) {
+                const int s = jv % kStages;
+                int ng;
+                const int row_k = rows_of(jv, ng);
+                const int key0 = kstart + jv * 128;
+                const bool partial = key0 + 128 > key_end;         // rows past the last key must read as zero
+                uint64_t* vbar = partial ? &bars[B_VRAW] : &bars[B_VFULL + s];
+                if (lane == 0) mbar_expect_tx(vbar, (uint32_t)ng * 16u * kDh);
+                __syncwarp();
+                if (lane < ng) tma_load_3d(smem_u32(sv + s * kTile + lane * 2048), &kvmap, vbar, 0, row_k + p.nkv * p.ps, t);
+                if (partial) {                                     // at most once per CTA: its last tile
+                    if (!mbar_wait(&bars[B_VRAW], 0u, abort_flag)) { if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, LOC_FLASH_VRAW); *abort_flag = 1; } break; }
+                    const int nvalid = key_end - key0;
+                    for (int idx = lane; idx < (128 - nvalid) * 8; idx += 32)
+                        *reinterpret_cast<uint4*>(sv + s * kTile + (nvalid + idx / 8) * 128 + (idx % 8) * 16) = make_uint4(0, 0, 0, 0);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars[B_VFULL + s]);
+                }
+                ++jv; progressed = true;
+            }
+            if (progressed) { idle = 0; clock = WaitClock(); continue; }
+            __nanosleep(64);
+            if ((++idle & 255u) == 255u && (*abort_flag || clock.expired() || idle > kSpin)) {
+                if (lane == 0) { report(p.status, PT_ERR_DEVICE_TIMEOUT, jk < n_tiles ? LOC_FLASH_KEMPTY : LOC_FLASH_VEMPTY); *abort_flag = 1; }
+                break;
             }
         }
         if (bad_page) report(p.status, PT_ERR_DEVICE_BOUNDS, LOC_DECODE_PAGE);
