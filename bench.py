@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the Parallel Track (PT) forward pass on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg3|cfg1|cfg4]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg3|cfg1|cfg4|cfg0|cfg2_kv8|cfg4_kv8|pt30b_prefill|pt30b_decode]
                     [--extra cfg3,cfg1] [--impl ours|reference]
 
 One JSON line on stdout.  A "step" is one pass of the whole hot path over one batch: one
@@ -495,7 +495,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2")
-    ap.add_argument("--extra", default="cfg3,cfg4,cfg4_kv8,cfg1,cfg0", help="comma-separated workloads reported under 'extra' (N=1 only); '' for none")
+    ap.add_argument("--extra", default="cfg3,cfg4,cfg4_kv8,cfg2_kv8,cfg1,cfg0", help="comma-separated workloads reported under 'extra' (N=1 only); '' for none")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--parallel", default="replicas", choices=["replicas", "tracks"],
                     help="N > 1: 'replicas' = every rank runs the whole model on its own batch (weak scaling, no collective); "

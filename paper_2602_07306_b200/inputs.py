@@ -101,6 +101,9 @@ WORKLOADS = {
                      dtype="bf16", mode="prefill", batch=8, seq=4096),
     "cfg4": Workload("cfg4", T=4, L=48, D=6, hidden=2048, heads=16, kv_heads=4, ffn=5632,
                      dtype="bf16", mode="decode", batch=256, seq=0, ragged=(512, 4096)),
+    # The batched decode workload with the cache in the library's E4M3 format.
+    "cfg2_kv8": Workload("cfg2_kv8", T=8, L=32, D=8, hidden=1024, heads=8, kv_heads=8, ffn=2816,
+                         dtype="bf16", mode="decode", batch=64, seq=2048),
     # The same ragged decode workload with the cache in the library's E4M3 format: the whole batch of 256 fits.
     "cfg4_kv8": Workload("cfg4_kv8", T=4, L=48, D=6, hidden=2048, heads=16, kv_heads=4, ffn=5632,
                          dtype="bf16", mode="decode", batch=256, seq=0, ragged=(512, 4096)),
