@@ -498,7 +498,7 @@ pt_status launch_decode_attn_e4m3(Call& k, const __nv_bfloat16* q, int layer, __
     const pt_model* m = k.m;
     const pt_kv_cache* c = k.c;
     const pt_config& g = m->cfg;
-    if (!(g.flags & 4)) return launch_decode_attn_e4m3_tc(k, q, layer, o);
+    if (!(g.flags & 4) && k.n_items <= 65535) return launch_decode_attn_e4m3_tc(k, q, layer, o);   // its key ranges are grid.y
     Dec8P pp{};
     AttnP& p = pp.a;
     p.q = q; p.o = o; p.bt = k.w.meta.bt; p.maxp = k.w.meta.maxp; p.kvlen = k.w.meta.kvlen;

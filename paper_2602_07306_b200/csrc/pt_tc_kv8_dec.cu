@@ -173,9 +173,11 @@ k_decode_attn_e4m3_tc(const __grid_constant__ CUtensorMap kvmap, const Dec8TcP p
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int32_t* item = p.items + (size_t)blockIdx.x * 4;
+    // the KV heads of one (track, sequence, key range) are neighbours in the grid: CTAs that run together read
+    // neighbouring 2 KB blocks of the same pages
+    const int32_t* item = p.items + (size_t)blockIdx.y * 4;
     const int b = item[0], kstart = item[1], kcount = item[2], split = item[3];
-    const int kvh = blockIdx.y, t = blockIdx.z;
+    const int kvh = blockIdx.x, t = blockIdx.z;
     const int G = p.nq / p.nkv;
 
     if (threadIdx.x == 0) {
@@ -558,7 +560,7 @@ pt_status launch_decode_attn_e4m3_tc(Call& k, const __nv_bfloat16* q, int layer,
         if (e != cudaSuccess) { set_error("cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
         done = true;
     }
-    cudaError_t e = launch_dependent(k_decode_attn_e4m3_tc, dim3(k.n_items, g.kv_heads, g.T), dim3(kThreads), (size_t)kSmem, k.st, kvmap, pp);
+    cudaError_t e = launch_dependent(k_decode_attn_e4m3_tc, dim3(g.kv_heads, k.n_items, g.T), dim3(kThreads), (size_t)kSmem, k.st, kvmap, pp);
     if (e != cudaSuccess) { set_error("k_decode_attn_e4m3_tc launch: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     if (k.max_splits > 1) return launch_decode_combine(p, g.T, m->dh, k.st);
