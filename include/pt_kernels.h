@@ -100,6 +100,30 @@ pt_status pt_kernel_decode_attn_static(const void* q, const void* pool_l, int64_
  * Asynchronous on `stream`; nothing is allocated. */
 pt_status pt_kernel_kv_quant_e4m3(const void* src, void* codes, float* scales, int64_t n, void* status, void* stream);
 
+/* Decode attention over one layer's slab of an E4M3 cache (pt_kv_dtype PT_KV_E4M3 in pt.h; Algorithm 1's attention of
+ * a single-token step, Section 2.1, over the cache format this library defines): for every track, sequence b and
+ * query head, softmax(q k^T / sqrt(128)) v over the kv_len[b] cached keys, where a cached vector is its 128 codes
+ * times its scale.  Head size 128 only.
+ *   q            device bf16 [T][B][nq * 128]
+ *   codes_l      device uint8, one layer: [T] slabs codes_track_stride BYTES apart, each [num_pages][K|V][nkv][ps][128];
+ *                128-byte aligned, stride a multiple of 128
+ *   scales_l     device fp32, the same order without the last dimension; slabs scales_track_stride FLOATS apart
+ *   block_table  device int32 [B][maxp]     kv_len  HOST int32 [B], each in [1, maxp * ps]
+ *   ps           page size, a multiple of 16 up to 64;  nkv <= 8;  nq / nkv <= 8
+ *   out          device bf16 [T][B][nq * 128]
+ *   impl         0: the tcgen05 kernel (8-bit MMAs), 1: the mma.sync kernel (codes converted to f16)
+ *   scratch      device, 256-byte aligned, at least pt_kernel_decode_attn_scratch_bytes(T, B, nq, 128) bytes
+ *   status       device int32[16], zeroed by the caller
+ * The key ranges are planned on the host and uploaded with an asynchronous copy on `stream`; everything else is
+ * asynchronous on `stream` too.  Nothing is allocated.  Errors: PT_ERR_INVALID_ARG / UNSUPPORTED / MISALIGNED /
+ * BUFFER_TOO_SMALL before anything is launched; a page number outside [0, num_pages) is reported in `status`. */
+pt_status pt_kernel_decode_attn_e4m3(const void* q, const void* codes_l, int64_t codes_track_stride,
+                                     const float* scales_l, int64_t scales_track_stride,
+                                     const int32_t* block_table, int32_t maxp, const int32_t* kv_len,
+                                     int32_t T, int32_t B, int32_t nq, int32_t nkv, int32_t ps,
+                                     int32_t num_pages, void* out, int32_t impl, void* scratch, size_t scratch_bytes,
+                                     void* status, void* stream);
+
 /* ---- the bounded wait, exercised ------------------------------------------------------------
  * Every device-side wait of the library (an mbarrier of a TMA -> MMA -> epilogue pipeline) gives up
  * after a time limit (2 s of device time, whatever the iteration counts), records PT_ERR_DEVICE_TIMEOUT with

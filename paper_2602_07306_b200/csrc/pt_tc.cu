@@ -506,6 +506,52 @@ extern "C" pt_status pt_kernel_decode_attn(const void* q, const void* pool_l, in
                                     num_pages, out, (char*)scratch, status, (cudaStream_t)stream);
 }
 
+extern "C" pt_status pt_kernel_decode_attn_e4m3(const void* q, const void* codes_l, int64_t codes_track_stride,
+                                                const float* scales_l, int64_t scales_track_stride,
+                                                const int32_t* block_table, int32_t maxp, const int32_t* kv_len,
+                                                int32_t T, int32_t B, int32_t nq, int32_t nkv, int32_t ps,
+                                                int32_t num_pages, void* out, int32_t impl, void* scratch, size_t scratch_bytes,
+                                                void* status, void* stream) {
+    using namespace pt;
+    const int dh = 128;
+    pt_status s = decode_attn_check_args(q, codes_l, block_table, maxp, kv_len, T, B, nq, nkv, dh, ps, num_pages, out, status);
+    if (s != PT_OK) return s;
+    if (!scales_l || !scratch) { set_error("null argument"); return PT_ERR_INVALID_ARG; }
+    if (ps % 16 || nkv > 8) { set_error("an E4M3 cache needs pages of a multiple of 16 tokens and at most 8 KV heads"); return PT_ERR_UNSUPPORTED; }
+    if (impl != 0 && impl != 1) { set_error("impl must be 0 or 1"); return PT_ERR_INVALID_ARG; }
+    if ((uintptr_t)codes_l % 128 || codes_track_stride % 128 || (uintptr_t)scales_l % 4 || (uintptr_t)scratch % 256) {
+        set_error("codes must be 128-byte, scales 4-byte, scratch 256-byte aligned"); return PT_ERR_MISALIGNED;
+    }
+    DecodeScratch d = decode_scratch_layout(T, B, nq, dh);
+    if (scratch_bytes < d.total) { set_error("scratch: %zu < %zu bytes", scratch_bytes, d.total); return PT_ERR_BUFFER_TOO_SMALL; }
+    cudaStream_t st = (cudaStream_t)stream;
+    std::vector<int32_t> host((d.o_part) / 4, 0);
+    int32_t* items = host.data() + d.o_items / 4;
+    int32_t* nsplit = host.data() + d.o_nsplit / 4;
+    int32_t* lens = host.data() + d.o_len / 4;
+    for (int b = 0; b < B; ++b) lens[b] = kv_len[b];
+    int n_items = 0, max_splits = 1;
+    plan_decode_splits(lens, B, ps, (int64_t)T * nkv, items, nsplit, &n_items, &max_splits);
+    cudaError_t e = cudaMemcpyAsync(scratch, host.data(), d.o_part, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) { set_error("cudaMemcpyAsync: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
+    char* sc = (char*)scratch;
+    AttnP p{};
+    p.q = (const __nv_bfloat16*)q; p.o = (__nv_bfloat16*)out; p.bt = block_table; p.maxp = maxp; p.kvlen = (const int32_t*)(sc + d.o_len);
+    p.B = B; p.S = 1; p.M = B; p.nq = nq; p.nkv = nkv; p.ps = ps; p.num_pages = num_pages;
+    p.scale_log2 = 1.4426950408889634f / sqrtf((float)dh);
+    p.status = (int*)status;
+    p.items = (const int32_t*)(sc + d.o_items); p.nsplit = (const int32_t*)(sc + d.o_nsplit);
+    p.part = (float*)(sc + d.o_part); p.max_splits = kMaxSplits;
+    Kv8Slab slab{};
+    slab.codes_l = (const uint8_t*)codes_l; slab.codes_tstride = codes_track_stride;
+    slab.scales_l = scales_l; slab.scales_tstride = scales_track_stride;
+    s = launch_decode_attn_e4m3_p(p, slab, T, n_items, max_splits, impl == 1, st);
+    if (s != PT_OK) return s;
+    e = cudaGetLastError();
+    if (e != cudaSuccess) { set_error("kernel launch failed: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
+    return PT_OK;
+}
+
 // ---- decode attention with built-in scratch -------------------------------------------------
 // The array lives in the library image, once per device that loads it.  In host code its name
 // is only a handle: the device address comes from cudaGetSymbolAddress, looked up once per

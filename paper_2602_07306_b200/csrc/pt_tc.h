@@ -156,7 +156,15 @@ pt_status launch_kv_quant(Call& k, int layer);
 pt_status launch_kv_dequant_ctx(Call& k, int layer);
 pt_status launch_flash_prefill_e4m3(Call& k, const __nv_bfloat16* q, __nv_bfloat16* o);
 pt_status launch_decode_attn_e4m3(Call& k, const __nv_bfloat16* q, int layer, __nv_bfloat16* o);
+// One layer's slab of an E4M3 cache as the decode kernels see it: codes [track][page][K|V][kv_head][slot][128] bytes
+// and one fp32 scale per vector in the same order, tracks a fixed stride apart.
+struct Kv8Slab {
+    const uint8_t* codes_l; int64_t codes_tstride;        // bytes between tracks
+    const float* scales_l; int64_t scales_tstride;        // floats between tracks
+};
+// p holds q, o, the block table, lengths, key ranges (items, nsplit), partial-result buffer, sizes and the status block
+pt_status launch_decode_attn_e4m3_p(const AttnP& p, const Kv8Slab& slab, int T, int n_items, int max_splits, bool mma_sync, cudaStream_t st);
 // pt_tc_kv8_dec.cu: the same on tcgen05 (the default; the mma.sync kernel serves config flag bit 2)
-pt_status launch_decode_attn_e4m3_tc(Call& k, const __nv_bfloat16* q, int layer, __nv_bfloat16* o);
+pt_status launch_decode_attn_e4m3_tc(const AttnP& p, const Kv8Slab& slab, int T, int n_items, int max_splits, cudaStream_t st);
 
 }  // namespace pt

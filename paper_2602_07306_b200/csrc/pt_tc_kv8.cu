@@ -494,21 +494,13 @@ pt_status launch_flash_prefill_e4m3(Call& k, const __nv_bfloat16* q, __nv_bfloat
     return launch_flash_prefill_p(p, g.T, m->dh, (g.flags & 2) != 0, k.st);
 }
 
-pt_status launch_decode_attn_e4m3(Call& k, const __nv_bfloat16* q, int layer, __nv_bfloat16* o) {
-    const pt_model* m = k.m;
-    const pt_kv_cache* c = k.c;
-    const pt_config& g = m->cfg;
-    if (!(g.flags & 4) && k.n_items <= 65535) return launch_decode_attn_e4m3_tc(k, q, layer, o);   // its key ranges are grid.y
+pt_status launch_decode_attn_e4m3_p(const AttnP& p, const Kv8Slab& slab, int T, int n_items, int max_splits, bool mma_sync, cudaStream_t st) {
+    if (!mma_sync && n_items <= 65535) return launch_decode_attn_e4m3_tc(p, slab, T, n_items, max_splits, st);   // its key ranges are grid.y
     Dec8P pp{};
-    AttnP& p = pp.a;
-    p.q = q; p.o = o; p.bt = k.w.meta.bt; p.maxp = k.w.meta.maxp; p.kvlen = k.w.meta.kvlen;
-    p.B = k.B; p.S = 1; p.M = k.M; p.nq = g.heads; p.nkv = g.kv_heads; p.ps = c->ps; p.num_pages = c->num_pages;
-    p.scale_log2 = 1.4426950408889634f / sqrtf((float)m->dh);
-    p.status = m->status();
-    p.items = k.items; p.nsplit = k.nsplit; p.part = k.w.part; p.max_splits = kMaxSplits;
-    pp.scales_l = c->scales + (size_t)layer * c->slab_vecs(); pp.scales_tstride = (int64_t)g.L * c->slab_vecs();
+    pp.a = p;
+    pp.scales_l = slab.scales_l; pp.scales_tstride = slab.scales_tstride;
     CUtensorMap kvmap;
-    pt_status s = make_codes_map(&kvmap, c->pool + (size_t)layer * c->slab_elems, c->ps, g.kv_heads, c->num_pages, g.T, (int64_t)g.L * c->slab_elems);
+    pt_status s = make_codes_map(&kvmap, slab.codes_l, p.ps, p.nkv, p.num_pages, T, slab.codes_tstride);
     if (s != PT_OK) return s;
     const int smem = 1024 + 4 * kDecStages * kSlotBytes + 4 * kDecStages * 32 * 4 + 4 * kDecStages * 8;
     static bool done_[kMaxDevices] = {};
@@ -518,11 +510,27 @@ pt_status launch_decode_attn_e4m3(Call& k, const __nv_bfloat16* q, int layer, __
         if (e != cudaSuccess) { set_error("cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
         done = true;
     }
-    cudaError_t e = launch_dependent(k_decode_attn_e4m3, dim3(k.n_items, g.kv_heads, g.T), dim3(kDecThreads), (size_t)smem, k.st, kvmap, pp);
+    cudaError_t e = launch_dependent(k_decode_attn_e4m3, dim3(n_items, p.nkv, T), dim3(kDecThreads), (size_t)smem, st, kvmap, pp);
     if (e != cudaSuccess) { set_error("k_decode_attn_e4m3 launch: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    if (k.max_splits > 1) return launch_decode_combine(p, g.T, m->dh, k.st);
+    if (max_splits > 1) return launch_decode_combine(p, T, kDh, st);
     return PT_OK;
+}
+
+pt_status launch_decode_attn_e4m3(Call& k, const __nv_bfloat16* q, int layer, __nv_bfloat16* o) {
+    const pt_model* m = k.m;
+    const pt_kv_cache* c = k.c;
+    const pt_config& g = m->cfg;
+    AttnP p{};
+    p.q = q; p.o = o; p.bt = k.w.meta.bt; p.maxp = k.w.meta.maxp; p.kvlen = k.w.meta.kvlen;
+    p.B = k.B; p.S = 1; p.M = k.M; p.nq = g.heads; p.nkv = g.kv_heads; p.ps = c->ps; p.num_pages = c->num_pages;
+    p.scale_log2 = 1.4426950408889634f / sqrtf((float)m->dh);
+    p.status = m->status();
+    p.items = k.items; p.nsplit = k.nsplit; p.part = k.w.part; p.max_splits = kMaxSplits;
+    Kv8Slab slab{};
+    slab.codes_l = (const uint8_t*)c->pool + (size_t)layer * c->slab_elems; slab.codes_tstride = (int64_t)g.L * c->slab_elems;
+    slab.scales_l = c->scales + (size_t)layer * c->slab_vecs(); slab.scales_tstride = (int64_t)g.L * c->slab_vecs();
+    return launch_decode_attn_e4m3_p(p, slab, g.T, k.n_items, k.max_splits, (g.flags & 4) != 0, k.st);
 }
 
 }  // namespace pt

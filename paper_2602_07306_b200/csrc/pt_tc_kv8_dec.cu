@@ -14,8 +14,8 @@
 // With keys on M every per-key quantity is a per-thread scalar: softmax thread r of 128 owns key r of the tile - its
 // K scale multiplies its 8 scores, its V scale its 8 probabilities, its row sums stay in registers until the end.
 // Only the tile's maxima (8 heads and the V scale) cross threads: redux.sync per warp, 36 floats of shared memory
-// and one named barrier per tile.  The reference maximum is raised only when it grows by more than 2^8 (the
-// accumulator is then rescaled in tensor memory), so rescales are rare.
+// and one named barrier per tile.  The reference maximum is raised only when it grows by more than 2^2 (the
+// accumulator is then rescaled in tensor memory), so rescales are rare; the bound keeps 64 p inside the E4M3 range.
 // Roles: warp 0 streams K and V tiles page by page with TMA (one 16 x 128-byte box per page and K|V) through
 // two-stage rings (so that three CTAs fit an SM: the kernel is bound by the latency of its copies, more CTAs hide it); warp 1 issues the MMAs (the scores of tile j+2 right behind P V of tile j: S^T is double-buffered in
 // tensor memory, P in shared memory); warps 2-5 are the softmax threads.  Every mbarrier wait is bounded; the named
@@ -34,6 +34,13 @@ constexpr int kStages = 2;
 constexpr int kTile = 128 * kDh;            // bytes of a K or V tile: 128 keys x 128 code bytes
 constexpr int kQBytes = 16 * kDh;           // q (and one P buffer): 16 rows of 128 bytes
 constexpr uint32_t kSpin = 1u << 26;
+// A head's reference maximum is raised (and the accumulator rescaled) when a tile's maximum exceeds it by more than
+// this many powers of two.  Until then a probability can reach 2^kLazyLog2; times the factor 64 of the P codes that
+// must stay inside the E4M3 range: 4 * 64 = 256 <= 448.
+#ifndef T8_LAZY_LOG2
+#define T8_LAZY_LOG2 2.0f
+#endif
+constexpr float kLazyLog2 = T8_LAZY_LOG2;
 
 enum { B_KFULL = 0, B_KEMPTY = 3, B_VFULL = 6, B_VEMPTY = 9, B_SFULL = 12, B_SEMPTY = 14, B_PFULL = 16, B_PEMPTY = 18,
        B_VRAW = 20, B_COUNT = 21 };
@@ -411,7 +418,7 @@ k_decode_attn_e4m3_tc(const __grid_constant__ CUtensorMap kvmap, const Dec8TcP p
                 const float* r = red + bb * 48 + h;
                 const float mx = fmaxf(fmaxf(r[0], r[12]), fmaxf(r[24], r[36]));
                 corr[h] = 1.0f;
-                if ((mx - m_ref[h]) > 8.0f) { corr[h] = ex2f(m_ref[h] - mx); m_ref[h] = mx; rescale = true; }
+                if ((mx - m_ref[h]) > kLazyLog2) { corr[h] = ex2f(m_ref[h] - mx); m_ref[h] = mx; rescale = true; }
             }
             {
                 const float* r = red + bb * 48 + 8;
@@ -538,20 +545,13 @@ pt_status make_codes_map3(CUtensorMap* out, const void* base, int64_t vecs, int6
 
 }  // namespace
 
-pt_status launch_decode_attn_e4m3_tc(Call& k, const __nv_bfloat16* q, int layer, __nv_bfloat16* o) {
-    const pt_model* m = k.m;
-    const pt_kv_cache* c = k.c;
-    const pt_config& g = m->cfg;
+pt_status launch_decode_attn_e4m3_tc(const AttnP& p, const Kv8Slab& slab, int T, int n_items, int max_splits, cudaStream_t st) {
     Dec8TcP pp{};
-    AttnP& p = pp.a;
-    p.q = q; p.o = o; p.bt = k.w.meta.bt; p.maxp = k.w.meta.maxp; p.kvlen = k.w.meta.kvlen;
-    p.B = k.B; p.S = 1; p.M = k.M; p.nq = g.heads; p.nkv = g.kv_heads; p.ps = c->ps; p.num_pages = c->num_pages;
-    p.scale_log2 = 1.4426950408889634f / sqrtf((float)m->dh);
-    p.status = m->status();
-    p.items = k.items; p.nsplit = k.nsplit; p.part = k.w.part; p.max_splits = kMaxSplits;
-    pp.scales_l = c->scales + (size_t)layer * c->slab_vecs(); pp.scales_tstride = (int64_t)g.L * c->slab_vecs();
+    pp.a = p;
+    pp.scales_l = slab.scales_l; pp.scales_tstride = slab.scales_tstride;
     CUtensorMap kvmap;
-    pt_status s = make_codes_map3(&kvmap, c->pool + (size_t)layer * c->slab_elems, c->slab_vecs(), g.T, (int64_t)g.L * c->slab_elems);
+    const int64_t slab_vecs = (int64_t)p.num_pages * 2 * p.nkv * p.ps;
+    pt_status s = make_codes_map3(&kvmap, slab.codes_l, slab_vecs, T, slab.codes_tstride);
     if (s != PT_OK) return s;
     static bool done_[kMaxDevices] = {};
     bool& done = done_[current_device()];
@@ -560,10 +560,10 @@ pt_status launch_decode_attn_e4m3_tc(Call& k, const __nv_bfloat16* q, int layer,
         if (e != cudaSuccess) { set_error("cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
         done = true;
     }
-    cudaError_t e = launch_dependent(k_decode_attn_e4m3_tc, dim3(g.kv_heads, k.n_items, g.T), dim3(kThreads), (size_t)kSmem, k.st, kvmap, pp);
+    cudaError_t e = launch_dependent(k_decode_attn_e4m3_tc, dim3(p.nkv, n_items, T), dim3(kThreads), (size_t)kSmem, st, kvmap, pp);
     if (e != cudaSuccess) { set_error("k_decode_attn_e4m3_tc launch: %s", cudaGetErrorString(e)); return PT_ERR_CUDA; }
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    if (k.max_splits > 1) return launch_decode_combine(p, g.T, m->dh, k.st);
+    if (max_splits > 1) return launch_decode_combine(p, T, kDh, st);
     return PT_OK;
 }
 

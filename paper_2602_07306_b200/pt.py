@@ -86,6 +86,8 @@ _PROTOS = {
                                      _P, _P, _SZ, _P, _P]),
     "pt_kernel_decode_attn_static": (_I32, [_P, _P, _I64, _P, _I32, C.POINTER(_I32), _I32, _I32, _I32, _I32, _I32, _I32, _I32,
                                             _P, _P, _P]),
+    "pt_kernel_decode_attn_e4m3": (_I32, [_P, _P, _I64, _P, _I64, _P, _I32, C.POINTER(_I32), _I32, _I32, _I32, _I32, _I32, _I32,
+                                          _P, _I32, _P, _SZ, _P, _P]),
     "pt_kernel_wait_selftest": (_I32, [_P, C.c_uint64, _P]),
     "pt_last_error": (C.c_char_p, []),
 }
@@ -517,6 +519,30 @@ def kernel_decode_attn(q, pool_l, block_table, kv_len, *, nq, nkv, dh, ps, scrat
                                           block_table.shape[1], plens, T, B, nq, nkv, dh, ps, pages, out.data_ptr(),
                                           scratch.data_ptr(), scratch.numel(), status.data_ptr(),
                                           torch.cuda.current_stream().cuda_stream))
+    return out, status
+
+
+def kernel_decode_attn_e4m3(q, codes_l, scales_l, block_table, kv_len, *, nq, nkv, ps, impl=0):
+    """q bf16 [T, B, nq*128]; codes_l uint8 [T, pages, 2, nkv, ps, 128]; scales_l fp32 [T, pages, 2, nkv, ps];
+    block_table int32 [B, maxp] (CUDA); kv_len: host ints [B]; impl 0 = tcgen05 kernel, 1 = mma.sync kernel.
+    Returns (out bf16 [T, B, nq*128], status int32[16])."""
+    import torch
+    T, B, _ = q.shape
+    pages = codes_l.shape[1]
+    assert q.is_contiguous() and codes_l.is_contiguous() and scales_l.is_contiguous() and block_table.is_contiguous()
+    assert q.dtype == torch.bfloat16 and codes_l.dtype == torch.uint8 and scales_l.dtype == torch.float32
+    assert block_table.dtype == torch.int32 and tuple(scales_l.shape) == tuple(codes_l.shape[:-1])
+    out = torch.empty_like(q)
+    status = torch.zeros(16, dtype=torch.int32, device=q.device)
+    n = _SZ()
+    check(lib().pt_kernel_decode_attn_scratch_bytes(T, B, nq, 128, C.byref(n)))
+    scratch = torch.empty(n.value, dtype=torch.uint8, device=q.device)
+    lens, plens = _i32arr(kv_len)
+    with torch.cuda.device(q.device):
+        check(lib().pt_kernel_decode_attn_e4m3(q.data_ptr(), codes_l.data_ptr(), codes_l.stride(0), scales_l.data_ptr(),
+                                               scales_l.stride(0), block_table.data_ptr(), block_table.shape[1], plens,
+                                               T, B, nq, nkv, ps, pages, out.data_ptr(), impl, scratch.data_ptr(),
+                                               scratch.numel(), status.data_ptr(), torch.cuda.current_stream().cuda_stream))
     return out, status
 
 

@@ -39,6 +39,10 @@ def _operands(T, M, N, K, seed):
     (1, 4096, 1024, 1024, 256, False),    # CTA pairs: more tiles than pairs, both accumulators in use
     (2, 176, 768, 512, 0, False),         # a large decode batch: one 256-row pair tile whose odd CTA holds 48 rows
     (3, 130, 256, 320, 0, False),         # the odd CTA holds two rows
+    (4, 176, 3072, 2048, 0, False),       # CTA pairs at decode size (a 176-row batch against a wide projection): the ring wraps five times
+    (2, 256, 5120, 384, 0, False),        # CTA pairs at decode size: exactly 256 rows, as many k-blocks as ring stages
+    (2, 300, 2816, 320, 0, False),        # CTA pairs at decode size: two 256-row tiles, the second with 44 rows in its even CTA only
+    (1, 512, 10368, 256, 0, False),       # CTA pairs at decode size: more tiles than pairs, N tail of half a tile
 ])
 def test_gemm_bf16_matches_definition(T, M, N, K, bn, fold):
     import torch

@@ -7,8 +7,14 @@
     same cache format: final output and every layer's stream within 2e-2 of the maximum and within the mean
     bound derived from the measured floor (tests/bf16_floor.py with kv8: the device quantises the K and V its
     bf16 GEMM produced, the oracle its exact ones, so a value near a code boundary lands one code step away;
-    that, not bf16 rounding, sets the floor); scales and cached values; page tables bit-exact.
+    that, not bf16 rounding, sets the floor); scales and cached values; page tables bit-exact;
+  * the two decode-attention kernels alone on caches the oracle quantised (both sides read the same codes and
+    scales, so only the kernels' own arithmetic differs): random scores, scores that climb steadily or jump by
+    2^5 / 2^7.5 after a key range's first tile (the running reference maximum and the range of the 8-bit
+    probabilities), V magnitudes that double along the sequence, one to eight query heads per KV head.
 """
+import functools
+
 import numpy as np
 import pytest
 
@@ -137,3 +143,95 @@ def test_e4m3_cache_gqa4_pages_of_32_tokens(flags):
 def test_e4m3_cache_gqa8_long_sequences_split_over_key_ranges(flags):
     # 700 cached keys and few sequences: the decode step splits every sequence over several key ranges
     run_kv8_case(_wl("kv8-gqa8", 2, 2, 2, 1024, 8, 1, 256), B=2, chunks=[512, 188], decode_steps=2, sync_op="mean", flags=flags)
+
+
+def _kv8_attention_case(T, B, nq, nkv, ps, lens, seed, climb_log2=0.0, climb_at=0, v_scale_steps=0):
+    """A random paged E4M3 cache (quantised by the oracle) and bf16 queries; the float64 result of oracle.attention
+    over code * scale.  With climb_log2 the first query head of every KV head sees scores that rise by that many
+    powers of two along a sequence (keys aligned with the query, growing in length): steadily from the first key to
+    the last, or, with climb_at, all at once at that key.  With v_scale_steps the magnitude of V doubles that many
+    times along a sequence."""
+    import torch
+    rng = np.random.default_rng(seed)
+    G, dh = nq // nkv, 128
+    maxp = max(-(-int(n) // ps) for n in lens)
+    pages = sum(-(-int(n) // ps) for n in lens) + 2
+    perm = I.free_list_permutation(pages, seed=seed)
+    bt = np.zeros((B, maxp), np.int32)
+    nxt = 0
+    for b, n in enumerate(lens):
+        k = -(-int(n) // ps)
+        bt[b, :k] = perm[nxt:nxt + k]
+        nxt += k
+    pool = rng.standard_normal((T, pages, 2, nkv, ps, dh))
+    q = rng.standard_normal((T, B, nq, dh))
+    if climb_log2 or v_scale_steps:
+        beta = 10.0
+        for t in range(T):
+            for b, n in enumerate(lens):
+                pos = np.arange(int(n))
+                pg, sl = bt[b, pos // ps], pos % ps
+                rise = (pos >= climb_at).astype(np.float64) if climb_at else pos / max(1, int(n) - 1)
+                # a score in powers of two is log2(e) * beta * alpha / sqrt(dh)
+                alpha = rise * climb_log2 * np.sqrt(dh) / (np.log2(np.e) * beta)
+                for h in range(nkv):
+                    if climb_log2:
+                        u = rng.standard_normal(dh)
+                        u /= np.linalg.norm(u)
+                        q[t, b, h * G] = beta * u
+                        pool[t, pg, 0, h, sl] = alpha[:, None] * u[None, :] + 0.3 * pool[t, pg, 0, h, sl]
+                    if v_scale_steps:
+                        pool[t, pg, 1, h, sl] *= np.exp2(np.floor(pos * v_scale_steps / int(n)))[:, None]
+    q = I.round_to_bf16(q.astype(np.float32)).astype(np.float64)
+    codes, scale = O.kv_quantize(pool.reshape(-1, dh))
+    deq = (codes * scale).reshape(pool.shape)
+    ref = np.zeros((T, B, nq * dh))
+    for t in range(T):
+        for b, n in enumerate(lens):
+            pos = np.arange(int(n))
+            k = deq[t, bt[b, pos // ps], 0, :, pos % ps, :]
+            v = deq[t, bt[b, pos // ps], 1, :, pos % ps, :]
+            ref[t, b] = O.attention(q[t, b].reshape(1, nq, dh), k, v, np.array([int(n) - 1])).reshape(-1)
+    code_bytes = torch.from_numpy(codes.astype(np.float32)).to(torch.float8_e4m3fn).view(torch.uint8)
+    dev = lambda a: a.to("cuda:0").contiguous()
+    return (dev(torch.from_numpy(q.reshape(T, B, nq * dh).astype(np.float32)).to(torch.bfloat16)),
+            dev(code_bytes.reshape(T, pages, 2, nkv, ps, dh)),
+            dev(torch.from_numpy(scale.reshape(T, pages, 2, nkv, ps).astype(np.float32))),
+            dev(torch.from_numpy(bt)), ref)
+
+
+@functools.lru_cache(maxsize=1)
+def _cached_case(T, B, nq, nkv, ps, lens, seed, climb, at, vsteps):
+    return _kv8_attention_case(T, B, nq, nkv, ps, list(lens), seed, climb_log2=climb, climb_at=at, v_scale_steps=vsteps)
+
+
+# The kernels keep q and the probabilities as pairs of E4M3 numbers (relative error 2^-8 per element) and write bf16.
+ATTN8_MAX, ATTN8_MEAN = 1e-2, 3e-3
+
+# With many sequences a key range is a whole sequence (the planner splits only to fill the machine), so one CTA walks
+# all of a sequence's tiles with one running reference maximum.
+MANY = 80
+
+
+@pytest.mark.parametrize("impl", [0, 1], ids=["tcgen05", "mma_sync"])
+@pytest.mark.parametrize("T,B,nq,nkv,ps,lens,climb,at,vsteps", [
+    (2, 3, 8, 2, 16, [1, 130, 700], 0.0, 0, 0),                 # random scores; one key, a tile and a bit, several tiles and ranges
+    (1, 2, 4, 1, 16, [2048, 700], 14.0, 0, 0),                  # a steady climb by 2^14 over many short key ranges
+    (1, 2, 8, 8, 32, [1500, 4097], 6.0, 0, 5),                  # one query head per KV head, V magnitudes double five times
+    (2, 1, 8, 1, 16, [3000], 30.0, 0, 0),                       # a steep climb (2^30): early keys underflow, eight heads per KV head
+    (2, MANY, 4, 2, 16, [384] * MANY, 5.0, 128, 0),             # the scores rise by 2^5 after the first tile and stay there: a reference
+                                                                # maximum that is not raised at once leaves probabilities of 32 for most keys
+    (2, MANY, 4, 2, 16, [400 + 3 * i for i in range(MANY)], 7.5, 200, 3),   # the same with 2^7.5 in mid-tile, ragged lengths, growing V
+], ids=["random", "climb14", "climb6_v32", "climb30", "step5", "step7.5_v8"])
+def test_e4m3_decode_attention_kernels_against_the_oracle(impl, T, B, nq, nkv, ps, lens, climb, at, vsteps):
+    import torch
+    from paper_2602_07306_b200 import pt
+    q, codes, scales, bt, ref = _cached_case(T, B, nq, nkv, ps, tuple(lens), len(lens) + nq, climb, at, vsteps)   # both kernels: the same case
+    out, status = pt.kernel_decode_attn_e4m3(q, codes, scales, bt, lens, nq=nq, nkv=nkv, ps=ps, impl=impl)
+    torch.cuda.synchronize()
+    assert status[:2].tolist() == [0, 0]
+    got = out.float().cpu().numpy().astype(np.float64)
+    mx, mean = Hp.rel_errs(got, ref)
+    Hp.record(f"e4m3 decode attention kernel ({'mma.sync' if impl else 'tcgen05'}), scores rising by 2^{climb:g}, {B} sequences of up to {max(lens)} keys",
+              mx, mean, ATTN8_MAX, ATTN8_MEAN)
+    assert mx <= ATTN8_MAX and mean <= ATTN8_MEAN, f"max-rel {mx:.3e}, mean-rel {mean:.3e}"
