@@ -61,7 +61,25 @@ def test_gemm_bf16_matches_definition(T, M, N, K, bn, fold):
     assert err <= 2e-6 * np.sqrt(K * (T if fold else 1)), f"max-rel {err:.3e}"     # fp32 accumulation of exact bf16 products
 
 
-def decode_case(T, B, nq, nkv, dh, ps, lens, seed):
+def _climbing_scores(rng, pool, q_rows, bt, b, t, n, nq, nkv, dh, ps, climb, at):
+    """Rewrites the keys of sequence b (positions 0..n-1) and the first query head of every KV head (rows q_rows of
+    q[t], shaped [rows, nq, dh]) so that the scores rise by `climb` powers of two along the sequence: keys and queries
+    share a direction, the keys' length grows steadily from the first key to the last or, with `at`, all at once at
+    that key.  A kernel that carries a running maximum has to raise it again and again (or once, late)."""
+    G = nq // nkv
+    pos = np.arange(n)
+    pg, sl = bt[b, pos // ps], pos % ps
+    rise = (pos >= at).astype(np.float64) if at else pos / max(1, n - 1)
+    beta = 10.0
+    alpha = rise * climb * np.sqrt(dh) / (np.log2(np.e) * beta)          # a score in powers of two: log2(e) beta alpha / sqrt(dh)
+    for h in range(nkv):
+        u = rng.standard_normal(dh)
+        u /= np.linalg.norm(u)
+        q_rows[:, h * G, :] = beta * u[None, :] + 0.1 * q_rows[:, h * G, :]
+        pool[t, pg, 0, h, sl] = alpha[:, None] * u[None, :] + 0.3 * pool[t, pg, 0, h, sl]
+
+
+def decode_case(T, B, nq, nkv, dh, ps, lens, seed, climb=0.0, at=0):
     """Random paged cache + queries; returns torch inputs and the float64 oracle result
     (oracle.attention on the gathered keys, one sequence and track at a time)."""
     import torch
@@ -76,8 +94,13 @@ def decode_case(T, B, nq, nkv, dh, ps, lens, seed):
         k = -(-int(n) // ps)
         bt[b, :k] = perm[nxt:nxt + k]
         nxt += k
-    pool = I.round_to_bf16(rng.standard_normal((T, pages, 2, nkv, ps, dh), dtype=np.float32))
-    q = I.round_to_bf16(rng.standard_normal((T, B, nq * dh), dtype=np.float32))
+    pool = rng.standard_normal((T, pages, 2, nkv, ps, dh), dtype=np.float32)
+    q = rng.standard_normal((T, B, nq * dh), dtype=np.float32)
+    if climb:
+        for t in range(T):
+            for b, n in enumerate(lens):
+                _climbing_scores(rng, pool, q[t, b:b + 1].reshape(1, nq, dh), bt, b, t, int(n), nq, nkv, dh, ps, climb, at)
+    pool, q = I.round_to_bf16(pool), I.round_to_bf16(q)
     ref = np.zeros((T, B, nq * dh))
     for t in range(T):
         for b, n in enumerate(lens):
@@ -90,17 +113,20 @@ def decode_case(T, B, nq, nkv, dh, ps, lens, seed):
     return dev(q, torch.bfloat16), dev(pool, torch.bfloat16), dev(bt, torch.int32), ref
 
 
-@pytest.mark.parametrize("T,B,nq,nkv,dh,ps,lens", [
-    (2, 3, 2, 2, 128, 16, [1, 17, 64]),                 # single token, page tails, exactly one tile
-    (1, 2, 8, 2, 64, 16, [300, 1023]),                  # GQA 4:1, several key ranges per sequence
-    (2, 4, 4, 1, 128, 16, [513, 4097, 2048, 15]),       # ragged, long, GQA 4:1
-    (1, 2, 4, 4, 32, 8, [100, 37]),                     # small heads, 8-token pages
-    (3, 2, 16, 2, 128, 32, [700, 90]),                  # GQA 8:1, 32-token pages
+@pytest.mark.parametrize("T,B,nq,nkv,dh,ps,lens,climb,at", [
+    (2, 3, 2, 2, 128, 16, [1, 17, 64], 0, 0),                 # single token, page tails, exactly one tile
+    (1, 2, 8, 2, 64, 16, [300, 1023], 0, 0),                  # GQA 4:1, several key ranges per sequence
+    (2, 4, 4, 1, 128, 16, [513, 4097, 2048, 15], 0, 0),       # ragged, long, GQA 4:1
+    (1, 2, 4, 4, 32, 8, [100, 37], 0, 0),                     # small heads, 8-token pages
+    (3, 2, 16, 2, 128, 32, [700, 90], 0, 0),                  # GQA 8:1, 32-token pages
+    (1, 2, 8, 2, 128, 16, [2048, 700], 14.0, 0),              # scores climbing by 2^14 along the sequence: the running maximum rises in every tile
+    (2, 80, 4, 2, 128, 16, [384] * 80, 7.5, 128),             # many sequences (one key range each): the scores jump by 2^7.5 after the first tile
+    (1, 1, 4, 1, 64, 16, [3000], 60.0, 0),                    # a climb by 2^60: the early keys' weights underflow
 ])
-def test_decode_attention_kernel_matches_oracle(T, B, nq, nkv, dh, ps, lens):
+def test_decode_attention_kernel_matches_oracle(T, B, nq, nkv, dh, ps, lens, climb, at):
     import torch
     from paper_2602_07306_b200 import pt
-    q, pool, bt, ref = decode_case(T, B, nq, nkv, dh, ps, lens, seed=sum(lens))
+    q, pool, bt, ref = decode_case(T, B, nq, nkv, dh, ps, lens, seed=sum(lens), climb=climb, at=at)
     out, status = pt.kernel_decode_attn(q, pool, bt, lens, nq=nq, nkv=nkv, dh=dh, ps=ps)
     torch.cuda.synchronize()
     assert status[:2].tolist() == [0, 0]
@@ -121,7 +147,7 @@ def test_decode_attention_kernel_reports_bad_page():
     assert torch.isfinite(out.float()).all()
 
 
-def prefill_case(T, B, S, nq, nkv, dh, ps, starts, seed):
+def prefill_case(T, B, S, nq, nkv, dh, ps, starts, seed, climb=0.0, at=0):
     """Random paged cache holding starts[b] + S keys per sequence (slots past a sequence's last
     key hold NaN: they must never reach a result) + queries for the last S positions; the
     float64 result comes from oracle.attention, one sequence and track at a time."""
@@ -138,8 +164,13 @@ def prefill_case(T, B, S, nq, nkv, dh, ps, starts, seed):
         k = -(-n // ps)
         bt[b, :k] = perm[nxt:nxt + k]
         nxt += k
-    pool = I.round_to_bf16(rng.standard_normal((T, pages, 2, nkv, ps, dh), dtype=np.float32))
-    q = I.round_to_bf16(rng.standard_normal((T, B * S, nq * dh), dtype=np.float32))
+    pool = rng.standard_normal((T, pages, 2, nkv, ps, dh), dtype=np.float32)
+    q = rng.standard_normal((T, B * S, nq * dh), dtype=np.float32)
+    if climb:
+        for t in range(T):
+            for b, n in enumerate(lens):
+                _climbing_scores(rng, pool, q[t, b * S:(b + 1) * S].reshape(S, nq, dh), bt, b, t, n, nq, nkv, dh, ps, climb, at)
+    pool, q = I.round_to_bf16(pool), I.round_to_bf16(q)
     ref = np.zeros((T, B * S, nq * dh))
     valid = np.zeros((pages, ps), bool)
     for t in range(T):
@@ -164,15 +195,21 @@ PREFILL_CASES = [
     (1, 2, 700, 2, 2, 64, 32, [513, 0]),             # 32-token pages, several CTAs per sequence
     (2, 1, 1024, 2, 1, 128, 16, [0]),                # keys end exactly on a tile boundary
     (1, 2, 1, 2, 2, 128, 16, [130, 0]),              # single new token per sequence
+    (1, 1, 1024, 2, 1, 128, 16, [0], 40.0, 0),       # scores climbing by 2^40 along the keys: every row's maximum keeps rising, tile after tile
+    (1, 2, 512, 2, 2, 128, 16, [300, 0], 7.5, 200),  # the scores jump by 2^7.5 at key 200: below the threshold at which the tensor-core kernel raises its reference
+    (1, 2, 512, 4, 2, 128, 16, [0, 130], 9.0, 330),  # ... and above it, in mid-tile
+    (1, 1, 700, 2, 2, 64, 32, [513], 20.0, 0),       # a climb over earlier context, head_dim 64, 32-token pages
 ]
 
 
 @pytest.mark.parametrize("impl", [0, 1])
-@pytest.mark.parametrize("T,B,S,nq,nkv,dh,ps,starts", PREFILL_CASES)
-def test_prefill_attention_kernel_matches_oracle(T, B, S, nq, nkv, dh, ps, starts, impl):
+@pytest.mark.parametrize("case", PREFILL_CASES, ids=[f"S{c[2]}-dh{c[5]}-start{max(c[7])}" + (f"-climb{c[8]:g}" if len(c) > 8 else "") for c in PREFILL_CASES])
+def test_prefill_attention_kernel_matches_oracle(case, impl):
     import torch
     from paper_2602_07306_b200 import pt
-    q, pool, bt, lens, ref = prefill_case(T, B, S, nq, nkv, dh, ps, starts, seed=S + sum(starts))
+    T, B, S, nq, nkv, dh, ps, starts = case[:8]
+    climb, at = (case[8], case[9]) if len(case) > 8 else (0.0, 0)
+    q, pool, bt, lens, ref = prefill_case(T, B, S, nq, nkv, dh, ps, starts, seed=S + sum(starts), climb=climb, at=at)
     out, status = pt.kernel_prefill_attn(q, pool, bt, lens, S=S, nq=nq, nkv=nkv, dh=dh, ps=ps, impl=impl)
     torch.cuda.synchronize()
     assert status[:2].tolist() == [0, 0]

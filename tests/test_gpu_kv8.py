@@ -222,7 +222,8 @@ MANY = 80
     (2, MANY, 4, 2, 16, [384] * MANY, 5.0, 128, 0),             # the scores rise by 2^5 after the first tile and stay there: a reference
                                                                 # maximum that is not raised at once leaves probabilities of 32 for most keys
     (2, MANY, 4, 2, 16, [400 + 3 * i for i in range(MANY)], 7.5, 200, 3),   # the same with 2^7.5 in mid-tile, ragged lengths, growing V
-], ids=["random", "climb14", "climb6_v32", "climb30", "step5", "step7.5_v8"])
+    (1, 2, 4, 2, 16, [900, 300], 0.0, 0, 24),                   # V magnitudes from 1 to 2^24 along a sequence: scales far apart in one tile's product
+], ids=["random", "climb14", "climb6_v32", "climb30", "step5", "step7.5_v8", "v_2^24"])
 def test_e4m3_decode_attention_kernels_against_the_oracle(impl, T, B, nq, nkv, ps, lens, climb, at, vsteps):
     import torch
     from paper_2602_07306_b200 import pt
