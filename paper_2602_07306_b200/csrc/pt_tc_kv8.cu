@@ -230,25 +230,49 @@ k_decode_attn_e4m3(const __grid_constant__ CUtensorMap kvmap, const Dec8P pp) {
 
     const int g = lane >> 2, q4 = lane & 3;
     // q fragments: k-steps 2kk and 2kk+1 take head_dim 32 kk + 8 q + {0..3} and + {4..7}
+    // q is a bf16 vector of any magnitude and f16 is narrow: every head is divided by the power of two at its largest
+    // element (so that it lies in [1, 2)) before the conversion and the scores are multiplied by it afterwards.
     uint32_t qf[kDh / 16][4];
+    float q_unit = 1.0f;
     {
         const __nv_bfloat16* qrow = p.q + ((size_t)t * p.M + b) * (size_t)(p.nq * kDh) + (size_t)(kvh * G + g) * kDh;
+        uint4 raw[kDh / 32];
+        float amax = 0.f;
 #pragma unroll
         for (int kk = 0; kk < kDh / 32; ++kk) {
+            raw[kk] = g < G ? *reinterpret_cast<const uint4*>(qrow + kk * 32 + q4 * 8) : make_uint4(0, 0, 0, 0);
+            const uint32_t wds[4] = {raw[kk].x, raw[kk].y, raw[kk].z, raw[kk].w};
 #pragma unroll
-            for (int h = 0; h < 2; ++h) { qf[2 * kk + h][0] = qf[2 * kk + h][1] = qf[2 * kk + h][2] = qf[2 * kk + h][3] = 0u; }
-            if (g < G) {
-                const uint4 raw = *reinterpret_cast<const uint4*>(qrow + kk * 32 + q4 * 8);
-                const uint32_t wds[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const float2 f0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wds[2 * h]));
-                    const float2 f1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wds[2 * h + 1]));
-                    qf[2 * kk + h][0] = pack_half2(f0.x, f0.y);
-                    qf[2 * kk + h][2] = pack_half2(f1.x, f1.y);
-                }
+            for (int i = 0; i < 4; ++i) {
+                const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wds[i]));
+                amax = fmaxf(amax, fmaxf(fabsf(f.x), fabsf(f.y)));
             }
         }
+        amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+        amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+        float q_inv = 1.0f;
+        {
+            const int xf = (int)(__float_as_uint(amax) >> 23) & 0xff;
+            if (amax > 0.f && amax <= 3.0e38f) {
+                const int e = min(max(xf - 127, -100), 100);
+                q_unit = __uint_as_float((uint32_t)(e + 127) << 23);
+                q_inv = __uint_as_float((uint32_t)(127 - e) << 23);
+            }
+        }
+#pragma unroll
+        for (int kk = 0; kk < kDh / 32; ++kk) {
+            const uint32_t wds[4] = {raw[kk].x, raw[kk].y, raw[kk].z, raw[kk].w};
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const float2 f0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wds[2 * h]));
+                const float2 f1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wds[2 * h + 1]));
+                qf[2 * kk + h][0] = pack_half2(f0.x * q_inv, f0.y * q_inv);
+                qf[2 * kk + h][1] = 0u;
+                qf[2 * kk + h][2] = pack_half2(f1.x * q_inv, f1.y * q_inv);
+                qf[2 * kk + h][3] = 0u;
+            }
+        }
+        q_unit *= p.scale_log2;
     }
     // byte offsets inside a slot, fixed for the thread (the swizzle's XOR is folded in once):
     //   K: row g (+8 for the second n-tile), the 8 bytes at head_dim 32 kk + 8 q
@@ -263,7 +287,10 @@ k_decode_attn_e4m3(const __grid_constant__ CUtensorMap kvmap, const Dec8P pp) {
     float o[kDh / 8][4];
 #pragma unroll
     for (int i = 0; i < kDh / 8; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
-    float m_run = -INFINITY, l_run = 0.f;
+    // The V codes enter the MMA as they are (exact in f16); a key's V scale goes into its probability, relative to the
+    // largest V scale this warp has met (v_ref, a power of two; the accumulator is rescaled when it grows), so that
+    // neither large nor small magnitudes of V leave the f16 range.
+    float m_run = -INFINITY, l_run = 0.f, v_ref = 0.f;
 
 #pragma unroll
     for (int s = 0; s < kDecStages; ++s) { int gi = warp + 4 * s; if (gi < npages) issue(gi); else cp_async_commit(); }
@@ -308,8 +335,8 @@ k_decode_attn_e4m3(const __grid_constant__ CUtensorMap kvmap, const Dec8P pp) {
                 mma_f16(s[nt], qf[2 * kk + 1], b2, b3);
             }
         }
-        s[0][0] *= sk01.x * p.scale_log2; s[0][1] *= sk01.y * p.scale_log2;
-        s[1][0] *= sk89.x * p.scale_log2; s[1][1] *= sk89.y * p.scale_log2;
+        s[0][0] *= sk01.x * q_unit; s[0][1] *= sk01.y * q_unit;
+        s[1][0] *= sk89.x * q_unit; s[1][1] *= sk89.y * q_unit;
         if (nvalid < 16) {
             if (2 * q4 >= nvalid) { s[0][0] = -INFINITY; sv01.x = 0.f; }
             if (2 * q4 + 1 >= nvalid) { s[0][1] = -INFINITY; sv01.y = 0.f; }
@@ -325,14 +352,19 @@ k_decode_attn_e4m3(const __grid_constant__ CUtensorMap kvmap, const Dec8P pp) {
         s[0][0] = ex2f(s[0][0] - mn); s[0][1] = ex2f(s[0][1] - mn);
         s[1][0] = ex2f(s[1][0] - mn); s[1][1] = ex2f(s[1][1] - mn);
         l_run = l_run * corr + ((s[0][0] + s[0][1]) + (s[1][0] + s[1][1]));
-        if (__any_sync(0xffffffffu, corr != 1.f)) {
+        float vmax = fmaxf(fmaxf(sv01.x, sv01.y), fmaxf(sv89.x, sv89.y));     // over the group's 16 keys (the same in every row g)
+        vmax = fmaxf(vmax, __shfl_xor_sync(0xffffffffu, vmax, 1));
+        vmax = fmaxf(vmax, __shfl_xor_sync(0xffffffffu, vmax, 2));
+        float ocorr = corr;
+        if (vmax > v_ref) { ocorr *= v_ref / vmax; v_ref = vmax; }           // powers of two: exact (v_ref starts at 0)
+        if (__any_sync(0xffffffffu, ocorr != 1.f)) {
 #pragma unroll
-            for (int i = 0; i < kDh / 8; ++i) { o[i][0] *= corr; o[i][1] *= corr; }
+            for (int i = 0; i < kDh / 8; ++i) { o[i][0] *= ocorr; o[i][1] *= ocorr; }
         }
+        const float vinv = v_ref > 0.f ? 1.0f / v_ref : 0.f;
         uint32_t pf[4];
-        pf[0] = pack_half2(s[0][0], s[0][1]); pf[1] = 0u;
-        pf[2] = pack_half2(s[1][0], s[1][1]); pf[3] = 0u;
-        const uint32_t hs01 = pack_half2(sv01.x, sv01.y), hs89 = pack_half2(sv89.x, sv89.y);
+        pf[0] = pack_half2(s[0][0] * (sv01.x * vinv), s[0][1] * (sv01.y * vinv)); pf[1] = 0u;
+        pf[2] = pack_half2(s[1][0] * (sv89.x * vinv), s[1][1] * (sv89.y * vinv)); pf[3] = 0u;
 #pragma unroll
         for (int m = 0; m < kDh / 32; ++m) {
             uint32_t w0, w1, w2, w3;
@@ -347,11 +379,7 @@ k_decode_attn_e4m3(const __grid_constant__ CUtensorMap kvmap, const Dec8P pp) {
             codes4_to_half(a01, b0[0], b0[1]); codes4_to_half(a23, b0[2], b0[3]);
             codes4_to_half(c01, b1[0], b1[1]); codes4_to_half(c23, b1[2], b1[3]);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                asm("mul.rn.f16x2 %0, %0, %1;" : "+r"(b0[i]) : "r"(hs01));
-                asm("mul.rn.f16x2 %0, %0, %1;" : "+r"(b1[i]) : "r"(hs89));
-                mma_f16(o[m * 4 + i], pf, b0[i], b1[i]);
-            }
+            for (int i = 0; i < 4; ++i) mma_f16(o[m * 4 + i], pf, b0[i], b1[i]);
         }
         __syncwarp();                                         // every lane is done reading the slot
         {
@@ -384,7 +412,7 @@ k_decode_attn_e4m3(const __grid_constant__ CUtensorMap kvmap, const Dec8P pp) {
 #pragma unroll
         for (int nt = 0; nt < kDh / 8; ++nt) {
             const int d0 = 32 * (nt >> 2) + 8 * q4 + (nt & 3);
-            dst[d0] = o[nt][0]; dst[d0 + 4] = o[nt][1];
+            dst[d0] = o[nt][0] * v_ref; dst[d0 + 4] = o[nt][1] * v_ref;
         }
         if (q4 == 0) { dst[kDh] = m_run; dst[kDh + 1] = l_run; }
     }
