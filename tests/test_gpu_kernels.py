@@ -122,6 +122,8 @@ def decode_case(T, B, nq, nkv, dh, ps, lens, seed, climb=0.0, at=0):
     (1, 2, 8, 2, 128, 16, [2048, 700], 14.0, 0),              # scores climbing by 2^14 along the sequence: the running maximum rises in every tile
     (2, 80, 4, 2, 128, 16, [384] * 80, 7.5, 128),             # many sequences (one key range each): the scores jump by 2^7.5 after the first tile
     (1, 1, 4, 1, 64, 16, [3000], 60.0, 0),                    # a climb by 2^60: the early keys' weights underflow
+    (4, 80, 4, 4, 64, 16, [16 + (37 * i) % 380 for i in range(77)] + [1500, 1100, 900], 0, 0),   # enough (sequence, track, KV head)
+                                                              # triples to fill the machine: only the sequences far above the mean length are split
 ])
 def test_decode_attention_kernel_matches_oracle(T, B, nq, nkv, dh, ps, lens, climb, at):
     import torch

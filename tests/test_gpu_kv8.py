@@ -223,7 +223,9 @@ MANY = 80
                                                                 # maximum that is not raised at once leaves probabilities of 32 for most keys
     (2, MANY, 4, 2, 16, [400 + 3 * i for i in range(MANY)], 7.5, 200, 3),   # the same with 2^7.5 in mid-tile, ragged lengths, growing V
     (1, 2, 4, 2, 16, [900, 300], 0.0, 0, 24),                   # V magnitudes from 1 to 2^24 along a sequence: scales far apart in one tile's product
-], ids=["random", "climb14", "climb6_v32", "climb30", "step5", "step7.5_v8", "v_2^24"])
+    (4, MANY, 4, 4, 16, [16 + (37 * i) % 190 for i in range(MANY - 2)] + [1200, 900], 3.0, 0, 2),   # a full machine without splits:
+                                                                # only the two sequences far above the mean length get several key ranges
+], ids=["random", "climb14", "climb6_v32", "climb30", "step5", "step7.5_v8", "v_2^24", "full_machine"])
 def test_e4m3_decode_attention_kernels_against_the_oracle(impl, T, B, nq, nkv, ps, lens, climb, at, vsteps):
     import torch
     from paper_2602_07306_b200 import pt
