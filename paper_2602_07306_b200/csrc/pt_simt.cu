@@ -3,6 +3,7 @@
 // pt_config.flags bit 0, a slow cross-check of the bf16 tensor-core path.  The track index is
 // a grid dimension of every kernel.
 #include "pt_tc.h"
+#include "pt_ptx.cuh"
 
 namespace pt {
 
@@ -15,9 +16,6 @@ template <class E> __device__ __forceinline__ void stf(E* p, float v);
 template <> __device__ __forceinline__ void stf<float>(float* p, float v) { *p = v; }
 template <> __device__ __forceinline__ void stf<__nv_bfloat16>(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
 
-__device__ __forceinline__ void report(int* status, int code, int loc) {
-    if (atomicCAS(status, 0, code) == 0) status[1] = loc;
-}
 
 // ---- weight packing: rows of one [rows, cols] source matrix go to mapped rows of the packed matrix.
 // kind: PT_WQ/PT_WK/PT_WV -> rows offset inside [Nqkv, H]; PT_WG/PT_WU -> interleaved in groups

@@ -12,6 +12,7 @@
 //                    of one sequence are merged by k_decode_combine.
 // Softmax runs in base 2: scores are scaled by log2(e)/sqrt(head_dim) once.
 #include "pt_tc.h"
+#include "pt_ptx.cuh"
 
 namespace pt {
 
@@ -20,7 +21,6 @@ namespace {
 constexpr int kTileKeys = 64;
 constexpr int kThreads = 128;
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
     int sz = valid ? 16 : 0;                         // 0 source bytes: the 16 destination bytes are zero-filled
@@ -42,9 +42,6 @@ __device__ __forceinline__ void mma_bf16(float* c, const uint32_t* a, uint32_t b
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&v);
-}
-__device__ __forceinline__ void report(int* status, int code, int loc) {
-    if (atomicCAS(status, 0, code) == 0) status[1] = loc;
 }
 
 // Byte offset of 16-byte chunk `chunk` of row `row` in a [rows][DH] bf16 tile whose chunks are
@@ -294,22 +291,6 @@ __device__ __forceinline__ void decode_merge_store(const AttnP& p, float* mg, fl
 constexpr int kDecStages = 3;
 constexpr uint32_t kDecSpin = 1u << 24;
 
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2) {
-    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-                 ::"r"(dst), "l"((uint64_t)map), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar)) : "memory");
-}
 
 // Byte offset of 16-byte chunk `chunk` of row `row` (0..15) inside one page block as the tensor
 // map lays it out: 128-byte-wide halves of 16 rows each, chunks XOR-swizzled with row % 8.

@@ -10,6 +10,7 @@
 #include <cuda_fp8.h>
 
 #include "pt_tc.h"
+#include "pt_ptx.cuh"
 
 namespace pt {
 
@@ -17,10 +18,6 @@ namespace {
 
 constexpr int kDh = 128;                   // the format's kernels are written for head_dim 128
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void report(int* status, int code, int loc) {
-    if (atomicCAS(status, 0, code) == 0) status[1] = loc;
-}
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -138,18 +135,6 @@ constexpr uint32_t kDecSpin = 1u << 24;
 constexpr int kSlotBytes = 2 * 16 * kDh;                  // K box + V box
 constexpr int kDecThreads = 128;
 
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
 __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2, int c3, int c4) {
     asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
                  ::"r"(dst), "l"((uint64_t)map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(smem_u32(bar)) : "memory");
@@ -442,20 +427,10 @@ k_decode_attn_e4m3(const __grid_constant__ CUtensorMap kvmap, const Dec8P pp) {
     }
 }
 
-typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
 // (code byte, slot, (K|V, head), page, track): a box is the 16 x 128 code bytes of one 16-token group of a K block and,
 // through the element stride nkv of the third dimension, of the V block of the same head
 pt_status make_codes_map(CUtensorMap* out, const void* base, int ps, int nkv, int64_t pages, int64_t tracks, int64_t track_stride_bytes) {
-    static EncodeFn enc = nullptr;
-    if (!enc) {
-        void* f = nullptr;
-        cudaDriverEntryPointQueryResult qr;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qr) == cudaSuccess && qr == cudaDriverEntryPointSuccess)
-            enc = (EncodeFn)f;
-    }
+    EncodeFn enc = get_encode();
     if (!enc) { set_error("cuTensorMapEncodeTiled is not available from this driver"); return PT_ERR_CUDA; }
     if (nkv > 8) { set_error("an E4M3 cache supports up to 8 KV heads per track"); return PT_ERR_UNSUPPORTED; }
     cuuint64_t dims[5] = {(cuuint64_t)kDh, (cuuint64_t)ps, (cuuint64_t)(2 * nkv), (cuuint64_t)pages, (cuuint64_t)tracks};

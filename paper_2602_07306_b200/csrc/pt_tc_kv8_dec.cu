@@ -23,6 +23,7 @@
 #include <cuda_fp8.h>
 
 #include "pt_tc.h"
+#include "pt_ptx.cuh"
 
 namespace pt {
 
@@ -59,30 +60,7 @@ constexpr float kLazyLog2 = T8_LAZY_LOG2;
 enum { B_KFULL = 0, B_KEMPTY = 3, B_VFULL = 6, B_VEMPTY = 9, B_SFULL = 12, B_SEMPTY = 14, B_PFULL = 16, B_PEMPTY = 18,
        B_VRAW = 20, B_COUNT = 21 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-#ifndef T8_SUSPEND_NS
-#define T8_SUSPEND_NS 0
-#endif
-__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-#if T8_SUSPEND_NS > 0
-    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
-                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"((uint32_t)T8_SUSPEND_NS) : "memory");
-#else
-    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-#endif
-    return ok != 0;
-}
+// (A suspend-time hint on mbarrier.try_wait, 1 or 10 us, was measured: no gain.)
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, bool relaxed = false) {
     WaitClock clock;
     for (uint32_t i = 0; i < kSpin; ++i) {
@@ -91,15 +69,6 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
         if ((i & 255) == 255 && (*abort_flag || clock.expired())) return false;
     }
     return false;
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2) {
-    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-                 ::"r"(dst), "l"((uint64_t)map), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint64_t* bar) {
-    asm volatile("{\n .reg .pred e;\n elect.sync _|e, 0xffffffff;\n @e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}" ::"r"(smem_u32(bar)) : "memory");
 }
 // D[tmem] (+)= A[smem] * B[smem], both operands E4M3
 __device__ __forceinline__ void mma_f8(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
@@ -132,9 +101,6 @@ __device__ __forceinline__ float ex2f(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
-}
-__device__ __forceinline__ void report(int* status, int code, int loc) {
-    if (atomicCAS(status, 0, code) == 0) status[1] = loc;
 }
 // float <-> an integer with the same order (so that redux.sync.max can reduce floats, -inf included)
 __device__ __forceinline__ int f2ord(float x) { int i = __float_as_int(x); return i ^ ((i >> 31) & 0x7fffffff); }
@@ -532,19 +498,9 @@ k_decode_attn_e4m3_tc(const __grid_constant__ CUtensorMap kvmap, const Dec8TcP p
     }
 }
 
-typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
 // (code byte, vector of a slab, track) with boxes of 16 vectors x 128 bytes in the 128-byte swizzle
 pt_status make_codes_map3(CUtensorMap* out, const void* base, int64_t vecs, int64_t tracks, int64_t track_stride_bytes) {
-    static EncodeFn enc = nullptr;
-    if (!enc) {
-        void* f = nullptr;
-        cudaDriverEntryPointQueryResult qr;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qr) == cudaSuccess && qr == cudaDriverEntryPointSuccess)
-            enc = (EncodeFn)f;
-    }
+    EncodeFn enc = get_encode();
     if (!enc) { set_error("cuTensorMapEncodeTiled is not available from this driver"); return PT_ERR_CUDA; }
     cuuint64_t dims[3] = {(cuuint64_t)kDh, (cuuint64_t)vecs, (cuuint64_t)tracks};
     cuuint64_t strides[2] = {(cuuint64_t)kDh, (cuuint64_t)track_stride_bytes};
