@@ -33,24 +33,26 @@ from paper_2602_07306_b200 import inputs as I  # noqa: E402
 # DRAM traffic of k_decode_attn_tma<128> from its ncu capture (profiles/decode_attn_tma_T8_B8_kv2049.md:
 # 8 sequences instead of 64, same kernel): dram read + write bytes per launch over the algorithmic K/V
 # bytes of that launch.  Traffic is proportional to the keys read, so a bench launch is scaled by its own
-# algorithmic bytes.  The counters belong to one version of the kernel's source file: its SHA-256 is kept
-# beside them, and when the file on disk differs the bench reports "traffic": null with the reason.
-DECODE_ATTN_TRAFFIC_RATIO = (541.27e6 + 4.17e6) / 537.13e6
-DECODE_ATTN_TRAFFIC_SOURCE = ("paper_2602_07306_b200/csrc/pt_tc_attn.cu",
-                              "5bf3ceba9ea530561f04d6d02805ec0201dd52d4c12a143183839cd5f3c53fe1")
+# algorithmic bytes.  The counters belong to one version of the kernel's source files: their SHA-256 is kept
+# beside them, and when the files on disk differ the bench reports "traffic": null with the reason.
+DECODE_ATTN_TRAFFIC_RATIO = (541.24e6 + 4.00e6) / 537.13e6
+DECODE_ATTN_TRAFFIC_SOURCE = (("paper_2602_07306_b200/csrc/pt_tc_attn.cu", "paper_2602_07306_b200/csrc/pt_ptx.cuh"),
+                              "58ea08e5b2a28ea033c2102a8313e6851f5d5a19e263cc48595495108d95f25c")
 
 
 def decode_attn_traffic_ratio():
-    """(ratio, None) while the kernel source is the one the counters were taken on, else (None, reason)."""
+    """(ratio, None) while the kernel's sources are the ones the counters were taken on, else (None, reason)."""
     import hashlib
-    path, want = DECODE_ATTN_TRAFFIC_SOURCE
+    paths, want = DECODE_ATTN_TRAFFIC_SOURCE
+    h = hashlib.sha256()
     try:
-        with open(os.path.join(ROOT, path), "rb") as f:
-            have = hashlib.sha256(f.read()).hexdigest()
+        for path in paths:
+            with open(os.path.join(ROOT, path), "rb") as f:
+                h.update(f.read())
     except OSError as e:
         return None, f"kernel source not readable: {e}"
-    if have != want:
-        return None, f"{path} changed since the ncu counters were taken"
+    if h.hexdigest() != want:
+        return None, f"{' or '.join(paths)} changed since the ncu counters were taken"
     return DECODE_ATTN_TRAFFIC_RATIO, None
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
