@@ -178,3 +178,34 @@ def test_bf16_decode_track_sync_on_both_sides_of_256_rows(B):
     every layer."""
     wl = small("bf16", T=3, L=2, D=1, H=128, nq=2, nkv=1, F=176)
     run_case(wl, B=B, S=2, decode_steps=2, check_pool=False)
+
+
+@pytest.mark.parametrize("kv_dtype", ["model", "e4m3"])
+def test_bf16_forward_is_reproducible_bit_for_bit(kv_dtype):
+    """The same chunked prefill and decode steps on two fresh caches give the same bits: outputs and cache pools.
+    (Every reduction of the path has a fixed order: k-blocks in a GEMM, tracks in the sync, key ranges in the merge.)"""
+    import torch
+    wl = I.Workload("repro", T=2, L=4, D=2, hidden=512, heads=4, kv_heads=1, ffn=352, dtype="bf16", mode="prefill",
+                    batch=3, seq=300, seed=0)
+    ws = I.WeightSource(wl, gain_jitter=0.1)
+    B, S, ps = 3, 300, 16
+    total = S + 3
+    pages = B * (-(-total // ps)) + 2
+    order = I.free_list_permutation(pages, seed=5)
+    seq_ids = [1, 4, 9]
+    model = Hp.make_model(wl, ws, max_pos=512)
+    x = Hp.to_dev(model, I.prefill_inputs(wl, batch=B, seq=S))
+    xd = [Hp.to_dev(model, I.decode_inputs(wl, batch=B, step=i)) for i in range(3)]
+    runs = []
+    for _ in range(2):
+        cache = model.new_cache(pages, ps, order, kv_dtype=kv_dtype)
+        cache.pool.zero_()
+        outs = [model.prefill(cache, x[:, :, :200].contiguous(), seq_ids).clone(), model.prefill(cache, x[:, :, 200:].contiguous(), seq_ids).clone()]
+        outs += [model.decode_step(cache, xi, seq_ids).clone() for xi in xd]
+        torch.cuda.synchronize()
+        assert model.device_status() == (0, 0)
+        runs.append((outs, cache.pool.clone()))
+    for a, b in zip(runs[0][0], runs[1][0]):
+        assert torch.equal(a, b)
+    assert torch.equal(runs[0][1], runs[1][1])
+    model.close()
