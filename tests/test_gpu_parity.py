@@ -182,8 +182,9 @@ def test_bf16_decode_track_sync_on_both_sides_of_256_rows(B):
 
 @pytest.mark.parametrize("kv_dtype", ["model", "e4m3"])
 def test_bf16_forward_is_reproducible_bit_for_bit(kv_dtype):
-    """The same chunked prefill and decode steps on two fresh caches give the same bits: outputs and cache pools.
-    (Every reduction of the path has a fixed order: k-blocks in a GEMM, tracks in the sync, key ranges in the merge.)"""
+    """The same chunked prefill and decode steps on two fresh caches give the same bits: outputs and cache pools
+    (every reduction of the path has a fixed order: k-blocks in a GEMM, tracks in the sync, key ranges in the merge);
+    and a third cache that hands out its pages in another order gives the same outputs from a different pool."""
     import torch
     wl = I.Workload("repro", T=2, L=4, D=2, hidden=512, heads=4, kv_heads=1, ffn=352, dtype="bf16", mode="prefill",
                     batch=3, seq=300, seed=0)
@@ -197,8 +198,8 @@ def test_bf16_forward_is_reproducible_bit_for_bit(kv_dtype):
     x = Hp.to_dev(model, I.prefill_inputs(wl, batch=B, seq=S))
     xd = [Hp.to_dev(model, I.decode_inputs(wl, batch=B, step=i)) for i in range(3)]
     runs = []
-    for _ in range(2):
-        cache = model.new_cache(pages, ps, order, kv_dtype=kv_dtype)
+    for free_order in (order, order, I.free_list_permutation(pages, seed=6)):
+        cache = model.new_cache(pages, ps, free_order, kv_dtype=kv_dtype)
         cache.pool.zero_()
         outs = [model.prefill(cache, x[:, :, :200].contiguous(), seq_ids).clone(), model.prefill(cache, x[:, :, 200:].contiguous(), seq_ids).clone()]
         outs += [model.decode_step(cache, xi, seq_ids).clone() for xi in xd]
@@ -208,4 +209,7 @@ def test_bf16_forward_is_reproducible_bit_for_bit(kv_dtype):
     for a, b in zip(runs[0][0], runs[1][0]):
         assert torch.equal(a, b)
     assert torch.equal(runs[0][1], runs[1][1])
+    for a, b in zip(runs[0][0], runs[2][0]):              # other pages for the same tokens: the same bits come out
+        assert torch.equal(a, b)
+    assert not torch.equal(runs[0][1], runs[2][1])
     model.close()
